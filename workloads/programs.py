@@ -1,0 +1,249 @@
+"""Combinator programs as plain records.
+
+A program is an ordered list of nodes; a node may only name earlier nodes as
+inputs, so every list is a DAG in topological order.  Slot layout by kind:
+
+  input        no slots (bound by the caller)
+  generate     [free...]                       n_array = 0
+  map          [xs, free...]                   n_array = 1
+  zipwith      [xs1..xsk, free...]             n_array = k (2..5)
+  backpermute  [src]                           index map named by idx_fn
+  gather       [idx, src]                      idx holds row-major linear indices
+  permute      [defaults, idx, vals]           combine op named by fn
+  fold         [src]                           reduces the innermost extent
+  scanl/scanr  [src]                           inclusive, per innermost row
+
+Slots at positions >= n_array are "free variable" reads (element-level
+indexing, always of element 0 here).  Function names are interpreted by each
+executor's own table; this file only spells them.
+"""
+from dataclasses import dataclass, field
+from typing import List, Tuple
+
+
+@dataclass
+class Node:
+    kind: str
+    dtype: str                      # 'f32' | 'i32' | 'u32'
+    shape: Tuple[int, ...]          # () for the scalar result of a rank-1 fold
+    inputs: Tuple[int, ...] = ()
+    n_array: int = 0
+    fn: str = ""
+    idx_fn: str = ""
+    iparam: Tuple[int, ...] = ()
+    fparam: Tuple[float, ...] = ()
+    force: Tuple[int, ...] = ()     # slots whose read is wrapped in force()
+    name: str = ""
+
+
+@dataclass
+class Program:
+    name: str
+    nodes: List[Node]
+    outputs: List[int]
+    names: dict = field(default_factory=dict)
+    index_bound: dict = field(default_factory=dict)   # exclusive bound of index-valued inputs
+
+    def __post_init__(self):
+        self.names = {nd.name: i for i, nd in enumerate(self.nodes) if nd.name}
+
+    def id(self, name):
+        return self.names[name]
+
+    def input_ids(self):
+        return [i for i, nd in enumerate(self.nodes) if nd.kind == "input"]
+
+
+def _inp(name, dtype, shape):
+    return Node("input", dtype, tuple(shape), name=name)
+
+
+# --------------------------------------------------------------------------
+# The five benchmark configurations
+# --------------------------------------------------------------------------
+
+def config1(n=1 << 16):
+    """1-D chain: y=map(2x+1) x; z=backpermute(reverse) y; w=zipWith(*) z x; s=fold(+) w."""
+    nodes = [
+        _inp("x", "f32", (n,)),
+        Node("map", "f32", (n,), (0,), 1, fn="affine", fparam=(2.0, 1.0), name="y"),
+        Node("backpermute", "f32", (n,), (1,), 1, idx_fn="reverse", name="z"),
+        Node("zipwith", "f32", (n,), (2, 0), 2, fn="mul", name="w"),
+        Node("fold", "f32", (), (3,), 1, fn="add", name="s"),
+    ]
+    return Program("config1", nodes, [4])
+
+
+def config2(rows=8192):
+    """2-D transpose-fuse-reduce: B=transpose A; C=A*B+0.5; rowsum=fold(+) C."""
+    sh = (rows, rows)
+    nodes = [
+        _inp("A", "f32", sh),
+        Node("backpermute", "f32", sh, (0,), 1, idx_fn="transpose", name="B"),
+        Node("zipwith", "f32", sh, (0, 1), 2, fn="mul_add_const", fparam=(0.5,), name="C"),
+        Node("fold", "f32", (rows,), (2,), 1, fn="add", name="rowsum"),
+    ]
+    return Program("config2", nodes, [3])
+
+
+def config3(n=1 << 26):
+    """Random gather + scan on int32: g=hash x; h=gather idx g; o=h&0xFFFF; out=scanl(+) o."""
+    nodes = [
+        _inp("x", "i32", (n,)),
+        _inp("idx", "i32", (n,)),
+        Node("map", "i32", (n,), (0,), 1, fn="hash_mul_xorshift", iparam=(2654435761, 13), name="g"),
+        Node("gather", "i32", (n,), (1, 2), 2, name="h"),
+        Node("map", "i32", (n,), (3,), 1, fn="and_mask", iparam=(0xFFFF,), name="o"),
+        Node("scanl", "i32", (n,), (4,), 1, fn="add", name="out"),
+    ]
+    return Program("config3", nodes, [5])
+
+
+def config4(rows=8192, cols=None, iters=4):
+    """Jacobi by horizontal fusion: per iteration five clamped shifts and four zipWiths."""
+    cols = rows if cols is None else cols
+    sh = (rows, cols)
+    nodes = [_inp("X", "f32", sh)]
+    prev = 0
+    for t in range(iters):
+        base = len(nodes)
+        shifts = [("c", 0, 0), ("n", -1, 0), ("s", 1, 0), ("e", 0, 1), ("w", 0, -1)]
+        for tag, dr, dc in shifts:
+            nodes.append(Node("backpermute", "f32", sh, (prev,), 1, idx_fn="shift_clamp",
+                              iparam=(dr, dc), name=f"{tag}{t}"))
+        c, n_, s, e, w = range(base, base + 5)
+        nodes.append(Node("zipwith", "f32", sh, (c, n_), 2, fn="add", name=f"t1_{t}"))
+        nodes.append(Node("zipwith", "f32", sh, (base + 5, s), 2, fn="add", name=f"t2_{t}"))
+        nodes.append(Node("zipwith", "f32", sh, (base + 6, e), 2, fn="add", name=f"t3_{t}"))
+        nodes.append(Node("zipwith", "f32", sh, (base + 7, w), 2, fn="add_scale",
+                          fparam=(0.2,), name=f"Y{t}"))
+        prev = base + 8
+    return Program("config4", nodes, [prev])
+
+
+def config5(n=1 << 27, bins=1 << 16):
+    """Scatter histogram + diamond: k=hash16 keys; vals=generate; hist=permute(+); total=fold; frac."""
+    nodes = [
+        _inp("keys", "u32", (n,)),
+        _inp("zeros", "f32", (bins,)),
+        Node("map", "u32", (n,), (0,), 1, fn="mul_mod", iparam=(40503, bins), name="k"),
+        Node("generate", "f32", (n,), (), 0, fn="imod_to_f32", iparam=(7,), name="vals"),
+        Node("permute", "f32", (bins,), (1, 2, 3), 3, fn="add", name="hist"),
+        Node("fold", "f32", (), (3,), 1, fn="add", name="total"),
+        Node("map", "f32", (bins,), (4, 5), 1, fn="div_free", name="frac"),
+    ]
+    return Program("config5", nodes, [6, 4, 5])
+
+
+# --------------------------------------------------------------------------
+# Programs the paper prints (Sections 1, 3.3, 3.4 and 5), as fixtures
+# --------------------------------------------------------------------------
+
+def single_loop(n=64):
+    """Section 1 `singleLoop`: reverse + two maps + zipWith3, fusible into one loop."""
+    nodes = [
+        _inp("as", "f32", (n,)),
+        Node("backpermute", "f32", (n,), (0,), 1, idx_fn="reverse", name="bs"),
+        Node("map", "f32", (n,), (0,), 1, fn="affine", fparam=(3.0, -1.0), name="cs"),
+        Node("map", "f32", (n,), (2,), 1, fn="affine", fparam=(0.5, 2.0), name="ds"),
+        Node("zipwith", "f32", (n,), (1, 2, 3), 3, fn="add3", name="result"),
+    ]
+    return Program("single_loop", nodes, [4])
+
+
+def simple1(n_is=40, n_xs=24):
+    nodes = [
+        _inp("is", "i32", (n_is,)), _inp("xs", "f32", (n_xs,)),
+        Node("map", "f32", (n_xs,), (1,), 1, fn="affine", fparam=(2.0, 1.0), name="as"),
+        Node("gather", "f32", (n_is,), (0, 2), 2, name="bs"),
+    ]
+    return Program("simple1", nodes, [3], index_bound={"is": n_xs})
+
+
+def simple2(n_is2=50, n_is1=30, n_xs=20):
+    nodes = [
+        _inp("is1", "i32", (n_is1,)), _inp("is2", "i32", (n_is2,)), _inp("xs", "f32", (n_xs,)),
+        Node("gather", "f32", (n_is1,), (0, 2), 2, name="as"),
+        Node("gather", "f32", (n_is2,), (1, 3), 2, name="bs"),
+    ]
+    return Program("simple2", nodes, [4], index_bound={"is1": n_xs, "is2": n_is1})
+
+
+def simple3(n_is=40, n_xs=24):
+    p = simple1(n_is, n_xs)
+    return Program("simple3", p.nodes, [2, 3], index_bound=p.index_bound)
+
+
+def simple4(n_is=20, m=12, n=7):
+    nodes = [
+        _inp("is", "i32", (n_is,)), _inp("xs", "f32", (m, n)),
+        Node("fold", "f32", (m,), (1,), 1, fn="add", name="as"),
+        Node("gather", "f32", (n_is,), (0, 2), 2, name="bs"),
+    ]
+    return Program("simple4", nodes, [3], index_bound={"is": m})
+
+
+def simple5(n=32):
+    nodes = [
+        _inp("is", "i32", (n,)), _inp("xs", "f32", (n,)),
+        Node("map", "f32", (n,), (1,), 1, fn="affine", fparam=(-1.5, 0.25), name="as"),
+        Node("gather", "f32", (n,), (0, 1), 2, name="bs"),
+        Node("zipwith", "f32", (n,), (2, 3), 2, fn="mul", name="cs"),
+    ]
+    return Program("simple5", nodes, [4], index_bound={"is": n})
+
+
+def scatter_example(n=48):
+    """Section 3.4 `scatterExample` after the structure-of-arrays split of `as`.
+
+    xs holds integers in [0, n/2) so that every index 2*x lands inside bs.
+    """
+    nodes = [
+        _inp("xs", "i32", (n,)),
+        Node("map", "i32", (n,), (0,), 1, fn="mul_const", iparam=(2,), name="as_i"),
+        Node("map", "i32", (n,), (0,), 1, fn="identity", name="as_v"),
+        Node("map", "i32", (n,), (0,), 1, fn="add_const", iparam=(1,), name="bs"),
+        Node("permute", "i32", (n,), (3, 1, 2), 3, fn="add", name="result"),
+    ]
+    return Program("scatter_example", nodes, [4], index_bound={"xs": n // 2})
+
+
+def scatter_example_paper_graph():
+    """The literal four-node graph of Section 4.1: `as` is one node feeding both
+    element slots of the scatter.  Only its structure is meaningful."""
+    nodes = [
+        _inp("xs", "i32", (8,)),
+        Node("map", "i32", (8,), (0,), 1, fn="identity", name="as"),
+        Node("map", "i32", (8,), (0,), 1, fn="add_const", iparam=(1,), name="bs"),
+        Node("permute", "i32", (8,), (2, 1, 1), 3, fn="add", name="result"),
+    ]
+    return Program("scatter_example_paper_graph", nodes, [3])
+
+
+def greedy_bottom_up_bad(n=16, m=1000):
+    """Section 5: a gathered rank-2 array that contracts only if both folds share its cluster."""
+    nodes = [
+        _inp("xs", "f32", (n,)),
+        Node("generate", "i32", (n, m), (), 0, fn="row_index", name="is"),
+        Node("gather", "f32", (n, m), (1, 0), 2, name="large"),
+        Node("fold", "f32", (n,), (2,), 1, fn="add", name="ys"),
+        Node("fold", "f32", (n,), (2,), 1, fn="mul", name="zs"),
+        Node("map", "f32", (n,), (3, 4), 1, fn="add_free", name="result"),
+    ]
+    return Program("greedy_bottom_up_bad", nodes, [5])
+
+
+def greedy_top_down_bad(n=4096):
+    """Section 5: greedy top-down fuses cs diagonally with bs; the optimum fuses cs into es."""
+    nodes = [
+        _inp("as", "f32", (n,)),
+        Node("map", "f32", (n,), (0,), 1, fn="affine", fparam=(2.0, 0.0), name="bs"),
+        Node("map", "f32", (n,), (1,), 1, fn="affine", fparam=(1.0, 1.0), name="cs"),
+        Node("generate", "f32", (n,), (1,), 0, fn="iota_plus_free", name="ds"),
+        Node("zipwith", "f32", (n,), (2, 3), 2, fn="add", name="es"),
+        Node("fold", "f32", (), (4,), 1, fn="add", name="result"),
+    ]
+    return Program("greedy_top_down_bad", nodes, [5])
+
+
+CONFIGS = {1: config1, 2: config2, 3: config3, 4: config4, 5: config5}
