@@ -1,0 +1,248 @@
+// extern "C" entry points declared in acc.h.
+#include <cstring>
+#include <map>
+#include <memory>
+
+#include "acc.h"
+#include "exec.h"
+#include "graph.h"
+
+using namespace acc;
+
+namespace {
+
+// Schedules are rebuilt only when the graph, its clustering or its bindings change.
+struct Cache {
+  uint32_t serial = ~0u;
+  Schedule sch;
+};
+std::map<const acc_graph*, std::unique_ptr<Cache[]>>& caches() {
+  static std::map<const acc_graph*, std::unique_ptr<Cache[]>> c;
+  return c;
+}
+
+int schedule_for(acc_graph* g, int executor, Schedule** out) {
+  if (executor != ACC_EXEC_FUSED && executor != ACC_EXEC_UNFUSED) return set_error(ACC_ERR_ARG, "unknown executor %d", executor);
+  auto& slot = caches()[g];
+  if (!slot) slot.reset(new Cache[2]);
+  Cache& c = slot[executor];
+  if (c.serial != g->run_serial) {
+    const int rc = build_schedule(*g, executor, c.sch);
+    if (rc != ACC_OK) return rc;
+    c.serial = g->run_serial;
+  }
+  *out = &c.sch;
+  return ACC_OK;
+}
+
+bool bad_node(const acc_graph* g, acc_node n) { return n < 0 || n >= (acc_node)g->nodes.size(); }
+
+}  // namespace
+
+extern "C" {
+
+int acc_graph_create(acc_graph** out) {
+  clear_error();
+  if (!out) return set_error(ACC_ERR_ARG, "out is null");
+  *out = new acc_graph();
+  return ACC_OK;
+}
+
+int acc_graph_destroy(acc_graph* g) {
+  clear_error();
+  if (!g) return set_error(ACC_ERR_ARG, "graph is null");
+  caches().erase(g);
+  delete g;
+  return ACC_OK;
+}
+
+acc_node acc_add_node(acc_graph* g, const acc_node_desc* d) {
+  clear_error();
+  if (!g || !d) return set_error(ACC_ERR_ARG, "null argument");
+  g->run_serial++;
+  return add_node(*g, *d);
+}
+
+int acc_mark_output(acc_graph* g, acc_node n) {
+  clear_error();
+  if (!g || bad_node(g, n)) return set_error(ACC_ERR_ARG, "bad node id");
+  if (is_input(g->nodes[n])) return set_error(ACC_ERR_ARG, "an input cannot be an output");
+  g->nodes[n].output = true;
+  g->has_pi = false;
+  g->run_serial++;
+  return ACC_OK;
+}
+
+int32_t acc_node_count(const acc_graph* g) { return g ? (int32_t)g->nodes.size() : ACC_ERR_ARG; }
+
+int acc_edges(const acc_graph* g, int32_t* F, int32_t* nF, int32_t* I, int32_t* nI, int32_t cap) {
+  clear_error();
+  if (!g || !nF || !nI) return set_error(ACC_ERR_ARG, "null argument");
+  int f = 0, i = 0;
+  for (const Edge& e : g->edges) {
+    int32_t* dst = e.fusible ? F : I;
+    int& k = e.fusible ? f : i;
+    if (dst && k < cap) { dst[2 * k] = e.a; dst[2 * k + 1] = e.b; }
+    ++k;
+  }
+  *nF = f;
+  *nI = i;
+  return ACC_OK;
+}
+
+int acc_check_partition(acc_graph* g, const int32_t* pi, int32_t n_nodes) {
+  clear_error();
+  if (!g || !pi) return set_error(ACC_ERR_ARG, "null argument");
+  if (n_nodes != (int32_t)g->nodes.size()) return set_error(ACC_ERR_ARG, "clustering has %d entries, graph has %zu nodes", n_nodes, g->nodes.size());
+  for (int i = 0; i < n_nodes; ++i)
+    if (!is_input(g->nodes[i]) && (pi[i] < 0 || pi[i] > n_nodes)) return set_error(ACC_ERR_ARG, "cluster number %d of node %d outside 0..n", pi[i], i);
+  return check_partition(*g, pi, nullptr);
+}
+
+int acc_set_partition(acc_graph* g, const int32_t* pi, int32_t n_nodes) {
+  const int rc = acc_check_partition(g, pi, n_nodes);
+  if (rc != ACC_OK) return rc;
+  g->pi.assign(pi, pi + n_nodes);
+  for (int i = 0; i < n_nodes; ++i)
+    if (is_input(g->nodes[i])) g->pi[i] = -1;
+  manifest_of(*g, g->pi.data(), g->manifest);
+  g->has_pi = true;
+  g->run_serial++;
+  return ACC_OK;
+}
+
+int acc_get_partition(const acc_graph* g, int32_t* out, int32_t n_nodes) {
+  clear_error();
+  if (!g || !out || n_nodes != (int32_t)g->nodes.size()) return set_error(ACC_ERR_ARG, "bad argument");
+  if (!g->has_pi) return set_error(ACC_ERR_NO_PARTITION, "no clustering set");
+  memcpy(out, g->pi.data(), sizeof(int32_t) * n_nodes);
+  return ACC_OK;
+}
+
+int acc_manifest(const acc_graph* g, int32_t* out, int32_t n_nodes) {
+  clear_error();
+  if (!g || !out || n_nodes != (int32_t)g->nodes.size()) return set_error(ACC_ERR_ARG, "bad argument");
+  if (!g->has_pi) return set_error(ACC_ERR_NO_PARTITION, "no clustering set");
+  for (int i = 0; i < n_nodes; ++i) out[i] = g->manifest[i];
+  return ACC_OK;
+}
+
+int acc_plan(acc_graph* g, int mode, int cost, int32_t* out) {
+  clear_error();
+  if (!g) return set_error(ACC_ERR_ARG, "graph is null");
+  std::vector<int32_t> pi;
+  const int rc = plan(*g, mode, cost, pi);
+  if (rc != ACC_OK) return rc;
+  if (out) memcpy(out, pi.data(), sizeof(int32_t) * pi.size());
+  return acc_set_partition(g, pi.data(), (int32_t)pi.size());
+}
+
+int64_t acc_enumerate(acc_graph* g, int32_t* out_pi, int64_t max_partitions) {
+  clear_error();
+  if (!g) return set_error(ACC_ERR_ARG, "graph is null");
+  std::vector<std::vector<int32_t>> all;
+  const int64_t cnt = enumerate_all(*g, all);
+  if (cnt < 0) return cnt;
+  const size_t n = g->nodes.size();
+  if (out_pi)
+    for (int64_t i = 0; i < cnt && i < max_partitions; ++i) memcpy(out_pi + i * n, all[i].data(), sizeof(int32_t) * n);
+  return cnt;
+}
+
+int acc_partition_cost(acc_graph* g, const int32_t* pi, int32_t n_nodes, int cost, double* out) {
+  clear_error();
+  if (!g || !pi || !out || n_nodes != (int32_t)g->nodes.size()) return set_error(ACC_ERR_ARG, "bad argument");
+  return partition_cost(*g, pi, cost, out);
+}
+
+int acc_bind(acc_graph* g, acc_node n, void* device_ptr, size_t bytes) {
+  clear_error();
+  if (!g || bad_node(g, n)) return set_error(ACC_ERR_ARG, "bad node id");
+  Node& nd = g->nodes[n];
+  if (bytes < (size_t)nd.count * 4) return set_error(ACC_ERR_UNBOUND, "node %d needs %zu bytes, buffer has %zu", n, (size_t)nd.count * 4, bytes);
+  if (!device_ptr && nd.count > 0) return set_error(ACC_ERR_ARG, "device pointer is null");
+  if (reinterpret_cast<uintptr_t>(device_ptr) & 15) return set_error(ACC_ERR_ARG, "device pointer is not 16-byte aligned");
+  nd.dev = device_ptr;
+  nd.dev_bytes = bytes;
+  g->run_serial++;
+  return ACC_OK;
+}
+
+int acc_bind_host(acc_graph* g, acc_node n, void* host_ptr, size_t bytes) {
+  clear_error();
+  if (!g || bad_node(g, n)) return set_error(ACC_ERR_ARG, "bad node id");
+  Node& nd = g->nodes[n];
+  if (!is_input(nd) && !nd.output) return set_error(ACC_ERR_ARG, "node %d is neither an input nor a marked output", n);
+  if (bytes < (size_t)nd.count * 4 || (!host_ptr && nd.count > 0)) return set_error(ACC_ERR_UNBOUND, "host buffer of node %d is null or too small", n);
+  nd.host = host_ptr;
+  nd.host_bytes = bytes;
+  return ACC_OK;
+}
+
+int acc_workspace_bytes(acc_graph* g, int executor, size_t* bytes) {
+  clear_error();
+  if (!g || !bytes) return set_error(ACC_ERR_ARG, "null argument");
+  Schedule* sch = nullptr;
+  const int rc = schedule_for(g, executor, &sch);
+  if (rc != ACC_OK) return rc;
+  *bytes = sch->total_bytes;
+  return ACC_OK;
+}
+
+int acc_run(acc_graph* g, void* workspace, size_t workspace_bytes, void* cuda_stream, int executor) {
+  clear_error();
+  if (!g) return set_error(ACC_ERR_ARG, "graph is null");
+  Schedule* sch = nullptr;
+  const int rc = schedule_for(g, executor, &sch);
+  if (rc != ACC_OK) return rc;
+  return run_schedule(*g, *sch, workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int acc_finish(acc_graph* g, void* workspace, void* cuda_stream) {
+  clear_error();
+  if (!g) return set_error(ACC_ERR_ARG, "graph is null");
+  return finish(*g, workspace, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int acc_run_e2e(acc_graph* g, void* workspace, size_t workspace_bytes, void* cuda_stream, int executor,
+                size_t* h2d_bytes, size_t* d2h_bytes) {
+  clear_error();
+  if (!g) return set_error(ACC_ERR_ARG, "graph is null");
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  size_t up = 0, down = 0;
+  for (Node& nd : g->nodes)
+    if (is_input(nd) && nd.host) {
+      if (!nd.dev) return set_error(ACC_ERR_UNBOUND, "a host-bound input has no device buffer");
+      const size_t b = (size_t)nd.count * 4;
+      if (b && cudaMemcpyAsync(nd.dev, nd.host, b, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return set_error(ACC_ERR_CUDA, "host-to-device copy failed: %s", cudaGetErrorString(cudaGetLastError()));
+      up += b;
+    }
+  const int rc = acc_run(g, workspace, workspace_bytes, cuda_stream, executor);
+  if (rc != ACC_OK) return rc;
+  for (Node& nd : g->nodes)
+    if (nd.output && nd.host) {
+      const size_t b = (size_t)nd.count * 4;
+      if (b && cudaMemcpyAsync(nd.host, nd.dev, b, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return set_error(ACC_ERR_CUDA, "device-to-host copy failed: %s", cudaGetErrorString(cudaGetLastError()));
+      down += b;
+    }
+  if (h2d_bytes) *h2d_bytes = up;
+  if (d2h_bytes) *d2h_bytes = down;
+  return finish(*g, workspace, stream);
+}
+
+int32_t acc_launch_count(const acc_graph* g) { return g ? g->launches : ACC_ERR_ARG; }
+
+int acc_last_schedule(const acc_graph* g, char* buf, size_t cap) {
+  if (!g || !buf || !cap) return ACC_ERR_ARG;
+  strncpy(buf, g->schedule.c_str(), cap - 1);
+  buf[cap - 1] = 0;
+  return ACC_OK;
+}
+
+const char* acc_last_error(void) { return last_error(); }
+
+int32_t acc_registry_size(void) { return registry_size(); }
+
+}  // extern "C"

@@ -1,0 +1,149 @@
+// Host-side launcher of a cluster instantiation: picks the skeleton from the cluster's
+// roots, the vector width from the shapes, sizes the grid to the machine and the scratch
+// region to the grid.
+#pragma once
+#include <algorithm>
+
+#include "../graph.h"
+#include "../registry.h"
+#include "skeletons.cuh"
+
+namespace acc {
+
+template <class CL>
+struct Launcher {
+  static constexpr int N = CL::c.n;
+  static constexpr bool kHasScan = dev::count_if<CL>(dev::is_scan_root) > 0;
+  static constexpr bool kHasRowFold = dev::count_if<CL>(dev::is_row_fold) > 0;
+  static constexpr int kScalarFolds = dev::count_if<CL>(dev::is_scalar_fold);
+  static constexpr int kScanTile = dev::kBlock * 16;
+
+  // Local id of the array whose index space root `i` iterates over, -1 if i is no root.
+  static int domain_of(int i) {
+    const CNode& n = CL::c.nodes[i];
+    if (dev::is_store_root(n) || dev::is_scan_root(n)) return i;
+    if (dev::is_fold_root(n)) return n.in[0];
+    if (dev::is_permute_root(n)) return n.in[1];
+    return -1;
+  }
+
+  // Iteration domain: shape of the first root's index space.
+  static bool domain(const ClusterLaunch& L, int& R, int& C) {
+    for (int i = 0; i < N; ++i) {
+      const int at = domain_of(i);
+      if (at >= 0) { R = L.nodes[at].R; C = L.nodes[at].C; return true; }
+    }
+    return false;
+  }
+
+  // Every root must iterate over the same domain (a legal cluster has one iteration size).
+  static bool domains_agree(const ClusterLaunch& L, int R, int C) {
+    for (int i = 0; i < N; ++i) {
+      const int at = domain_of(i);
+      if (at >= 0 && (L.nodes[at].R != R || L.nodes[at].C != C)) return false;
+    }
+    return true;
+  }
+
+  // 128-bit accesses need every array's innermost extent and base address to allow them.
+  static bool vec_ok(const ClusterLaunch& L, int C) {
+    if (C % 4) return false;
+    for (int i = 0; i < N; ++i) {
+      const CNode& n = CL::c.nodes[i];
+      if (!n.member) {
+        bool as_array = false;                         // free variables are scalar reads
+        for (int j = 0; j < N; ++j)
+          for (int s = 0; s < CL::c.nodes[j].narr; ++s)
+            if (CL::c.nodes[j].member && CL::c.nodes[j].in[s] == i) as_array = true;
+        if (!as_array) continue;
+      } else if (!dev::is_store_root(n) && !dev::is_scan_root(n)) {
+        continue;                                      // never written with a vector store
+      }
+      if (L.nodes[i].C % 4 || (reinterpret_cast<uintptr_t>(L.nodes[i].ptr) & 15)) return false;
+    }
+    return true;
+  }
+
+  static int stream_grid(int R, int C, bool vec) {
+    const int64_t chunks = (int64_t)R * (C / (vec ? 4 : 1));
+    const int64_t want = (chunks + dev::kBlock - 1) / dev::kBlock;
+    return (int)std::max<int64_t>(1, std::min<int64_t>(want, (int64_t)sm_count() * 8));
+  }
+
+  static int64_t scratch_bytes(const ClusterLaunch& L) {
+    int R, C;
+    if (!domain(L, R, C)) return ACC_ERR_NO_KERNEL;
+    if (kHasScan) return 16 + (int64_t)(((int64_t)R * C + kScanTile - 1) / kScanTile) * 8;
+    if (kHasRowFold) return 0;
+    int64_t words = dev::stream_acc64_off(kScalarFolds, sm_count() * 8);
+    for (int i = 0; i < N; ++i)
+      if (dev::is_f32_add_permute(CL::c.nodes[i])) words += 2 * (int64_t)L.nodes[i].R * L.nodes[i].C;
+    return words * 4;
+  }
+
+  static void fill(const ClusterLaunch& L, dev::Args<N>& a, int R, int C) {
+    for (int i = 0; i < N; ++i) a.n[i] = L.nodes[i];
+    a.R = R;
+    a.C = C;
+    a.scratch = L.scratch;
+    a.status = L.status;
+    a.spin_limit = L.spin_limit;
+    a.grid = sm_count() * 8;             // the partials' layout is sized for the largest grid
+  }
+
+  static int launch(const ClusterLaunch& L) {
+    int R, C;
+    if (!domain(L, R, C)) return set_error(ACC_ERR_NO_KERNEL, "cluster without a root");
+    if (!domains_agree(L, R, C)) return set_error(ACC_ERR_SHAPE, "members of one cluster iterate over different sizes");
+    const bool vec = vec_ok(L, C);
+    // scatters on integers work in place on a copy of the defaults
+    for (int i = 0; i < N; ++i) {
+      const CNode& n = CL::c.nodes[i];
+      if (dev::is_permute_root(n) && !dev::is_f32_add_permute(n)) {
+        const size_t bytes = (size_t)L.nodes[i].R * L.nodes[i].C * 4;
+        if (bytes && cudaMemcpyAsync(const_cast<void*>(L.nodes[i].ptr), L.nodes[n.in[0]].ptr, bytes,
+                                     cudaMemcpyDeviceToDevice, L.stream) != cudaSuccess)
+          return set_error(ACC_ERR_CUDA, "copy of scatter defaults failed: %s", cudaGetErrorString(cudaGetLastError()));
+      }
+    }
+    dev::Args<N> a;
+    fill(L, a, R, C);
+    if constexpr (kHasScan) {
+      if (R != 1) return set_error(ACC_ERR_NO_KERNEL, "scans of rank-2 arrays are not instantiated");
+      if (C == 0) return ACC_OK;
+      const int tiles = (C + kScanTile - 1) / kScanTile;
+      const int grid = std::min(tiles, sm_count() * 6);
+      if (vec) dev::k_scan<CL, true><<<grid, dev::kBlock, 0, L.stream>>>(a, tiles);
+      else dev::k_scan<CL, false><<<grid, dev::kBlock, 0, L.stream>>>(a, tiles);
+    } else if constexpr (kHasRowFold) {
+      if (R == 0) return ACC_OK;
+      const int grid = std::min(R, sm_count() * 16);
+      if (vec) dev::k_rowfold<CL, true><<<grid, dev::kBlock, 0, L.stream>>>(a);
+      else dev::k_rowfold<CL, false><<<grid, dev::kBlock, 0, L.stream>>>(a);
+    } else {
+      // an empty domain still runs one block: a scatter must copy its defaults out
+      const int grid = stream_grid(R, C, vec);
+      if (vec) dev::k_stream<CL, true><<<grid, dev::kBlock, 0, L.stream>>>(a);
+      else dev::k_stream<CL, false><<<grid, dev::kBlock, 0, L.stream>>>(a);
+    }
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return set_error(ACC_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+    return ACC_OK;
+  }
+};
+
+template <class CL>
+struct Registrar {
+  explicit Registrar(const char* name) {
+    register_kernel(KernelEntry{signature(CL::c), name, &Launcher<CL>::scratch_bytes, &Launcher<CL>::launch});
+  }
+};
+
+#define ACC_CAT2(a, b) a##b
+#define ACC_CAT(a, b) ACC_CAT2(a, b)
+// Instantiates the kernels of cluster MASK of program PROG and registers them under NAME.
+#define ACC_CLUSTER(PROG, MASK, NAME)                                              \
+  struct ACC_CAT(Cl_, NAME) { static constexpr CCluster c = extract(PROG, MASK); }; \
+  static Registrar<ACC_CAT(Cl_, NAME)> ACC_CAT(reg_, NAME)(#NAME);
+
+}  // namespace acc

@@ -1,0 +1,390 @@
+// The three kernel skeletons a fused cluster is instantiated into.
+//
+//   k_stream   grid-stride pass over the cluster's iteration domain; stores every manifest
+//              element-wise member, accumulates whole-array folds (warp shuffles, block
+//              tree, ordered cross-block combine by the last block) and applies permutes
+//              with atomics.
+//   k_rowfold  one block per row of a rank-2 domain; folds of the innermost extent end in a
+//              block reduction, no atomics.
+//   k_scan     single-pass inclusive scan with decoupled look-back (tiles are claimed from
+//              an atomic ticket so that a tile's predecessors are always already running);
+//              the scanned operand is evaluated in registers.
+//
+// Each is templated on the cluster description (what to evaluate) and on VEC (whether four
+// consecutive elements move as one 128-bit access).
+#pragma once
+#include "eval.cuh"
+
+namespace acc {
+namespace dev {
+
+constexpr int kBlock = 256;
+constexpr uint32_t kStatusTimeout = 1u;
+constexpr uint32_t kStatusIndex = 2u;
+
+template <int FN, int DT>
+__device__ __forceinline__ uint32_t warp_reduce(uint32_t v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = combine<FN, DT>(v, __shfl_down_sync(0xFFFFFFFFu, v, o));
+  return v;
+}
+
+// Reduces over the block; the result is valid in thread 0.  `red` holds kBlock/32 words.
+template <int FN, int DT>
+__device__ __forceinline__ uint32_t block_reduce(uint32_t v, uint32_t* red) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  v = warp_reduce<FN, DT>(v);
+  __syncthreads();
+  if (lane == 0) red[warp] = v;
+  __syncthreads();
+  if (warp == 0) {
+    v = lane < kBlock / 32 ? red[lane] : identity_of<FN, DT>();
+    v = warp_reduce<FN, DT>(v);
+  }
+  return v;
+}
+
+// ---- compile-time layout of a cluster's roots ------------------------------------------
+template <class CL> constexpr int count_if(bool (*pred)(const CNode&), int upto = CL::c.n) {
+  int k = 0;
+  for (int i = 0; i < upto; ++i) k += pred(CL::c.nodes[i]) ? 1 : 0;
+  return k;
+}
+constexpr bool is_f32_add_permute(const CNode& n) { return is_permute_root(n) && n.dtype == ACC_F32 && n.fn == ACC_FN_ADD; }
+constexpr bool is_scalar_fold(const CNode& n) { return is_fold_root(n) && n.rank == 0; }
+constexpr bool is_row_fold(const CNode& n) { return is_fold_root(n) && n.rank > 0; }
+
+template <class CL> constexpr int first_scan() {
+  for (int i = 0; i < CL::c.n; ++i)
+    if (is_scan_root(CL::c.nodes[i])) return i;
+  return -1;
+}
+
+// Rank of the iteration domain: taken from the first root.
+template <class CL> constexpr int domain_rank() {
+  for (int i = 0; i < CL::c.n; ++i) {
+    const CNode& n = CL::c.nodes[i];
+    if (is_store_root(n) || is_scan_root(n)) return n.rank;
+    if (is_fold_root(n)) return CL::c.nodes[n.in[0]].rank;
+    if (is_permute_root(n)) return CL::c.nodes[n.in[1]].rank;
+  }
+  return 1;
+}
+
+// Scratch layout of k_stream (32-bit words): [0] ticket, [4 ..) one partial per block per
+// scalar fold, then (8-byte aligned) one fp64 accumulator per bin per fp32 '+' permute.
+__host__ __device__ inline uint32_t stream_partials_off() { return 4; }
+__host__ __device__ inline uint32_t stream_acc64_off(int n_scalar_folds, int grid) {
+  return (4u + (uint32_t)(n_scalar_folds * grid) + 1u) & ~1u;
+}
+
+template <int FN, int DT>
+__device__ __forceinline__ void permute_update(uint32_t* out, double* acc64, uint32_t bins, uint32_t k, uint32_t x,
+                                               uint32_t* status) {
+  if (k >= bins) { atomicOr(status, kStatusIndex); return; }
+  if constexpr (DT == ACC_F32 && FN == ACC_FN_ADD) {
+    // lanes of the warp that hit the same bin are summed first; one fp64 atomic per bin and warp
+    const unsigned peers = __match_any_sync(__activemask(), k);
+    double sum = 0.0;
+    for (unsigned t = peers; t; t &= t - 1) sum += (double)__shfl_sync(peers, f_(x), __ffs(t) - 1);
+    if ((int)(threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(acc64 + k, sum);
+  } else if constexpr (FN == ACC_FN_ADD) {
+    atomicAdd(out + k, x);
+  } else if constexpr (FN == ACC_FN_MIN) {
+    if constexpr (DT == ACC_I32) atomicMin(reinterpret_cast<int*>(out) + k, (int)x); else atomicMin(out + k, x);
+  } else {
+    if constexpr (DT == ACC_I32) atomicMax(reinterpret_cast<int*>(out) + k, (int)x); else atomicMax(out + k, x);
+  }
+}
+
+// fp64 accumulators of the I-th member (an fp32 '+' permute): after those of earlier ones.
+template <class CL, int I, class A>
+__device__ __forceinline__ double* acc64_of(const A& a, double* base) {
+  static_for<0, I>([&](auto jc) {
+    constexpr int j = decltype(jc)::value;
+    if constexpr (is_f32_add_permute(CL::c.nodes[j])) base += a.n[j].R * a.n[j].C;
+  });
+  return base;
+}
+
+// =========================================================================================
+template <class CL, bool VEC>
+__global__ void __launch_bounds__(kBlock) k_stream(const __grid_constant__ Args<CL::c.n> a) {
+  constexpr int N = CL::c.n;
+  constexpr int W = VEC ? 4 : 1;
+  constexpr int DR = domain_rank<CL>();
+  constexpr int NF = count_if<CL>(is_scalar_fold);
+  constexpr int NP64 = count_if<CL>(is_f32_add_permute);
+  using IX = std::conditional_t<VEC, Ix4, Ix>;
+  __shared__ uint32_t red[kBlock / 32];
+  __shared__ bool last_block;
+
+  uint32_t acc[N];
+  static_for<0, N>([&](auto ic) {
+    constexpr int i = decltype(ic)::value;
+    constexpr CNode nd = CL::c.nodes[i];
+    if constexpr (is_scalar_fold(nd)) acc[i] = identity_of<nd.fn, nd.dtype>();
+  });
+  double* acc64_base = reinterpret_cast<double*>(a.scratch + stream_acc64_off(NF, a.grid));
+
+  const uint32_t per_row = (uint32_t)a.C / W;
+  const uint32_t total = (uint32_t)a.R * per_row;
+  const uint32_t stride = gridDim.x * kBlock;
+  for (uint32_t q = blockIdx.x * kBlock + threadIdx.x; q < total; q += stride) {
+    IX ix;
+    if constexpr (DR <= 1) { ix.r = 0; ix.c = (int)(q * W); }
+    else { const uint32_t r = q / per_row; ix.r = (int)r; ix.c = (int)((q - r * per_row) * W); }
+    static_for<0, N>([&](auto ic) {
+      constexpr int i = decltype(ic)::value;
+      constexpr CNode nd = CL::c.nodes[i];
+      if constexpr (is_store_root(nd)) {
+        st(reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr)), a.n[i].C, ix, eval<CL, i>(a, ix));
+      } else if constexpr (is_scalar_fold(nd)) {
+        const auto v = eval<CL, nd.in[0]>(a, ix);
+        if constexpr (VEC) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) acc[i] = combine<nd.fn, nd.dtype>(acc[i], v.v[j]);
+        } else {
+          acc[i] = combine<nd.fn, nd.dtype>(acc[i], v);
+        }
+      } else if constexpr (is_permute_root(nd)) {
+        const auto k = eval<CL, nd.in[1]>(a, ix);
+        const auto x = eval<CL, nd.in[2]>(a, ix);
+        uint32_t* out = reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr));
+        const uint32_t bins = (uint32_t)(a.n[i].R * a.n[i].C);
+        double* acc64 = acc64_of<CL, i>(a, acc64_base);
+        if constexpr (VEC) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) permute_update<nd.fn, nd.dtype>(out, acc64, bins, k.v[j], x.v[j], a.status);
+        } else {
+          permute_update<nd.fn, nd.dtype>(out, acc64, bins, k, x, a.status);
+        }
+      }
+    });
+  }
+
+  if constexpr (NF > 0 || NP64 > 0) {
+    // partial of every scalar fold, then the block that arrives last finishes the job
+    static_for<0, N>([&](auto ic) {
+      constexpr int i = decltype(ic)::value;
+      constexpr CNode nd = CL::c.nodes[i];
+      if constexpr (is_scalar_fold(nd)) {
+        constexpr int ord = count_if<CL>(is_scalar_fold, i);
+        const uint32_t v = block_reduce<nd.fn, nd.dtype>(acc[i], red);
+        if (threadIdx.x == 0) a.scratch[stream_partials_off() + ord * a.grid + blockIdx.x] = v;
+      }
+    });
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) last_block = atomicAdd(a.scratch, 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (!last_block) return;
+    __threadfence();
+    static_for<0, N>([&](auto ic) {
+      constexpr int i = decltype(ic)::value;
+      constexpr CNode nd = CL::c.nodes[i];
+      if constexpr (is_scalar_fold(nd)) {
+        constexpr int ord = count_if<CL>(is_scalar_fold, i);
+        const volatile uint32_t* part = a.scratch + stream_partials_off() + ord * a.grid;
+        uint32_t v = identity_of<nd.fn, nd.dtype>();
+        for (int b = threadIdx.x; b < (int)gridDim.x; b += kBlock) v = combine<nd.fn, nd.dtype>(v, part[b]);
+        v = block_reduce<nd.fn, nd.dtype>(v, red);
+        if (threadIdx.x == 0) *reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr)) = v;
+      } else if constexpr (is_f32_add_permute(nd)) {
+        const volatile double* acc64 = acc64_of<CL, i>(a, acc64_base);
+        const float* defaults = reinterpret_cast<const float*>(a.n[nd.in[0]].ptr);
+        float* out = reinterpret_cast<float*>(const_cast<void*>(a.n[i].ptr));
+        const int bins = a.n[i].R * a.n[i].C;
+        for (int b = threadIdx.x; b < bins; b += kBlock) out[b] = (float)((double)defaults[b] + acc64[b]);
+      }
+    });
+  }
+}
+
+// =========================================================================================
+template <class CL, bool VEC>
+__global__ void __launch_bounds__(kBlock) k_rowfold(const __grid_constant__ Args<CL::c.n> a) {
+  constexpr int N = CL::c.n;
+  constexpr int W = VEC ? 4 : 1;
+  using IX = std::conditional_t<VEC, Ix4, Ix>;
+  __shared__ uint32_t red[kBlock / 32];
+  for (int r = blockIdx.x; r < a.R; r += gridDim.x) {
+    uint32_t acc[N];
+    static_for<0, N>([&](auto ic) {
+      constexpr int i = decltype(ic)::value;
+      constexpr CNode nd = CL::c.nodes[i];
+      if constexpr (is_row_fold(nd)) acc[i] = identity_of<nd.fn, nd.dtype>();
+    });
+    for (int c = threadIdx.x * W; c < a.C; c += kBlock * W) {
+      const IX ix{r, c};
+      static_for<0, N>([&](auto ic) {
+        constexpr int i = decltype(ic)::value;
+        constexpr CNode nd = CL::c.nodes[i];
+        if constexpr (is_store_root(nd)) {
+          st(reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr)), a.n[i].C, ix, eval<CL, i>(a, ix));
+        } else if constexpr (is_row_fold(nd)) {
+          const auto v = eval<CL, nd.in[0]>(a, ix);
+          if constexpr (VEC) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i] = combine<nd.fn, nd.dtype>(acc[i], v.v[j]);
+          } else {
+            acc[i] = combine<nd.fn, nd.dtype>(acc[i], v);
+          }
+        }
+      });
+    }
+    static_for<0, N>([&](auto ic) {
+      constexpr int i = decltype(ic)::value;
+      constexpr CNode nd = CL::c.nodes[i];
+      if constexpr (is_row_fold(nd)) {
+        const uint32_t v = block_reduce<nd.fn, nd.dtype>(acc[i], red);
+        if (threadIdx.x == 0) reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr))[r] = v;
+      }
+    });
+  }
+}
+
+// =========================================================================================
+// Scratch layout of k_scan: word [0] ticket; from byte 16 one 64-bit tile state per tile:
+// (flag << 32) | value, flag 0 = nothing yet, 1 = the tile's own total, 2 = inclusive prefix.
+constexpr int kScanRows = 4;                     // 128-bit chunks per thread
+constexpr uint64_t kFlagAggregate = 1, kFlagPrefix = 2;
+
+__device__ __forceinline__ uint64_t ld_state(const uint64_t* p) {
+  return *reinterpret_cast<const volatile uint64_t*>(p);
+}
+__device__ __forceinline__ void st_state(uint64_t* p, uint64_t flag, uint32_t v) {
+  *reinterpret_cast<volatile uint64_t*>(p) = (flag << 32) | v;
+}
+
+template <class CL, bool VEC>
+__global__ void __launch_bounds__(kBlock) k_scan(const __grid_constant__ Args<CL::c.n> a, int n_tiles) {
+  constexpr int N = CL::c.n;
+  constexpr int W = VEC ? 4 : 1;
+  constexpr int ROWS = VEC ? kScanRows : kScanRows * 4;   // 16 elements per thread either way
+  constexpr int TILE = kBlock * 16;
+  using IX = std::conditional_t<VEC, Ix4, Ix>;
+  constexpr int S = first_scan<CL>();
+  static_assert(S >= 0, "k_scan needs a scan member");
+  constexpr CNode sn = CL::c.nodes[S];
+  constexpr int FN = sn.fn, DT = sn.dtype;
+  static_assert(sn.kind == ACC_SCANL, "right-to-left scans are not instantiated");
+
+  __shared__ uint32_t warp_total[kBlock / 32];
+  __shared__ uint32_t tile_prefix;
+  __shared__ int tile_id;
+  uint64_t* states = reinterpret_cast<uint64_t*>(a.scratch + 4);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int n = a.C;                                       // rank-1 domain
+
+  for (;;) {
+    __syncthreads();
+    if (threadIdx.x == 0) tile_id = (int)atomicAdd(a.scratch, 1u);
+    __syncthreads();
+    const int tile = tile_id;
+    if (tile >= n_tiles) return;
+    const int warp_base = tile * TILE + warp * (TILE / (kBlock / 32));
+
+    uint32_t val[ROWS][W];
+    uint32_t carry = identity_of<FN, DT>();                // running total of this warp's earlier rows
+#pragma unroll
+    for (int j = 0; j < ROWS; ++j) {
+      const int c = warp_base + (j * 32 + lane) * W;
+      const bool live = c < n;
+      if (live) {
+        const IX ix{0, c};
+        const auto v = eval<CL, sn.in[0]>(a, ix);
+        if constexpr (VEC) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) val[j][e] = v.v[e];
+        } else {
+          val[j][0] = v;
+        }
+        static_for<0, N>([&](auto ic) {
+          constexpr int i = decltype(ic)::value;
+          if constexpr (is_store_root(CL::c.nodes[i]))
+            st(reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr)), a.n[i].C, ix, eval<CL, i>(a, ix));
+        });
+      } else {
+#pragma unroll
+        for (int e = 0; e < W; ++e) val[j][e] = identity_of<FN, DT>();
+      }
+      // inclusive scan inside the thread, then across the warp
+#pragma unroll
+      for (int e = 1; e < W; ++e) val[j][e] = combine<FN, DT>(val[j][e - 1], val[j][e]);
+      uint32_t incl = val[j][W - 1];
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl = combine<FN, DT>(t, incl);
+      }
+      uint32_t excl = __shfl_up_sync(0xFFFFFFFFu, incl, 1);
+      if (lane == 0) excl = identity_of<FN, DT>();
+      excl = combine<FN, DT>(carry, excl);
+#pragma unroll
+      for (int e = 0; e < W; ++e) val[j][e] = combine<FN, DT>(excl, val[j][e]);
+      carry = combine<FN, DT>(carry, __shfl_sync(0xFFFFFFFFu, incl, 31));
+    }
+    if (lane == 0) warp_total[warp] = carry;
+    __syncthreads();
+    uint32_t offset = identity_of<FN, DT>();               // total of the warps before this one
+    uint32_t tile_total = identity_of<FN, DT>();
+#pragma unroll
+    for (int w = 0; w < kBlock / 32; ++w) {
+      const uint32_t t = warp_total[w];
+      if (w < warp) offset = combine<FN, DT>(offset, t);
+      tile_total = combine<FN, DT>(tile_total, t);
+    }
+
+    if (warp == 0) {
+      uint32_t exclusive = identity_of<FN, DT>();
+      if (tile == 0) {
+        if (lane == 0) st_state(states, kFlagPrefix, tile_total);
+      } else {
+        if (lane == 0) st_state(states + tile, kFlagAggregate, tile_total);
+        int look = tile - 1;
+        uint32_t spins = 0;
+        bool gave_up = false;
+        for (;;) {
+          const int idx = look - lane;
+          uint64_t s = idx >= 0 ? ld_state(states + idx) : (kFlagPrefix << 32) | identity_of<FN, DT>();
+          while (__any_sync(0xFFFFFFFFu, (s >> 32) == 0)) {
+            if (++spins > a.spin_limit) { gave_up = true; break; }
+            __nanosleep(20);
+            if (idx >= 0) s = ld_state(states + idx);
+          }
+          if (gave_up) break;
+          const unsigned done = __ballot_sync(0xFFFFFFFFu, (s >> 32) == kFlagPrefix);
+          const int stop = done ? __ffs(done) - 1 : 31;
+          uint32_t part = lane <= stop ? (uint32_t)s : identity_of<FN, DT>();
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) part = combine<FN, DT>(part, __shfl_xor_sync(0xFFFFFFFFu, part, o));
+          exclusive = combine<FN, DT>(part, exclusive);
+          if (done) break;
+          look -= 32;
+        }
+        if (gave_up && lane == 0) atomicOr(a.status, kStatusTimeout);
+        if (lane == 0) st_state(states + tile, kFlagPrefix, combine<FN, DT>(exclusive, tile_total));
+      }
+      if (lane == 0) tile_prefix = exclusive;
+    }
+    __syncthreads();
+    const uint32_t base = combine<FN, DT>(tile_prefix, offset);
+    uint32_t* out = reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[S].ptr));
+#pragma unroll
+    for (int j = 0; j < ROWS; ++j) {
+      const int c = warp_base + (j * 32 + lane) * W;
+      if (c < n) {
+        if constexpr (VEC) {
+          st(out, n, Ix4{0, c}, V4{{combine<FN, DT>(base, val[j][0]), combine<FN, DT>(base, val[j][1]),
+                                    combine<FN, DT>(base, val[j][2]), combine<FN, DT>(base, val[j][3])}});
+        } else {
+          out[c] = combine<FN, DT>(base, val[j][0]);
+        }
+      }
+    }
+  }
+}
+
+}  // namespace dev
+}  // namespace acc

@@ -1,0 +1,176 @@
+// Execution of a program: clusters in ascending cluster number, one kernel launch per
+// cluster on the caller's stream (Section 4.1: "clusters are executed in the ascending
+// order of their cluster numbers").  The unfused executor is the same machinery with
+// every combinator its own cluster.
+#include <algorithm>
+#include <cstring>
+#include <map>
+
+#include "cluster.h"
+#include "exec.h"
+#include "graph.h"
+#include "registry.h"
+
+namespace acc {
+
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Cuts the cluster formed by `members` (ascending) out of the graph, mirroring the
+// build-time extract(): externals appear just before their first use.
+static bool extract_runtime(const Graph& g, const std::vector<int>& members, const std::vector<uint8_t>& man, CCluster& c) {
+  c = CCluster{};
+  std::map<int, int> local;
+  std::vector<uint8_t> in_cluster(g.nodes.size(), 0);
+  for (int m : members) in_cluster[m] = 1;
+  for (int m : members) {
+    const acc_node_desc& d = g.nodes[m].d;
+    for (int s = 0; s < d.n_inputs; ++s) {
+      const int a = d.inputs[s];
+      if (!in_cluster[a] && !local.count(a)) {
+        if (c.n >= kMaxCluster) return false;
+        CNode e{ACC_INPUT, g.nodes[a].d.dtype, g.nodes[a].d.rank, 0, 0, 0, 0, {-1, -1, -1, -1, -1, -1}, false, true};
+        local[a] = c.n;
+        c.source[c.n] = a;
+        c.nodes[c.n++] = e;
+      }
+    }
+    if (c.n >= kMaxCluster) return false;
+    CNode n{d.kind, d.dtype, d.rank, d.fn_id, d.idx_fn_id, d.n_inputs, d.n_array_inputs, {-1, -1, -1, -1, -1, -1}, true, man[m] != 0};
+    if (d.kind != ACC_BACKPERMUTE) n.idxfn = 0;
+    if (d.kind == ACC_BACKPERMUTE || d.kind == ACC_GATHER) n.fn = 0;
+    for (int s = 0; s < d.n_inputs; ++s) n.in[s] = local[d.inputs[s]];
+    local[m] = c.n;
+    c.source[c.n] = m;
+    c.nodes[c.n++] = n;
+  }
+  return true;
+}
+
+static dev::NodeArg node_arg(const Node& n, const void* ptr) {
+  dev::NodeArg a{};
+  a.ptr = ptr;
+  a.ip0 = (int32_t)(uint32_t)(n.d.iparam[0] & 0xFFFFFFFFll);
+  a.ip1 = (int32_t)(uint32_t)(n.d.iparam[1] & 0xFFFFFFFFll);
+  a.fp0 = (float)n.d.fparam[0];
+  a.fp1 = (float)n.d.fparam[1];
+  a.R = n.d.rank == 2 ? (int32_t)n.d.shape[0] : 1;
+  a.C = n.d.rank == 2 ? (int32_t)n.d.shape[1] : (n.d.rank == 1 ? (int32_t)n.d.shape[0] : 1);
+  return a;
+}
+
+int build_schedule(Graph& g, int executor, Schedule& sch) {
+  const int n = (int)g.nodes.size();
+  sch = Schedule{};
+  std::vector<int32_t> pi;
+  if (executor == ACC_EXEC_FUSED) {
+    if (!g.has_pi) return set_error(ACC_ERR_NO_PARTITION, "no clustering set: call acc_set_partition or acc_plan first");
+    pi = g.pi;
+  } else if (executor == ACC_EXEC_UNFUSED) {
+    pi.assign(n, -1);
+    int c = 0;
+    for (int i = 0; i < n; ++i)
+      if (!is_input(g.nodes[i])) pi[i] = c++;
+  } else {
+    return set_error(ACC_ERR_ARG, "unknown executor %d", executor);
+  }
+  std::vector<uint8_t> man;
+  manifest_of(g, pi.data(), man);
+
+  // buffers: bound ones stay where they are, other manifest arrays go into the workspace
+  sch.array_off.assign(n, SIZE_MAX);
+  size_t off = 0;
+  for (int i = 0; i < n; ++i) {
+    const Node& nd = g.nodes[i];
+    if (is_input(nd) || nd.output) {
+      if (!nd.dev && nd.count > 0)
+        return set_error(ACC_ERR_UNBOUND, "node %d (%s) has no device buffer", i, is_input(nd) ? "input" : "output");
+      continue;
+    }
+    if (!man[i] || nd.dev) continue;
+    sch.array_off[i] = off;
+    off += align_up((size_t)std::max<int64_t>(nd.count, 1) * 4, 256);
+  }
+  sch.array_bytes = off;
+
+  std::map<int, std::vector<int>> clusters;
+  for (int i = 0; i < n; ++i)
+    if (!is_input(g.nodes[i])) clusters[pi[i]].push_back(i);
+  size_t ctrl = 256;                                    // status word first
+  for (auto& kv : clusters) {
+    ClusterStep st;
+    st.first_node = kv.second.front();
+    st.n_members = (int)kv.second.size();
+    if (!extract_runtime(g, kv.second, man, st.cc))
+      return set_error(ACC_ERR_NO_KERNEL, "cluster at node %d has more than %d local nodes", st.first_node, kMaxCluster);
+    const std::string sig = signature(st.cc);
+    st.kernel = find_kernel(sig);
+    if (!st.kernel)
+      return set_error(ACC_ERR_NO_KERNEL, "no kernel instantiated for the cluster of %d nodes starting at node %d [%s]",
+                       st.n_members, st.first_node, sig.c_str());
+    st.launch.n = st.cc.n;
+    for (int li = 0; li < st.cc.n; ++li) st.launch.nodes[li] = node_arg(g.nodes[st.cc.source[li]], nullptr);
+    const int64_t sb = st.kernel->scratch_bytes(st.launch);
+    if (sb < 0) return set_error((int)sb, "cluster at node %d: no scratch layout", st.first_node);
+    st.scratch_off = ctrl;
+    st.scratch_bytes = (size_t)sb;
+    ctrl += align_up((size_t)sb, 256);
+    sch.steps.push_back(st);
+  }
+  sch.ctrl_bytes = ctrl;
+  sch.total_bytes = ctrl + sch.array_bytes;
+  sch.manifest = man;
+  sch.pi = pi;
+  return ACC_OK;
+}
+
+static void* buffer_of(const Graph& g, const Schedule& sch, char* ws, int node) {
+  const Node& nd = g.nodes[node];
+  if (nd.dev) return nd.dev;
+  if (sch.array_off[node] == SIZE_MAX) return nullptr;
+  return ws + sch.ctrl_bytes + sch.array_off[node];
+}
+
+int run_schedule(Graph& g, Schedule& sch, void* workspace, size_t ws_bytes, cudaStream_t stream) {
+  if (!workspace) return set_error(ACC_ERR_WORKSPACE, "workspace is null, %zu bytes needed", sch.total_bytes);
+  if (reinterpret_cast<uintptr_t>(workspace) & 255) return set_error(ACC_ERR_WORKSPACE, "workspace is not 256-byte aligned");
+  if (ws_bytes < sch.total_bytes) return set_error(ACC_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", ws_bytes, sch.total_bytes);
+  char* ws = static_cast<char*>(workspace);
+  if (cudaMemsetAsync(ws, 0, sch.ctrl_bytes, stream) != cudaSuccess)
+    return set_error(ACC_ERR_CUDA, "clearing the control region failed: %s", cudaGetErrorString(cudaGetLastError()));
+  g.launches = 0;
+  g.schedule.clear();
+  for (ClusterStep& st : sch.steps) {
+    for (int li = 0; li < st.cc.n; ++li) {
+      const int node = st.cc.source[li];
+      const CNode& cn = st.cc.nodes[li];
+      void* p = (!cn.member || cn.manifest) ? buffer_of(g, sch, ws, node) : nullptr;
+      if ((!cn.member || cn.manifest) && !p && g.nodes[node].count > 0)
+        return set_error(ACC_ERR_UNBOUND, "node %d is read or written by the cluster at node %d but has no buffer", node, st.first_node);
+      st.launch.nodes[li].ptr = p;
+    }
+    st.launch.scratch = reinterpret_cast<uint32_t*>(ws + st.scratch_off);
+    st.launch.status = reinterpret_cast<uint32_t*>(ws);
+    st.launch.stream = stream;
+    const int rc = st.kernel->launch(st.launch);
+    if (rc != ACC_OK) return rc;
+    g.launches += 1;
+    char item[48];
+    snprintf(item, sizeof item, "%s%d:%d", g.schedule.empty() ? "" : " ", st.first_node, st.n_members);
+    g.schedule += item;
+  }
+  return ACC_OK;
+}
+
+int finish(Graph& g, void* workspace, cudaStream_t stream) {
+  uint32_t status = 0;
+  if (workspace && cudaMemcpyAsync(&status, workspace, 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+    return set_error(ACC_ERR_CUDA, "reading the status word failed: %s", cudaGetErrorString(cudaGetLastError()));
+  const cudaError_t e = cudaStreamSynchronize(stream);
+  if (e != cudaSuccess) return set_error(ACC_ERR_CUDA, "stream failed: %s", cudaGetErrorString(e));
+  g.host_status = status;
+  if (status & 1u) return set_error(ACC_ERR_DEVICE_TIMEOUT, "a device-side wait ran out of iterations");
+  if (status & 2u) return set_error(ACC_ERR_INDEX_RANGE, "a scatter index fell outside its destination");
+  return ACC_OK;
+}
+
+}  // namespace acc

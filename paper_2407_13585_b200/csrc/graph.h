@@ -1,0 +1,69 @@
+// Runtime data-dependence graph of a combinator program (Section 4.1 of the paper:
+// nodes, fusible edges F, infusible edges I) and the state attached to it.
+#pragma once
+#include <cstdarg>
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include "acc.h"
+
+namespace acc {
+
+struct Node {
+  acc_node_desc d{};
+  bool     output = false;
+  int64_t  count = 0;          // number of elements
+  void*    dev = nullptr;      // caller-bound device buffer
+  size_t   dev_bytes = 0;
+  void*    host = nullptr;     // caller-bound host buffer (end-to-end runs)
+  size_t   host_bytes = 0;
+};
+
+// One edge per input slot of the consumer.
+struct Edge {
+  int  a, b, slot;
+  bool fusible;   // may be fused when a and b share a cluster
+  bool ordered;   // the slot traverses the array in a definite order (Table 1)
+};
+
+struct Graph {
+  std::vector<Node> nodes;
+  std::vector<Edge> edges;
+  std::vector<int32_t> pi;         // stored clustering, -1 for inputs
+  bool has_pi = false;
+  std::vector<uint8_t> manifest;   // under the stored clustering
+  // bookkeeping of the last run
+  int32_t launches = 0;
+  std::string schedule;
+  uint32_t host_status = 0;
+  uint32_t run_serial = 0;         // bumped by every change that invalidates a schedule
+};
+
+inline bool is_input(const Node& n) { return n.d.kind == ACC_INPUT; }
+inline bool gather_like(const Node& n) { return n.d.kind == ACC_GATHER || n.d.kind == ACC_BACKPERMUTE; }
+
+int  set_error(int code, const char* fmt, ...);
+const char* last_error();
+void clear_error();
+
+// graph.cpp
+int  add_node(Graph& g, const acc_node_desc& d);
+
+// legality.cpp
+struct Solution {
+  std::vector<uint8_t> manifest;   // per node
+  std::vector<int32_t> order;      // d^o per node (for PERMUTE: order of its idx/vals slots), -1 for inputs
+};
+int  check_partition(const Graph& g, const int32_t* pi, Solution* sol, bool quiet = false);
+void manifest_of(const Graph& g, const int32_t* pi, std::vector<uint8_t>& man);
+
+// planner.cpp
+int     plan(Graph& g, int mode, int cost, std::vector<int32_t>& out);
+int64_t enumerate_all(const Graph& g, std::vector<std::vector<int32_t>>& out);
+int     partition_cost(const Graph& g, const int32_t* pi, int cost, double* out);
+bool    canonical_numbering(const Graph& g, const std::vector<int>& block_of, int n_blocks, std::vector<int32_t>& pi);
+
+}  // namespace acc
+
+struct acc_graph : acc::Graph {};

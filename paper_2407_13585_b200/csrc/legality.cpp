@@ -1,0 +1,176 @@
+// Legality of a clustering pi: the paper's Figure 3 evaluated for given pi, plus the
+// top-level rules of Section 3.4 and the splitting step of Section 4.1.
+//
+// Within a cluster, x_ab = 0 is forced for every edge (Figure 3: x_ab <= pi_b - pi_a), so
+// the order equalities d^o_a = d^i_b of all inner edges must hold together.  They are
+// solved by union-find over one order variable per node; constants come from scans (0/1)
+// and from the source slot of gather-like nodes (their label).  Manifest arrays need an
+// order in {0,1}.  Order classes that stay free are 0 or 1; which one matters only for
+// whether two reads of a common outside parent are shared, i.e. for connectivity, and is
+// settled by a small exhaustive search.
+#include <algorithm>
+#include <map>
+
+#include "graph.h"
+
+namespace acc {
+
+void manifest_of(const Graph& g, const int32_t* pi, std::vector<uint8_t>& man) {
+  const int n = (int)g.nodes.size();
+  man.assign(n, 0);
+  std::vector<uint8_t> has_out(n, 0);
+  for (const Edge& e : g.edges) {
+    has_out[e.a] = 1;
+    if (is_input(g.nodes[e.a]) || pi[e.a] != pi[e.b] || !e.fusible) man[e.a] = 1;
+  }
+  for (int i = 0; i < n; ++i)
+    if (is_input(g.nodes[i]) || g.nodes[i].output || !has_out[i]) man[i] = 1;
+}
+
+namespace {
+
+struct Dsu {
+  std::vector<int> p;
+  explicit Dsu(int n) : p(n) { for (int i = 0; i < n; ++i) p[i] = i; }
+  int find(int x) { while (p[x] != x) { p[x] = p[p[x]]; x = p[x]; } return x; }
+  void unite(int a, int b) { p[find(a)] = find(b); }
+};
+
+constexpr int kFree = -1;
+
+struct ClusterCheck {
+  const Graph& g;
+  const std::vector<int>& members;         // ascending node ids
+  const std::vector<uint8_t>& man;
+  const std::vector<int>& label;           // label per gather-like node, else 0
+  std::vector<int> local;                  // node id -> index in members, -1 outside
+
+  ClusterCheck(const Graph& g_, const std::vector<int>& m, const std::vector<uint8_t>& man_, const std::vector<int>& lab)
+      : g(g_), members(m), man(man_), label(lab), local(g_.nodes.size(), -1) {
+    for (int i = 0; i < (int)m.size(); ++i) local[m[i]] = i;
+  }
+
+  // Order of slot `slot` of member b: a constant label, or b's own order variable (kFree).
+  int slot_const(int b, int slot) const {
+    const int k = g.nodes[b].d.kind;
+    if (k == ACC_BACKPERMUTE || (k == ACC_GATHER && slot == 1)) return label[b];
+    return kFree;
+  }
+
+  int run(std::vector<int32_t>* order_out) {
+    const int m = (int)members.size();
+    Dsu cls(m);
+    for (const Edge& e : g.edges) {
+      if (local[e.a] < 0 || local[e.b] < 0) continue;
+      if (slot_const(e.b, e.slot) == kFree) cls.unite(local[e.a], local[e.b]);
+    }
+    std::vector<int> value(m, kFree);        // per class root
+    std::vector<uint8_t> zero_one(m, 0);
+    auto pin = [&](int node_local, int v) -> bool {
+      const int r = cls.find(node_local);
+      if (value[r] != kFree && value[r] != v) return false;
+      value[r] = v;
+      return true;
+    };
+    for (int i = 0; i < m; ++i) {
+      const int a = members[i];
+      const int k = g.nodes[a].d.kind;
+      if (k == ACC_SCANL && !pin(i, 0)) return ACC_ERR_ILLEGAL_TRAVERSAL;
+      if (k == ACC_SCANR && !pin(i, 1)) return ACC_ERR_ILLEGAL_TRAVERSAL;
+      if (man[a] || k == ACC_PERMUTE) zero_one[cls.find(i)] = 1;
+    }
+    for (const Edge& e : g.edges) {
+      if (local[e.a] < 0 || local[e.b] < 0) continue;
+      const int c = slot_const(e.b, e.slot);
+      if (c != kFree && !pin(local[e.a], c)) return ACC_ERR_ILLEGAL_TRAVERSAL;
+    }
+    for (int i = 0; i < m; ++i) {
+      const int r = cls.find(i);
+      if (zero_one[r] && value[r] > 1) return ACC_ERR_ILLEGAL_TRAVERSAL;
+    }
+    // connectivity: fused edges, or reads of one outside parent in one order
+    Dsu base(m);
+    for (const Edge& e : g.edges)
+      if (local[e.a] >= 0 && local[e.b] >= 0) base.unite(local[e.a], local[e.b]);
+    struct Read { int parent, cls, node; };
+    std::vector<Read> reads;                 // reads through a node's own order variable
+    for (const Edge& e : g.edges) {
+      if (local[e.b] < 0 || local[e.a] >= 0 || !e.ordered) continue;
+      if (slot_const(e.b, e.slot) != kFree) continue;   // a label is unique: never shared with another node
+      reads.push_back({e.a, cls.find(local[e.b]), local[e.b]});
+    }
+    std::vector<int> free_cls;
+    for (const Read& r : reads)
+      if (value[r.cls] == kFree && std::find(free_cls.begin(), free_cls.end(), r.cls) == free_cls.end()) free_cls.push_back(r.cls);
+    const int k = (int)free_cls.size();
+    const uint32_t combos = k > 16 ? 1u : (1u << k);
+    std::vector<int> trial(value);
+    for (uint32_t bits = 0; bits < combos; ++bits) {
+      for (int j = 0; j < k; ++j) trial[free_cls[j]] = k > 16 ? 0 : int((bits >> j) & 1u);
+      Dsu conn = base;
+      std::map<std::pair<int, int>, int> first;
+      for (const Read& r : reads) {
+        auto key = std::make_pair(r.parent, trial[r.cls]);
+        auto it = first.find(key);
+        if (it == first.end()) first[key] = r.node; else conn.unite(it->second, r.node);
+      }
+      bool one = true;
+      for (int i = 1; i < m && one; ++i) one = conn.find(i) == conn.find(0);
+      if (one) {
+        if (order_out)
+          for (int i = 0; i < m; ++i) {
+            const int r = cls.find(i);
+            (*order_out)[members[i]] = trial[r] == kFree ? 0 : trial[r];
+          }
+        return ACC_OK;
+      }
+    }
+    return ACC_ERR_DISCONNECTED;
+  }
+};
+
+}  // namespace
+
+int check_partition(const Graph& g, const int32_t* pi, Solution* sol, bool quiet) {
+  const int n = (int)g.nodes.size();
+  auto fail = [&](int code, const char* what, int a, int b) {
+    return quiet ? code : set_error(code, "illegal clustering: %s (nodes %d, %d)", what, a, b);
+  };
+  for (const Edge& e : g.edges) {
+    if (is_input(g.nodes[e.a])) continue;
+    if (pi[e.a] > pi[e.b]) return fail(ACC_ERR_ILLEGAL_ORDER, "a consumer runs before its producer", e.a, e.b);
+    if (!e.fusible && pi[e.a] == pi[e.b]) return fail(ACC_ERR_ILLEGAL_INFUSIBLE, "infusible edge inside one cluster", e.a, e.b);
+  }
+  for (int j = 0; j < n; ++j) {
+    if (g.nodes[j].d.kind != ACC_PERMUTE) continue;
+    const int dest = g.nodes[j].d.inputs[0];
+    for (const Edge& e : g.edges)
+      if (e.a == dest && e.b != j && !(pi[e.b] < pi[j]))
+        return fail(ACC_ERR_ILLEGAL_SCATTER, "another use of a scatter destination is not earlier", e.b, j);
+  }
+  std::vector<uint8_t> man;
+  manifest_of(g, pi, man);
+  std::vector<int> label(n, 0);
+  int next = 2;
+  for (int i = 0; i < n; ++i)
+    if (gather_like(g.nodes[i])) label[i] = next++;
+  std::map<int, std::vector<int>> clusters;
+  for (int i = 0; i < n; ++i)
+    if (!is_input(g.nodes[i])) clusters[pi[i]].push_back(i);
+  std::vector<int32_t> order(n, -1);
+  for (auto& kv : clusters) {
+    ClusterCheck cc(g, kv.second, man, label);
+    const int rc = cc.run(&order);
+    if (rc != ACC_OK)
+      return fail(rc, rc == ACC_ERR_DISCONNECTED ? "a cluster does not hang together through a fused array"
+                                                 : "traversal orders cannot be matched",
+                  kv.second.front(), kv.second.back());
+  }
+  if (sol) {
+    sol->manifest = man;
+    sol->order = order;
+  }
+  return ACC_OK;
+}
+
+}  // namespace acc

@@ -1,0 +1,36 @@
+// Registry of build-time kernel instantiations, keyed by cluster signature.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <string>
+
+#include "cluster.h"
+#include "device/eval.cuh"
+
+namespace acc {
+
+// Everything a launcher needs for one cluster of one run.  nodes[] is indexed by the
+// cluster's local ids and carries pointers, constants and shapes.
+struct ClusterLaunch {
+  dev::NodeArg nodes[kMaxCluster];
+  int n = 0;
+  uint32_t* scratch = nullptr;   // zeroed region of scratch_bytes() bytes, 16-byte aligned
+  uint32_t* status = nullptr;
+  uint32_t spin_limit = 1u << 22;
+  cudaStream_t stream = nullptr;
+};
+
+struct KernelEntry {
+  std::string sig;
+  const char* name;
+  int64_t (*scratch_bytes)(const ClusterLaunch&);   // >= 0, or a negative acc_status
+  int (*launch)(const ClusterLaunch&);               // acc_status; asynchronous
+};
+
+void register_kernel(const KernelEntry& e);
+const KernelEntry* find_kernel(const std::string& sig);
+int registry_size();
+int sm_count();
+
+}  // namespace acc
