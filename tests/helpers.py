@@ -1,0 +1,95 @@
+"""Shared pieces of the GPU parity tests: run a program through the C ABI, run the
+oracle on the same inputs, compare array by array."""
+import numpy as np
+
+from oracle import interp, legality
+
+TOL = 1e-5          # |gpu - oracle_fp64| <= TOL * sum|x_i| for fp32 folds, scans and scatters
+
+
+def oracle_run(prog, inputs_np):
+    return interp.run(prog.nodes, inputs_np)
+
+
+def accumulating(nd):
+    return nd.kind in ("fold", "scanl", "scanr", "permute") and nd.dtype == "f32"
+
+
+def count_of(nd):
+    return int(np.prod(nd.shape, dtype=np.int64)) if len(nd.shape) else 1
+
+
+def gpu_run(prog, inputs_t, pi=None, executor=None, bind_all=True, runs=1):
+    """Runs `prog` on the GPU.  pi=None with executor=UNFUSED runs one kernel per node.
+    Returns ({node: numpy array} for every manifest non-input node, Graph)."""
+    import torch
+    from paper_2407_13585_b200 import binding as B
+
+    executor = B.FUSED if executor is None else executor
+    g = B.Graph(prog.nodes, prog.outputs)
+    if pi is not None:
+        g.set_partition(pi)
+    bufs = {}
+    for i, nd in enumerate(prog.nodes):
+        if nd.kind == "input":
+            bufs[i] = inputs_t[i].cuda().contiguous()
+            g.bind(i, bufs[i])
+        elif bind_all or i in prog.outputs:
+            bufs[i] = torch.full((max(count_of(nd), 4),), -12345, dtype=torch.int32, device="cuda")
+            g.bind(i, bufs[i])
+    for _ in range(runs):
+        g.run(executor)
+    torch.cuda.synchronize()
+    man = [True] * len(prog.nodes) if executor == B.UNFUSED else g.manifest()
+    out = {}
+    for i, nd in enumerate(prog.nodes):
+        if nd.kind == "input" or not man[i] or i not in bufs:
+            continue
+        a = bufs[i][:count_of(nd)].cpu().numpy()
+        a = a.view(np.float32) if nd.dtype == "f32" else a.view(np.uint32)
+        out[i] = a.reshape(tuple(nd.shape))
+    return out, g
+
+
+def compare(prog, ref, got, what=""):
+    """Element-by-element comparison of every array in `got` with the oracle result `ref`.
+
+    Integer arrays and fp32 element chains: bit-exact.  fp32 fold/scan/scatter outputs:
+    |gpu - fp64 reference| <= 1e-5 * sum|x_i| (+ half an ulp of the result for the final
+    rounding).  A map that divides such an output by such a total inherits both bounds.
+    """
+    nodes = prog.nodes
+    loose = set()
+    for i, nd in enumerate(nodes):
+        if accumulating(nd) or any(s in loose for s in nd.inputs):
+            loose.add(i)
+    for i, a in got.items():
+        nd = nodes[i]
+        r = ref.values[i]
+        assert a.shape == r.shape, (what, i, a.shape, r.shape)
+        if i not in loose:
+            au, ru = a.view(np.uint32).reshape(-1), r.view(np.uint32).reshape(-1)
+            if not np.array_equal(au, ru):
+                bad = np.flatnonzero(au != ru)
+                raise AssertionError(f"{what} node {i} ({nd.name}): {bad.size} of {a.size} elements differ, first at "
+                                     f"{bad[0]}: gpu {a.reshape(-1)[bad[0]]!r} oracle {r.reshape(-1)[bad[0]]!r}")
+            continue
+        if accumulating(nd):
+            exact, scale = ref.exact[i], ref.abs_sum[i]
+            bound = TOL * scale + np.abs(exact) * 2.0 ** -24 + 1e-30
+            err = np.abs(a.astype(np.float64) - exact)
+            assert np.all(err <= bound), (what, i, nd.name, float((err / bound).max()))
+        elif nd.fn == "div_free":
+            h, t = nd.inputs[0], nd.inputs[1]
+            he, te = ref.exact[h], float(ref.exact[t])
+            frac = he / te
+            bound = ((TOL * ref.abs_sum[h] + np.abs(frac) * TOL * float(ref.abs_sum[t])) / abs(te)
+                     + np.abs(frac) * 2.0 ** -22 + 1e-30)
+            err = np.abs(a.astype(np.float64) - frac)
+            assert np.all(err <= bound), (what, i, nd.name, float((err / bound).max()))
+        else:
+            assert np.allclose(a, r, rtol=1e-4, atol=1e-6), (what, i, nd.name)
+
+
+def all_partitions(prog):
+    return legality.enumerate_partitions(prog.nodes, prog.outputs)

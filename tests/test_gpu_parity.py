@@ -1,0 +1,124 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the
+same seeded inputs, element by element, under every legal clustering of the small
+programs and under the unfused executor.  Sizes span several tiles and a ragged tail."""
+import numpy as np
+import pytest
+
+import workloads as W
+from helpers import all_partitions, compare, gpu_run, oracle_run
+
+pytestmark = pytest.mark.gpu
+
+
+def np_inputs(inputs_t):
+    return {k: v.cpu().numpy() for k, v in inputs_t.items()}
+
+
+def check_program(prog, partitions="all", runs=1):
+    from paper_2407_13585_b200 import binding as B
+    inputs_t = W.make_inputs(prog)
+    ref = oracle_run(prog, np_inputs(inputs_t))
+    got, g = gpu_run(prog, inputs_t, None, B.UNFUSED)
+    assert g.launch_count() == sum(nd.kind != "input" for nd in prog.nodes)
+    compare(prog, ref, got, f"{prog.name} unfused")
+    pis = all_partitions(prog) if partitions == "all" else partitions
+    for pi in pis:
+        got, g = gpu_run(prog, inputs_t, pi, B.FUSED, runs=runs)
+        assert g.launch_count() == len({c for c in pi if c >= 0})
+        compare(prog, ref, got, f"{prog.name} pi={pi}")
+    return len(pis)
+
+
+# several tiles plus a ragged tail; multiples of four (128-bit path) and not (scalar path)
+@pytest.mark.parametrize("n", [1, 3, 4, 31, 1024, 4099, 70000, 1 << 16])
+def test_config1_all_partitions(n):
+    assert check_program(W.config1(n)) == 8
+
+
+@pytest.mark.parametrize("rows", [1, 4, 33, 100, 256])
+def test_config2_all_partitions(rows):
+    assert check_program(W.config2(rows)) == 4
+
+
+@pytest.mark.parametrize("n", [1, 4, 64, 4096, 8192, 1 << 17])
+def test_config3_all_partitions(n):
+    assert check_program(W.config3(n)) == 8
+
+
+def test_config3_ragged_lengths():
+    # lengths that are not powers of two: the scan's last tile is partial, the scalar path runs
+    for n in (5, 4097, 12289 + 3):
+        prog = W.config3(n)
+        prog.name = "fixture"                     # generic index inputs bounded by n
+        prog.index_bound = {"idx": n, "x": 1 << 30}
+        check_program(prog)
+
+
+@pytest.mark.parametrize("rows,cols", [(1, 4), (3, 5), (8, 8), (33, 64), (64, 33), (130, 260)])
+def test_config4_iteration_cuts(rows, cols):
+    prog = W.config4(rows, cols, iters=2)
+    per_iter = [-1] + [0] * 9 + [1] * 9
+    cuts = [per_iter]
+    # {c,n,t1}, the other shifts alone, {t2,t3,Y}
+    cuts.append([-1, 0, 0, 1, 2, 3, 0, 4, 4, 4] + [c + 5 for c in (0, 0, 1, 2, 3, 0, 4, 4, 4)])
+    # shifts alone, the four sums fused
+    cuts.append([-1, 0, 1, 2, 3, 4, 5, 5, 5, 5] + [c + 6 for c in (0, 1, 2, 3, 4, 5, 5, 5, 5)])
+    check_program(prog, cuts)
+
+
+def test_config4_four_iterations_planned():
+    from paper_2407_13585_b200 import binding as B
+    prog = W.config4(96, 128, iters=4)
+    g = B.Graph(prog.nodes, prog.outputs)
+    for mode in ("greedy_topdown", "greedy_bottomup"):
+        pi = g.plan(mode)
+        assert len({c for c in pi if c >= 0}) == 4        # one cluster per iteration is the legal minimum
+        check_program(prog, [pi])
+
+
+@pytest.mark.parametrize("n,bins", [(1, 1), (7, 4), (1000, 16), (4096, 256), (100003, 1 << 10), (1 << 18, 1 << 16)])
+def test_config5_all_partitions(n, bins):
+    assert check_program(W.config5(n, bins)) == 10
+
+
+def test_runs_are_repeatable():
+    # a racy fold, scan or scatter would differ between runs; integer outputs must be identical
+    check_program(W.config3(1 << 16), runs=3)
+    check_program(W.config5(1 << 16, 256), runs=3)
+
+
+PAPER_EXAMPLES = [W.scatter_example(64), W.single_loop(100), W.simple1(), W.simple2(), W.simple4(), W.simple5(),
+                  W.greedy_bottom_up_bad(16, 100), W.greedy_top_down_bad(1000)]
+
+
+@pytest.mark.parametrize("prog", PAPER_EXAMPLES, ids=lambda p: p.name)
+def test_paper_examples_all_partitions(prog):
+    # the programs the paper prints (Sections 1, 3.3, 3.4, 5), under every legal clustering:
+    # gathers pushed through maps, gathers and a fold; a scatter fed by fused maps; two folds sharing a gather
+    assert check_program(prog) >= 2
+
+
+def test_empty_arrays_run():
+    # element-wise clusters over zero elements are legal no-ops (a fold over nothing is rejected when built)
+    prog = W.config4(0, 8, iters=1)
+    check_program(prog, [[-1] + [0] * 9])
+
+
+def test_scatter_out_of_range_is_reported():
+    import torch
+    from paper_2407_13585_b200 import binding as B
+    prog = W.config5(1024, 16)
+    g = B.Graph(prog.nodes, prog.outputs)
+    g.plan("enumerate")
+    # break the hash's modulus so that indices leave the 16 bins: the kernel must skip and report, not write
+    bad = W.config5(1024, 16)
+    bad.nodes[2].iparam = (40503, 64)
+    g = B.Graph(bad.nodes, bad.outputs)
+    g.plan("enumerate")
+    inputs = W.make_inputs(bad)
+    bufs = [inputs[0].cuda(), inputs[1].cuda(), torch.zeros(16, device="cuda"), torch.zeros(1, device="cuda"),
+            torch.zeros(16, device="cuda")]
+    g.bind(0, bufs[0]); g.bind(1, bufs[1]); g.bind(4, bufs[2]); g.bind(5, bufs[3]); g.bind(6, bufs[4])
+    with pytest.raises(B.AccError) as e:
+        g.run()
+    assert e.value.status == "ACC_ERR_INDEX_RANGE"

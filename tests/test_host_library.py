@@ -1,0 +1,216 @@
+"""Host side of the CUDA library (no GPU needed): the shared object loads and exports
+the declared C ABI, graph building validates, the legality checker and the enumerator
+agree with the oracle's independent model on the paper's programs and on random small
+graphs, and the planners behave as Section 5 of the paper describes."""
+import ctypes
+import os
+import random
+import re
+
+import pytest
+
+import workloads as W
+from workloads import Node
+from oracle import legality as L
+from paper_2407_13585_b200 import binding as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _inp(name, dtype="i32", shape=(8,)):
+    return Node("input", dtype, tuple(shape), name=name)
+
+
+def test_library_exports_every_declared_symbol():
+    text = re.sub(r"/\*.*?\*/", "", open(os.path.join(ROOT, "include", "acc.h")).read(), flags=re.S)
+    declared = set(re.findall(r"\b(acc_[a-z0-9_]+)\s*\(", text))
+    assert {"acc_graph_create", "acc_add_node", "acc_set_partition", "acc_run"} <= declared
+    lib = ctypes.CDLL(B.LIB_PATH)
+    for name in sorted(declared):
+        assert hasattr(lib, name), name
+    assert B.registry_size() >= 40
+
+
+PROGRAMS = [W.config1(64), W.config2(8), W.config3(64), W.config4(8, 8, iters=1), W.config5(256, 16),
+            W.scatter_example(16), W.scatter_example_paper_graph(), W.single_loop(16), W.simple1(), W.simple2(),
+            W.simple3(), W.simple4(), W.simple5(), W.greedy_bottom_up_bad(4, 5), W.greedy_top_down_bad(16)]
+
+
+@pytest.mark.parametrize("prog", PROGRAMS, ids=lambda p: p.name)
+def test_enumeration_equals_oracle(prog):
+    g = B.Graph(prog.nodes, prog.outputs)
+    assert g.enumerate() == L.enumerate_partitions(prog.nodes, prog.outputs)
+    F, I = g.edges()
+    oF, oI = L.graph_sets(prog.nodes)
+    assert set(F) - set(I) == oF and set(I) == oI
+
+
+def _random_program(rng):
+    nodes = [_inp("a"), _inp("b")]
+    for _ in range(rng.randint(2, 5)):
+        k = rng.choice(["map", "map", "zipwith", "backpermute", "gather", "scanl", "scanr", "permute"])
+        pick = lambda: rng.randrange(len(nodes))
+        force = (0,) if rng.random() < 0.15 else ()
+        if k == "map":
+            nodes.append(Node("map", "i32", (8,), (pick(),), 1, fn="identity", force=force))
+        elif k == "zipwith":
+            nodes.append(Node("zipwith", "i32", (8,), (pick(), pick()), 2, fn="add", force=force))
+        elif k == "backpermute":
+            nodes.append(Node("backpermute", "i32", (8,), (pick(),), 1, idx_fn="reverse"))
+        elif k == "gather":
+            nodes.append(Node("gather", "i32", (8,), (pick(), pick()), 2))
+        elif k in ("scanl", "scanr"):
+            nodes.append(Node(k, "i32", (8,), (pick(),), 1, fn="add"))
+        else:
+            nodes.append(Node("permute", "i32", (8,), (pick(), pick(), pick()), 3, fn="add"))
+    used = {s for nd in nodes for s in nd.inputs}
+    outputs = [i for i in range(2, len(nodes)) if i not in used] or [len(nodes) - 1]
+    if rng.random() < 0.3:
+        outputs.append(rng.randrange(2, len(nodes)))
+    return nodes, sorted(set(outputs))
+
+
+def test_checker_equals_oracle_on_random_graphs():
+    rng = random.Random(1234)
+    total = 0
+    for _ in range(150):
+        nodes, outputs = _random_program(rng)
+        g = B.Graph(nodes, outputs)
+        mine, ref = g.enumerate(), L.enumerate_partitions(nodes, outputs)
+        assert mine == ref, (nodes, outputs)
+        total += len(ref)
+        # and on arbitrary (mostly illegal) numberings
+        for _ in range(10):
+            pi = [-1, -1] + [rng.randrange(len(nodes) - 2) for _ in range(len(nodes) - 2)]
+            assert (g.check_partition(pi) == "ACC_OK") == L.check(nodes, outputs, pi)[0], (nodes, outputs, pi)
+    assert total > 500
+
+
+def test_check_partition_names_the_broken_rule():
+    p = W.scatter_example_paper_graph()
+    g = B.Graph(p.nodes, p.outputs)
+    assert g.check_partition([-1, 0, 1, 1]) == "ACC_ERR_ILLEGAL_INFUSIBLE"
+    assert g.check_partition([-1, 1, 2, 0]) == "ACC_ERR_ILLEGAL_ORDER"
+    q = W.simple3()
+    assert B.Graph(q.nodes, q.outputs).check_partition([-1, -1, 0, 0]) == "ACC_ERR_ILLEGAL_TRAVERSAL"
+    nodes = [_inp("a"), _inp("b"), Node("map", "i32", (8,), (0,), 1, fn="identity"), Node("map", "i32", (8,), (1,), 1, fn="identity")]
+    assert B.Graph(nodes, [2, 3]).check_partition([-1, -1, 0, 0]) == "ACC_ERR_DISCONNECTED"
+    nodes = [_inp("xs"), Node("map", "i32", (8,), (0,), 1, fn="identity"), Node("map", "i32", (8,), (0,), 1, fn="identity"),
+             Node("map", "i32", (8,), (2,), 1, fn="identity"), Node("permute", "i32", (8,), (2, 1, 1), 3, fn="add")]
+    assert B.Graph(nodes, [3, 4]).check_partition([-1, 0, 0, 2, 1]) == "ACC_ERR_ILLEGAL_SCATTER"
+    with pytest.raises(B.AccError) as e:
+        g.set_partition([-1, 0, 1, 1])
+    assert e.value.status == "ACC_ERR_ILLEGAL_INFUSIBLE" and "infusible" in str(e.value)
+    with pytest.raises(B.AccError):
+        g.set_partition([0, 0, 0])                      # wrong length
+
+
+def test_set_partition_and_manifest():
+    p = W.config1(64)
+    g = B.Graph(p.nodes, p.outputs)
+    with pytest.raises(B.AccError) as e:
+        g.get_partition()
+    assert e.value.status == "ACC_ERR_NO_PARTITION"
+    g.set_partition([7, 0, 0, 1, 1])
+    assert g.get_partition() == [-1, 0, 0, 1, 1]
+    assert g.manifest() == [True, False, True, False, True]      # y fused into z, w into s
+
+
+def test_add_node_validation():
+    g = B.Graph()
+    x = g.add_node(_inp("x", "f32", (4, 6)))
+    bad = [
+        Node("map", "f32", (4, 5), (x,), 1, fn="affine"),                          # shape
+        Node("map", "f32", (4, 6), (x,), 1, fn="mul"),                             # arity
+        Node("map", "f32", (4, 6), (3,), 1, fn="affine"),                          # unknown input
+        Node("backpermute", "f32", (4, 6), (x,), 1, idx_fn="transpose"),           # transpose needs (6,4)
+        Node("fold", "f32", (6,), (x,), 1, fn="add"),                              # outer extent
+        Node("fold", "f32", (4,), (x,), 1, fn="affine"),                           # not a combine operator
+        Node("gather", "f32", (4, 6), (x, x), 2),                                  # float index array
+        Node("scanl", "f32", (4, 5), (x,), 1, fn="add"),
+    ]
+    for nd in bad:
+        with pytest.raises(B.AccError):
+            g.add_node(nd)
+    empty = g.add_node(_inp("e", "f32", (3, 0)))
+    with pytest.raises(B.AccError) as e:
+        g.add_node(Node("fold", "f32", (3,), (empty,), 1, fn="add"))              # fold without a seed over nothing
+    assert e.value.status == "ACC_ERR_SHAPE"
+    d = B.make_desc(Node("map", "f32", (4, 6), (x,), 1, fn="affine"))
+    d.kind = B.KIND["foldseg"]
+    with pytest.raises(B.AccError) as e:
+        g.add_node(d)
+    assert e.value.status == "ACC_ERR_UNSUPPORTED"
+    assert g.n == 2
+
+
+def test_planner_enumerate_finds_the_paper_optima():
+    p = W.greedy_bottom_up_bad(16, 1000)
+    g = B.Graph(p.nodes, p.outputs)
+    best = g.plan("enumerate", "bytes")
+    assert best == [-1, 0, 0, 0, 0, 1]                   # `large` contracted: gather and both folds in one cluster
+    bu = g.plan("greedy_bottomup")
+    assert bu[3] == bu[5] and bu[4] != bu[3]             # ys went with result first; zs cannot join any more
+    g.set_partition(bu)
+    assert g.manifest()[2]                               # ... so `large` is written to memory
+    assert g.partition_cost(bu) > 5 * g.partition_cost(best)
+    assert g.plan("greedy_topdown") == best
+
+    q = W.greedy_top_down_bad(4096)
+    h = B.Graph(q.nodes, q.outputs)
+    best = h.plan("enumerate", "bytes")
+    assert best == [-1, 0, 1, 1, 1, 1]                   # cs fused vertically into es
+    td = h.plan("greedy_topdown")
+    assert td[1] == td[2] and td[2] != td[4]             # cs fused diagonally with bs instead
+    assert h.partition_cost(td) > h.partition_cost(best)
+    assert h.plan("greedy_bottomup") == best
+
+
+def test_planner_scatter_example_prefers_fusing_into_the_scatter():
+    p = W.scatter_example_paper_graph()
+    g = B.Graph(p.nodes, p.outputs)
+    assert g.plan("enumerate", "reads_writes") == [-1, 1, 0, 1]       # Figure 4, right-hand clustering
+
+
+def _bytes_of(nd):
+    c = 1
+    for e in nd.shape:
+        c *= e
+    return 4 * max(1, c)
+
+
+def test_costs_agree_with_oracle_traffic():
+    for prog in (W.config1(64), W.config5(256, 16), W.simple5(), W.single_loop(16), W.config2(8)):
+        g = B.Graph(prog.nodes, prog.outputs)
+        for pi in L.enumerate_partitions(prog.nodes, prog.outputs):
+            r, w = L.traffic(prog.nodes, prog.outputs, pi)
+            assert g.partition_cost(pi, "reads") == r, (prog.name, pi)
+            assert g.partition_cost(pi, "reads_writes") == r + w
+            assert g.partition_cost(pi, "arrays") == w
+            assert g.partition_cost(pi, "clusters") == len({c for c in pi if c >= 0})
+            rb, wb = L.traffic(prog.nodes, prog.outputs, pi, weight=_bytes_of)
+            assert g.partition_cost(pi, "bytes") == rb + wb
+
+
+def test_greedy_on_jacobi_finds_one_cluster_per_iteration():
+    p = W.config4(64, 64, iters=4)
+    g = B.Graph(p.nodes, p.outputs)
+    for mode in ("greedy_topdown", "greedy_bottomup"):
+        pi = g.plan(mode)
+        assert L.check(p.nodes, p.outputs, pi)[0]
+        blocks = [pi[1 + 9 * t: 10 + 9 * t] for t in range(4)]
+        assert all(len(set(b)) == 1 for b in blocks) and len({b[0] for b in blocks}) == 4
+    with pytest.raises(B.AccError) as e:
+        g.plan("enumerate")
+    assert e.value.status == "ACC_ERR_TOO_LARGE"
+
+
+def test_unbound_buffers_are_reported_without_a_device():
+    p = W.config1(1 << 10)
+    g = B.Graph(p.nodes, p.outputs)
+    with pytest.raises(B.AccError) as e:
+        g.workspace_bytes(B.UNFUSED)
+    assert e.value.status == "ACC_ERR_UNBOUND"           # input and output buffers come from the caller
+    with pytest.raises(B.AccError) as e:
+        g.workspace_bytes(B.FUSED)
+    assert e.value.status == "ACC_ERR_NO_PARTITION"
