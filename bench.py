@@ -1,0 +1,366 @@
+"""Benchmark of the fused-cluster executor on the five synthetic programs.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One step = one pass of all five programs (1-D chain, transpose-fuse-reduce, random
+gather + scan, four Jacobi iterations, scatter histogram + diamond) through
+`acc_run(FUSED)` under the planner's clustering.  The metric is effective HBM
+bandwidth: compulsory bytes (every program input read once + every program output
+written once) divided by device time.  Rank 0 prints one JSON line.
+
+With N > 1 every rank runs an independent replica on its own GPU (the path has no
+exchange step); the value is the sum of bytes over ranks divided by the slowest rank.
+`--impl reference` times the CPU oracle on a bounded sample of the same programs.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "fused-pipeline effective HBM bandwidth (compulsory bytes / time), 5 synthetic programs"
+FULL = {1: dict(n=1 << 16), 2: dict(rows=8192), 3: dict(n=1 << 26), 4: dict(rows=8192), 5: dict(n=1 << 27)}
+SAMPLE = {1: dict(n=1 << 16), 2: dict(rows=4096), 3: dict(n=1 << 24), 4: dict(rows=4096), 5: dict(n=1 << 25)}
+ORDER = [2, 3, 4, 5, 1]
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def count_of(nd):
+    c = 1
+    for e in nd.shape:
+        c *= int(e)
+    return c
+
+
+def compulsory_bytes(prog):
+    ins = sum(count_of(prog.nodes[i]) for i in prog.input_ids())
+    outs = sum(count_of(prog.nodes[i]) for i in prog.outputs)
+    return 4 * (ins + outs)
+
+
+def elements_of(prog):
+    return max(count_of(nd) for nd in prog.nodes)
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(index), "--query-gpu=" + self.QUERY, "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            text, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            return out
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in text.splitlines():
+            f = [t.strip() for t in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+class Workload:
+    """One program at one size: graph, device buffers, pinned host mirrors."""
+
+    def __init__(self, cfg, sizes, device, host=True):
+        import torch
+        import workloads as W
+        from paper_2407_13585_b200 import binding as B
+        self.cfg = cfg
+        self.prog = W.CONFIGS[cfg](**sizes)
+        self.bytes = compulsory_bytes(self.prog)
+        self.elements = elements_of(self.prog)
+        self.g = B.Graph(self.prog.nodes, self.prog.outputs)
+        n_ops = sum(nd.kind != "input" for nd in self.prog.nodes)
+        self.plan_mode = "enumerate" if n_ops <= 12 else "greedy_topdown"
+        self.pi = self.g.plan(self.plan_mode, "bytes")
+        self.inputs = W.make_inputs(self.prog, device=device)
+        self.outputs = {}
+        self.host = {}
+        for i, t in self.inputs.items():
+            self.g.bind(i, t)
+            if host:
+                h = torch.empty(t.shape, dtype=t.dtype, pin_memory=True)
+                h.copy_(t)
+                self.host[i] = h
+                self.g.bind_host(i, h)
+        for o in self.prog.outputs:
+            nd = self.prog.nodes[o]
+            dt = torch.float32 if nd.dtype == "f32" else torch.int32
+            t = torch.empty(max(count_of(nd), 4), dtype=dt, device=device)
+            self.outputs[o] = t
+            self.g.bind(o, t)
+            if host:
+                h = torch.empty(max(count_of(nd), 4), dtype=dt, pin_memory=True)
+                self.host[o] = h
+                self.g.bind_host(o, h)
+        self.ws = {}
+        self.B = B
+
+    def run(self, executor):
+        # each executor keeps its own workspace so that switching does not reallocate
+        g = self.g
+        if executor not in self.ws:
+            g.workspace = None
+            self.ws[executor] = g.ensure_workspace(executor)
+        g.workspace = self.ws[executor]
+        g.run(executor, finish=False)
+
+    def finish(self):
+        self.g.finish()
+
+
+def time_region(fn, reps):
+    import torch
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    start.record()
+    for _ in range(reps):
+        fn()
+    end.record()
+    torch.cuda.synchronize()
+    return start.elapsed_time(end) / reps
+
+
+def oracle_sample_time():
+    """Runs the oracle once on the bounded sample of every program; returns (bytes, seconds, description)."""
+    import workloads as W
+    from oracle import interp
+    total_b, total_s = 0, 0.0
+    for cfg in ORDER:
+        prog = W.CONFIGS[cfg](**SAMPLE[cfg])
+        inputs = {k: v.numpy() for k, v in W.make_inputs(prog).items()}
+        t0 = time.perf_counter()
+        interp.run(prog.nodes, inputs)
+        total_s += time.perf_counter() - t0
+        total_b += compulsory_bytes(prog)
+        del inputs
+    desc = "oracle.interp on configs 2-5 at 1/4 of the elements (4096^2, 2^24, 4096^2 x 4 iterations, 2^25) and config 1 in full"
+    return total_b, total_s, desc
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample_time()
+    steps = max(1, min(args.steps, 3))
+    tb = ts = 0.0
+    desc = ""
+    for _ in range(steps):
+        b, s, desc = oracle_sample_time()
+        tb += b
+        ts += s
+    value = tb / ts / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus, "steps": steps,
+        "warmup": min(args.warmup, 1), "ms_per_step": ts / steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32/i32", "data": "synthetic",
+        "config": {"workload": "configs 1-5 back to back (bounded sample)", "sample": desc},
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2407_13585_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    loads = [Workload(cfg, FULL[cfg], device) for cfg in ORDER]
+    step_bytes = sum(w.bytes for w in loads)
+
+    def step():
+        for w in loads:
+            w.run(B.FUSED)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    for w in loads:
+        w.finish()
+
+    barrier()
+    sampler = ClockSampler(local) if rank == 0 else None
+    ms_step = time_region(step, args.steps)
+    clocks = sampler.stop() if sampler else {}
+    barrier()
+    launches = sum(w.g.launch_count() for w in loads)
+    for w in loads:
+        w.finish()
+    if world > 1:
+        t = torch.tensor([ms_step], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_step = float(t.item())
+    value = world * step_bytes / (ms_step * 1e-3) / 1e9
+
+    # per program: fused and unfused executors side by side (rank 0's GPU)
+    per = {}
+    reps = max(3, min(args.steps, 20))
+    for w in loads:
+        for _ in range(3):
+            w.run(B.FUSED)
+        ms_f = time_region(lambda: w.run(B.FUSED), reps)
+        n_f = w.g.launch_count()
+        w.finish()
+        for _ in range(3):
+            w.run(B.UNFUSED)
+        ms_u = time_region(lambda: w.run(B.UNFUSED), reps)
+        n_u = w.g.launch_count()
+        w.finish()
+        w.ws.pop(B.UNFUSED, None)
+        w.g.workspace = w.ws[B.FUSED]
+        torch.cuda.empty_cache()
+        per[w.cfg] = {
+            "clustering": w.pi, "planner": w.plan_mode, "ms_fused": ms_f, "ms_unfused": ms_u, "speedup": ms_u / ms_f,
+            "launches_fused": n_f, "launches_unfused": n_u, "compulsory_bytes": w.bytes,
+            "effective_gbs": w.bytes / ms_f / 1e6, "pct_of_8TBs": 100.0 * w.bytes / ms_f / 1e6 / NOMINAL_HBM_GBS,
+            "gelem_s": w.elements / ms_f / 1e6,
+        }
+
+    # end to end: pinned host inputs in, outputs out, every step
+    def e2e_step():
+        up = down = 0
+        for w in loads:
+            w.g.workspace = w.ws[B.FUSED]
+            u, d = w.g.run_e2e(B.FUSED)
+            up, down = up + u, down + d
+        return up, down
+
+    e2e_step()
+    barrier()
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    e2e_reps = max(1, min(args.steps, 5))
+    for _ in range(e2e_reps):
+        up, down = e2e_step()
+    t1.record()
+    torch.cuda.synchronize()
+    ms_e2e = t0.elapsed_time(t1) / e2e_reps
+    if world > 1:
+        t = torch.tensor([ms_e2e], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item())
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # the kernel that takes the largest share of a step
+    kernel_bytes = {2: lambda w: w.bytes, 3: lambda w: w.bytes, 4: lambda w: 8 * w.elements, 5: lambda w: w.bytes, 1: lambda w: w.bytes}
+    kernel_launches = {2: 1, 3: 1, 4: 4, 5: 1, 1: 1}
+    top = max(per, key=lambda c: per[c]["ms_fused"])
+    wtop = [w for w in loads if w.cfg == top][0]
+    peak, peak_kind = measured_peak()
+    achieved = kernel_bytes[top](wtop) / (per[top]["ms_fused"] / kernel_launches[top]) / 1e6
+    names = {2: "k_rowfold<transpose+zip+fold>", 3: "k_scan<hash+gather+mask+scan>", 4: "k_stream<jacobi iteration>",
+             5: "k_stream<hash+generate+permute+fold>", 1: "k_stream<chain>"}
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": None, "kernel": names[top], "of": peak_kind,
+                "bytes_per_launch": kernel_bytes[top](wtop), "launches_per_step": kernel_launches[top]}
+
+    cpu = None
+    if world == 1:
+        b, s, desc = oracle_sample_time()
+        cpu = {"value": b / s / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": desc, "seconds": s}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32/i32", "data": "synthetic",
+        "config": {"workload": "configs 1-5 back to back, full sizes (2^16; 8192^2; 2^26; 8192^2 x 4 iterations; 2^27 keys, 2^16 bins)",
+                   "l2": "every program but config 1 streams more than the 126 MB L2 between reuses; no explicit flush",
+                   "parallelism": "replicas only" if world > 1 else "1 GPU", "compulsory_bytes_per_step": step_bytes},
+        "pct_of_8TBs": 100.0 * value / world / NOMINAL_HBM_GBS,
+        "clocks": {"sm_mhz": clocks.get("sm_mhz"), "sm_max_mhz": clocks.get("sm_max_mhz"), "reasons": clocks.get("reasons", []),
+                   "samples": clocks.get("samples", 0)},
+        "e2e": {"value": world * step_bytes / (ms_e2e * 1e-3) / 1e9, "unit": "GB/s", "h2d_bytes_per_step": up,
+                "d2h_bytes_per_step": down, "ms_per_step": ms_e2e},
+        "gpu_launches": launches * args.steps,
+        "roofline": roofline,
+        "cpu_baseline": cpu,
+        "per_config": per,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
