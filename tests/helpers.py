@@ -86,7 +86,9 @@ def compare(prog, ref, got, what=""):
             bound = ((TOL * ref.abs_sum[h] + np.abs(frac) * TOL * float(ref.abs_sum[t])) / abs(te)
                      + np.abs(frac) * 2.0 ** -22 + 1e-30)
             err = np.abs(a.astype(np.float64) - frac)
-            assert np.all(err <= bound), (what, i, nd.name, float((err / bound).max()))
+            undefined = np.isnan(frac)             # 0/0 when the total is zero: both sides must say so
+            assert np.array_equal(np.isnan(a), undefined), (what, i, nd.name)
+            assert np.all((err <= bound) | undefined), (what, i, nd.name, float(np.nanmax(err / bound)))
         else:
             assert np.allclose(a, r, rtol=1e-4, atol=1e-6), (what, i, nd.name)
 

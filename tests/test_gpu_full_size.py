@@ -1,0 +1,88 @@
+"""GPU parity at the benchmark's full sizes, in the configuration bench.py times: the
+planner's clustering, the fused executor, inputs drawn on the device.  Configs 2, 3 and 5
+are compared with the oracle on every output element; config 4 on row bands (top edge,
+middle, bottom edge) that the oracle recomputes from the same input rows."""
+import numpy as np
+import pytest
+
+import workloads as W
+from helpers import compare, oracle_run
+
+pytestmark = pytest.mark.gpu
+
+
+def run_full(prog, mode):
+    import torch
+    from paper_2407_13585_b200 import binding as B
+    g = B.Graph(prog.nodes, prog.outputs)
+    pi = g.plan(mode, "bytes")
+    inputs = W.make_inputs(prog, device="cuda")
+    for i, t in inputs.items():
+        g.bind(i, t)
+    outs = {}
+    for o in prog.outputs:
+        nd = prog.nodes[o]
+        cnt = int(np.prod(nd.shape, dtype=np.int64)) if nd.shape else 1
+        outs[o] = torch.full((max(cnt, 4),), -1, dtype=torch.int32, device="cuda")
+        g.bind(o, outs[o])
+    g.run(B.FUSED)
+    g.run(B.FUSED)                     # a second run over the same workspace must give the same arrays
+    torch.cuda.synchronize()
+    got = {}
+    for o, t in outs.items():
+        nd = prog.nodes[o]
+        cnt = int(np.prod(nd.shape, dtype=np.int64)) if nd.shape else 1
+        a = t[:cnt].cpu().numpy()
+        got[o] = (a.view(np.float32) if nd.dtype == "f32" else a.view(np.uint32)).reshape(tuple(nd.shape))
+    return got, inputs, pi, g
+
+
+def test_config2_full():
+    prog = W.config2(8192)
+    got, inputs, pi, g = run_full(prog, "enumerate")
+    assert pi == [-1, 0, 0, 0] and g.launch_count() == 1
+    ref = oracle_run(prog, {k: v.cpu().numpy() for k, v in inputs.items()})
+    compare(prog, ref, got, "config2 full")
+
+
+def test_config3_full():
+    prog = W.config3(1 << 26)
+    got, inputs, pi, g = run_full(prog, "enumerate")
+    assert pi == [-1, -1, 0, 0, 0, 0] and g.launch_count() == 1
+    ref = oracle_run(prog, {k: v.cpu().numpy() for k, v in inputs.items()})
+    compare(prog, ref, got, "config3 full")
+
+
+def test_config5_full():
+    prog = W.config5(1 << 27, 1 << 16)
+    got, inputs, pi, g = run_full(prog, "enumerate")
+    assert pi == [-1, -1, 0, 0, 0, 0, 1] and g.launch_count() == 2
+    ref = oracle_run(prog, {k: v.cpu().numpy() for k, v in inputs.items()})
+    compare(prog, ref, got, "config5 full")
+    # the hottest bin holds far more than 2^24: plain fp32 accumulation would have lost its small addends
+    assert ref.exact[4].max() > 2 ** 24
+
+
+def test_config1_full():
+    prog = W.config1(1 << 16)
+    got, inputs, pi, g = run_full(prog, "enumerate")
+    assert g.launch_count() == 1
+    ref = oracle_run(prog, {k: v.cpu().numpy() for k, v in inputs.items()})
+    compare(prog, ref, got, "config1 full")
+
+
+def test_config4_full_on_row_bands():
+    rows = cols = 8192
+    iters = 4
+    prog = W.config4(rows, cols, iters)
+    got, inputs, pi, g = run_full(prog, "greedy_topdown")
+    assert g.launch_count() == iters
+    X = inputs[0]
+    Y = got[prog.outputs[0]]
+    for lo, hi in ((0, 48), (4000, 4040), (rows - 48, rows)):
+        # the band plus `iters` halo rows on each open side determines the band's output exactly
+        a, b = max(0, lo - iters), min(rows, hi + iters)
+        sub = W.config4(b - a, cols, iters)
+        ref = oracle_run(sub, {0: X[a:b].cpu().numpy()})
+        want = ref.values[sub.outputs[0]][lo - a: hi - a]
+        assert np.array_equal(Y[lo:hi].view(np.uint32), want.view(np.uint32)), (lo, hi)
