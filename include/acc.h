@@ -232,6 +232,40 @@ int32_t acc_launch_count(const acc_graph* g);
  * copied into buf (truncated to cap-1 characters). */
 int acc_last_schedule(const acc_graph* g, char* buf, size_t cap);
 
+/* Inclusive left-to-right prefix sum of n int32 values with wrap-around,
+ * out[i] = in[0] + ... + in[i], for callers that cannot give the library a
+ * workspace.  (The paper has no counterpart: this is a packaging variant of
+ * the scan kernel, not a combinator or a rule of its own.)
+ *
+ * Who needs it: code that may not allocate device memory where it calls us --
+ * a serving or real-time loop in which cudaMalloc's implicit device-wide
+ * synchronisation is unacceptable, a plug-in or callback that receives raw
+ * device pointers but no allocator, a process whose memory budget is fixed
+ * up front.  acc_run needs a caller-allocated workspace for the scan's tile
+ * states; this entry point keeps them in a fixed array inside the library's
+ * device image instead (about 128 KiB, resident on every GPU that loads the
+ * library until the process exits) and calls no cudaMalloc, cudaFree or any
+ * other allocating routine.
+ *
+ *   in, out      DEVICE pointers to n int32 each, owned by the caller, not
+ *                overlapping; 16-byte alignment and n % 4 == 0 select the
+ *                128-bit path, anything else the scalar one.
+ *   n            0 .. ACC_STATIC_SCAN_MAX_ELEMENTS; more is refused with
+ *                ACC_ERR_TOO_LARGE and nothing is launched.
+ *   cuda_stream  a cudaStream_t of the current device (null = default stream).
+ *
+ * The call enqueues a clear of the part of the array it uses and the scan, then
+ * WAITS for the stream and returns ACC_OK, ACC_ERR_DEVICE_TIMEOUT (a bounded
+ * wait between tiles ran out; out is then not valid) or ACC_ERR_CUDA.
+ * The first call on each device looks up the array's device address (with
+ * that device current); make that first call outside any stream capture.
+ * All calls on one GPU share the one array, which keeps the previous call's
+ * contents between calls: two calls whose work overlaps on the same GPU
+ * (different streams or threads) race on it and give undefined results --
+ * serialise them.  Calls on different GPUs are independent. */
+#define ACC_STATIC_SCAN_MAX_ELEMENTS (1ll << 26)
+int acc_scanl_add_i32_static(const int32_t* in, int32_t* out, int64_t n, void* cuda_stream);
+
 /* Message for the last failing call on this thread ("" if none). */
 const char* acc_last_error(void);
 /* Number of build-time kernel instantiations in the registry. */

@@ -92,6 +92,7 @@ def load_library(path=LIB_PATH):
         "acc_run_e2e": (C.c_int, [p, p, sz, p, C.c_int, C.POINTER(sz), C.POINTER(sz)]),
         "acc_launch_count": (i32, [p]),
         "acc_last_schedule": (C.c_int, [p, C.c_char_p, sz]),
+        "acc_scanl_add_i32_static": (C.c_int, [p, p, i64, p]),
         "acc_last_error": (C.c_char_p, []),
         "acc_registry_size": (i32, []),
     }
@@ -278,6 +279,17 @@ class Graph:
         buf = C.create_string_buffer(4096)
         lib().acc_last_schedule(self._h, buf, 4096)
         return buf.value.decode()
+
+
+def scanl_add_i32_static(src, dst):
+    """acc_scanl_add_i32_static on two int32 CUDA tensors: inclusive wrapping prefix sum of `src`
+    into `dst` using the library's built-in scratch array.  Nothing is allocated here or in the
+    library, so it can be called from code that must not touch the device allocator.  Waits for
+    the current stream; calls that overlap on one GPU race on the shared scratch."""
+    assert src.is_cuda and dst.is_cuda and src.is_contiguous() and dst.is_contiguous()
+    assert src.element_size() == 4 and dst.numel() >= src.numel()
+    _check(lib().acc_scanl_add_i32_static(C.c_void_p(src.data_ptr()), C.c_void_p(dst.data_ptr()), src.numel(),
+                                          Graph._stream()))
 
 
 def registry_size():
