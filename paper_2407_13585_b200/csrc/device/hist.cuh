@@ -1,0 +1,217 @@
+// k_hist: the skeleton for a cluster whose permute is an fp32 '+' scatter into few enough
+// bins to keep them on chip.
+//
+// Measured on B200: shared-memory integer atomics sustain about 1000 G updates/s on a
+// Zipf-skewed key stream, fp32 shared-memory atomics about 56 G/s (they retry on every
+// collision, and a hot bin collides all the time), atomics into a partner CTA's shared
+// memory 140 G/s.  So the bins are 32-bit *integers* in the CTA's own shared memory:
+//
+//  * a value x is added as the integer x * 2^S when that product is an integer below 2^19
+//    in magnitude -- exact, one native atomic.  S is picked per CTA from the largest
+//    magnitude among the first elements it sees;
+//  * any other value (not a multiple of 2^-S, too large, not finite) is added to the global
+//    fp64 accumulator of its bin directly -- exact as well, slower;
+//  * a bin that reaches 2^29 in magnitude is emptied into its fp64 accumulator by the thread
+//    that crossed the line, so bins never overflow;
+//  * at the end every CTA adds its bins into the fp64 accumulators, and the block that
+//    finishes last turns those into the fp32 result on top of the defaults.
+//
+// Every partial sum is exact, so the result is the fp32 rounding of the exact fp64-combined
+// sum whatever the order of arrival.  When the bins of one scatter exceed one CTA's shared
+// memory, a group of G = 2, 4 or 8 neighbouring CTAs splits them: all CTAs of a group walk
+// the same elements (the second reader hits L2) and each updates only the bins it owns.
+// Store roots and whole-array folds of an element are handled by one CTA of the group.
+#pragma once
+#include "skeletons.cuh"
+
+namespace acc {
+namespace dev {
+
+constexpr int kHistBlock = 1024;
+constexpr int kHistMaxBinsPerCta = 56 * 1024;   // 224 KiB of 32-bit bins per CTA
+constexpr int kHistUnroll = 2;                  // independent chunks in flight per thread
+constexpr int kHistElementCap = 1 << 19;        // largest |x * 2^S| taken on the integer path
+constexpr int kHistSpillAt = 1 << 29;           // a bin is emptied once it reaches this magnitude
+
+template <class CL> constexpr int the_f32_add_permute() {
+  for (int i = 0; i < CL::c.n; ++i)
+    if (is_f32_add_permute(CL::c.nodes[i])) return i;
+  return -1;
+}
+
+template <class CL, bool VEC>
+__global__ void __launch_bounds__(kHistBlock, 1)
+k_hist(const __grid_constant__ Args<CL::c.n> a, int per_cta, int per_cta_shift, int group) {
+  constexpr int N = CL::c.n;
+  constexpr int W = VEC ? 4 : 1;
+  constexpr int U = kHistUnroll;
+  constexpr int DR = domain_rank<CL>();
+  constexpr int NF = count_if<CL>(is_scalar_fold);
+  constexpr int P = the_f32_add_permute<CL>();
+  static_assert(P >= 0, "k_hist needs an fp32 '+' permute");
+  constexpr CNode pn = CL::c.nodes[P];
+  using IX = std::conditional_t<VEC, Ix4, Ix>;
+  using VAL = val_of<IX>;
+  extern __shared__ int bins_smem[];
+  __shared__ uint32_t red[kHistBlock / 32];
+  __shared__ bool last_block;
+  __shared__ float sample_max;
+
+  const uint32_t rank = blockIdx.x % (uint32_t)group;          // which slice of the bins this CTA owns
+  const uint32_t team = blockIdx.x / (uint32_t)group;          // which share of the elements its group walks
+  const uint32_t n_teams = gridDim.x / (uint32_t)group;
+  for (int i = threadIdx.x; i < per_cta; i += kHistBlock) bins_smem[i] = 0;
+
+  uint32_t acc[N];
+  static_for<0, N>([&](auto ic) {
+    constexpr int i = decltype(ic)::value;
+    constexpr CNode nd = CL::c.nodes[i];
+    if constexpr (is_scalar_fold(nd)) acc[i] = identity_of<nd.fn, nd.dtype>();
+  });
+  const uint32_t n_bins = (uint32_t)(a.n[P].R * a.n[P].C);
+  const uint32_t per_row = (uint32_t)a.C / W;
+  const uint32_t total = (uint32_t)a.R * per_row;
+  const uint32_t stride = n_teams * kHistBlock;
+  double* acc64 = reinterpret_cast<double*>(a.scratch + stream_acc64_off(NF, a.grid));
+
+  auto index_of = [&](uint32_t q) {
+    IX ix;
+    if constexpr (DR <= 1) { ix.r = 0; ix.c = (int)(q * W); }
+    else { const uint32_t r = q / per_row; ix.r = (int)r; ix.c = (int)((q - r * per_row) * W); }
+    return ix;
+  };
+
+  // scale: the first chunk of every thread gives the magnitude to expect
+  {
+    float m = 0.0f;
+    const uint32_t q = team * kHistBlock + threadIdx.x;
+    if (q < total) {
+      const VAL v = eval<CL, pn.in[2]>(a, index_of(q));
+      if constexpr (VEC) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) m = fmaxf(m, fabsf(f_(v.v[j])));
+      } else {
+        m = fabsf(f_(v));
+      }
+    }
+    if (!(m < 3.0e38f)) m = 0.0f;                              // ignore infinities and NaNs here
+    const uint32_t top = block_reduce_n<ACC_FN_MAX, ACC_F32, kHistBlock>(u_(m), red);
+    if (threadIdx.x == 0) sample_max = f_(top);
+  }
+  __syncthreads();
+  int S = 0;
+  if (sample_max > 0.0f) {
+    int e;
+    frexpf(sample_max, &e);                                    // sample_max = f * 2^e, f in [0.5, 1)
+    S = min(max(18 - e, -100), 100);                           // sample_max * 2^S in [2^17, 2^18)
+  }
+  const float up = exp2f((float)S);
+  const double down = exp2((double)-S);
+
+  auto scatter_one = [&](uint32_t k, uint32_t xbits) {
+    if (k >= n_bins) { atomicOr(a.status, kStatusIndex); return; }
+    const uint32_t owner = per_cta_shift >= 0 ? (k >> per_cta_shift) : (k / (uint32_t)per_cta);
+    if (owner != rank) return;
+    const float x = f_(xbits);
+    if (x == 0.0f) return;
+    const float t = __fmul_rn(x, up);                          // exact whenever |t| >= 1 (no underflow)
+    if (fabsf(t) >= 1.0f && fabsf(t) < (float)kHistElementCap && t == rintf(t)) {
+      const int v = (int)t;
+      int* slot = bins_smem + (k - owner * (uint32_t)per_cta);
+      const int old = atomicAdd(slot, v);
+      if (abs(old + v) >= kHistSpillAt && abs(old) < kHistSpillAt) {
+        const int taken = atomicExch(slot, 0);
+        atomicAdd(acc64 + k, (double)taken * down);
+      }
+    } else {
+      atomicAdd(acc64 + k, (double)x);
+    }
+  };
+
+  uint32_t it = 0;
+  for (uint32_t q0 = team * kHistBlock + threadIdx.x; q0 < total; q0 += stride * U, it += U) {
+    // evaluate U independent chunks first so that their loads are in flight together
+    VAL key[U], val[U];
+    bool live[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const uint32_t q = q0 + u * stride;
+      live[u] = q < total;
+      if (live[u]) {
+        const IX ix = index_of(q);
+        key[u] = eval<CL, pn.in[1]>(a, ix);
+        val[u] = eval<CL, pn.in[2]>(a, ix);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      if (!live[u]) continue;
+      if ((it + u) % (uint32_t)group == rank) {                // this CTA's turn for the element-wise side
+        const IX ix = index_of(q0 + u * stride);
+        static_for<0, N>([&](auto ic) {
+          constexpr int i = decltype(ic)::value;
+          constexpr CNode nd = CL::c.nodes[i];
+          if constexpr (is_store_root(nd)) {
+            st(reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr)), a.n[i].C, ix, eval<CL, i>(a, ix));
+          } else if constexpr (is_scalar_fold(nd)) {
+            const auto v = eval<CL, nd.in[0]>(a, ix);
+            if constexpr (VEC) {
+#pragma unroll
+              for (int j = 0; j < 4; ++j) acc[i] = combine<nd.fn, nd.dtype>(acc[i], v.v[j]);
+            } else {
+              acc[i] = combine<nd.fn, nd.dtype>(acc[i], v);
+            }
+          }
+        });
+      }
+      if constexpr (VEC) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) scatter_one(key[u].v[j], val[u].v[j]);
+      } else {
+        scatter_one(key[u], val[u]);
+      }
+    }
+  }
+
+  __syncthreads();
+  for (int i = threadIdx.x; i < per_cta; i += kHistBlock) {
+    const int v = bins_smem[i];
+    const uint32_t bin = rank * (uint32_t)per_cta + i;
+    if (v != 0 && bin < n_bins) atomicAdd(acc64 + bin, (double)v * down);
+  }
+
+  static_for<0, N>([&](auto ic) {
+    constexpr int i = decltype(ic)::value;
+    constexpr CNode nd = CL::c.nodes[i];
+    if constexpr (is_scalar_fold(nd)) {
+      constexpr int ord = count_if<CL>(is_scalar_fold, i);
+      const uint32_t v = block_reduce_n<nd.fn, nd.dtype, kHistBlock>(acc[i], red);
+      if (threadIdx.x == 0) a.scratch[stream_partials_off() + ord * a.grid + blockIdx.x] = v;
+    }
+  });
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) last_block = atomicAdd(a.scratch, 1u) == gridDim.x - 1;
+  __syncthreads();
+  if (!last_block) return;
+  __threadfence();
+  static_for<0, N>([&](auto ic) {
+    constexpr int i = decltype(ic)::value;
+    constexpr CNode nd = CL::c.nodes[i];
+    if constexpr (is_scalar_fold(nd)) {
+      constexpr int ord = count_if<CL>(is_scalar_fold, i);
+      const volatile uint32_t* part = a.scratch + stream_partials_off() + ord * a.grid;
+      uint32_t v = identity_of<nd.fn, nd.dtype>();
+      for (int b = threadIdx.x; b < (int)gridDim.x; b += kHistBlock) v = combine<nd.fn, nd.dtype>(v, part[b]);
+      v = block_reduce_n<nd.fn, nd.dtype, kHistBlock>(v, red);
+      if (threadIdx.x == 0) *reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr)) = v;
+    }
+  });
+  const volatile double* sums = acc64;
+  const float* defaults = reinterpret_cast<const float*>(a.n[pn.in[0]].ptr);
+  float* out = reinterpret_cast<float*>(const_cast<void*>(a.n[P].ptr));
+  for (uint32_t b = threadIdx.x; b < n_bins; b += kHistBlock) out[b] = (float)((double)defaults[b] + sums[b]);
+}
+
+}  // namespace dev
+}  // namespace acc

@@ -6,6 +6,7 @@
 
 #include "../graph.h"
 #include "../registry.h"
+#include "hist.cuh"
 #include "skeletons.cuh"
 
 namespace acc {
@@ -17,6 +18,9 @@ struct Launcher {
   static constexpr bool kHasRowFold = dev::count_if<CL>(dev::is_row_fold) > 0;
   static constexpr int kScalarFolds = dev::count_if<CL>(dev::is_scalar_fold);
   static constexpr int kScanTile = dev::kBlock * 16;
+  // exactly one scatter, fp32 '+': its bins can live in shared memory (k_hist)
+  static constexpr bool kHistShape = !kHasScan && !kHasRowFold && dev::count_if<CL>(dev::is_permute_root) == 1 &&
+                                     dev::count_if<CL>(dev::is_f32_add_permute) == 1;
 
   // Local id of the array whose index space root `i` iterates over, -1 if i is no root.
   static int domain_of(int i) {
@@ -91,6 +95,8 @@ struct Launcher {
     a.grid = sm_count() * 8;             // the partials' layout is sized for the largest grid
   }
 
+  static int launch_hist(const ClusterLaunch& L, dev::Args<N>& a, int R, int C, bool vec);
+
   static int launch(const ClusterLaunch& L) {
     int R, C;
     if (!domain(L, R, C)) return set_error(ACC_ERR_NO_KERNEL, "cluster without a root");
@@ -121,6 +127,10 @@ struct Launcher {
       if (vec) dev::k_rowfold<CL, true><<<grid, dev::kBlock, 0, L.stream>>>(a);
       else dev::k_rowfold<CL, false><<<grid, dev::kBlock, 0, L.stream>>>(a);
     } else {
+      if constexpr (kHistShape) {
+        const int rc = launch_hist(L, a, R, C, vec);
+        if (rc != 1) return rc;                        // 1 = not worth it or does not fit: stream instead
+      }
       // an empty domain still runs one block: a scatter must copy its defaults out
       const int grid = stream_grid(R, C, vec);
       if (vec) dev::k_stream<CL, true><<<grid, dev::kBlock, 0, L.stream>>>(a);
@@ -131,6 +141,42 @@ struct Launcher {
     return ACC_OK;
   }
 };
+
+// On-chip histogram path.  Returns ACC_OK after a launch, an error, or 1 when the generic
+// streaming kernel should run instead (more bins than eight CTAs' shared memory holds, or too
+// few elements per bin to repay clearing and flushing the on-chip bins).
+template <class CL>
+int Launcher<CL>::launch_hist(const ClusterLaunch& L, dev::Args<N>& a, int R, int C, bool vec) {
+  if constexpr (kHistShape) {
+    constexpr int P = dev::the_f32_add_permute<CL>();
+    const int64_t bins = (int64_t)L.nodes[P].R * L.nodes[P].C;
+    const int64_t total = (int64_t)R * C;
+    if (bins <= 0 || total < 8 * bins) return 1;
+    int group = 1;
+    while (group <= 8 && (bins + group - 1) / group > dev::kHistMaxBinsPerCta) group *= 2;
+    if (group > 8 || group > sm_count()) return 1;
+    const int per_cta = (int)((bins + group - 1) / group);
+    int shift = -1;
+    if ((per_cta & (per_cta - 1)) == 0)
+      for (shift = 0; (1 << shift) < per_cta; ++shift) {}
+    auto kern = vec ? dev::k_hist<CL, true> : dev::k_hist<CL, false>;
+    const size_t smem = (size_t)per_cta * 4;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return set_error(ACC_ERR_CUDA, "shared-memory opt-in failed: %s", cudaGetErrorString(cudaGetLastError()));
+    const int64_t chunks = total / (vec ? 4 : 1);
+    const int64_t per_team = (int64_t)dev::kHistBlock * dev::kHistUnroll;
+    const int64_t want = (chunks + per_team - 1) / per_team;
+    const int teams = (int)std::max<int64_t>(1, std::min<int64_t>(want, sm_count() / group));
+    const int grid = teams * group;                       // one CTA per SM: all of them are resident together
+    if (grid > a.grid) return 1;
+    kern<<<grid, dev::kHistBlock, smem, L.stream>>>(a, per_cta, shift, group);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return set_error(ACC_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+    return ACC_OK;
+  } else {
+    return 1;
+  }
+}
 
 template <class CL>
 struct Registrar {

@@ -29,19 +29,24 @@ __device__ __forceinline__ uint32_t warp_reduce(uint32_t v) {
   return v;
 }
 
-// Reduces over the block; the result is valid in thread 0.  `red` holds kBlock/32 words.
-template <int FN, int DT>
-__device__ __forceinline__ uint32_t block_reduce(uint32_t v, uint32_t* red) {
+// Reduces over a block of THREADS threads; the result is valid in thread 0.  `red` holds
+// THREADS/32 words.
+template <int FN, int DT, int THREADS>
+__device__ __forceinline__ uint32_t block_reduce_n(uint32_t v, uint32_t* red) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   v = warp_reduce<FN, DT>(v);
   __syncthreads();
   if (lane == 0) red[warp] = v;
   __syncthreads();
   if (warp == 0) {
-    v = lane < kBlock / 32 ? red[lane] : identity_of<FN, DT>();
+    v = lane < THREADS / 32 ? red[lane] : identity_of<FN, DT>();
     v = warp_reduce<FN, DT>(v);
   }
   return v;
+}
+template <int FN, int DT>
+__device__ __forceinline__ uint32_t block_reduce(uint32_t v, uint32_t* red) {
+  return block_reduce_n<FN, DT, kBlock>(v, red);
 }
 
 // ---- compile-time layout of a cluster's roots ------------------------------------------

@@ -76,7 +76,10 @@ def test_config4_four_iterations_planned():
         check_program(prog, [pi])
 
 
-@pytest.mark.parametrize("n,bins", [(1, 1), (7, 4), (1000, 16), (4096, 256), (100003, 1 << 10), (1 << 18, 1 << 16)])
+# few elements per bin: atomics on global accumulators; many: bins in shared memory, of one CTA
+# (up to 48 Ki bins) or split over a cluster of CTAs (2^16 bins over two, 3 * 2^16 over eight)
+@pytest.mark.parametrize("n,bins", [(1, 1), (7, 4), (1000, 16), (4096, 256), (100003, 1 << 10), (1 << 18, 1 << 16),
+                                    (1 << 20, 1 << 16), (3 << 19, 50000), (3 << 20, 3 << 16)])
 def test_config5_all_partitions(n, bins):
     assert check_program(W.config5(n, bins)) == 10
 
@@ -122,3 +125,55 @@ def test_scatter_out_of_range_is_reported():
     with pytest.raises(B.AccError) as e:
         g.run()
     assert e.value.status == "ACC_ERR_INDEX_RANGE"
+
+
+def _weighted_histogram(n, bins):
+    """keys, zeros, vals as inputs; k = hash keys; hist = permute(+) zeros k vals."""
+    from workloads import Node, Program
+    nodes = [Node("input", "u32", (n,), name="keys"), Node("input", "f32", (bins,), name="zeros"),
+             Node("input", "f32", (n,), name="vals"),
+             Node("map", "u32", (n,), (0,), 1, fn="mul_mod", iparam=(40503, bins), name="k"),
+             Node("permute", "f32", (bins,), (1, 3, 2), 3, fn="add", name="hist")]
+    return Program("weighted_histogram", nodes, [4])
+
+
+@pytest.mark.parametrize("flavour", ["floats", "dyadic", "outliers", "one_hot_bin"])
+def test_scatter_add_of_arbitrary_fp32_values(flavour):
+    # the on-chip histogram adds multiples of its quantum as integers and everything else in fp64:
+    # random floats (mostly the fp64 route), signed multiples of 1/8 (integer route), a few huge,
+    # tiny, infinite values among them, and one bin hit by every element (bins spill into fp64)
+    import torch
+    from paper_2407_13585_b200 import binding as B
+    n, bins = 1 << 20, 4096
+    prog = _weighted_histogram(n, bins)
+    keys = W.zipf_keys(3, 0, n)
+    defaults = W.uniform_f32(3, 2, bins)
+    if flavour == "floats":
+        vals = W.uniform_f32(3, 4, n)
+    elif flavour == "dyadic":
+        vals = torch.round(W.uniform_f32(3, 4, n) * 64) / 8
+    elif flavour == "outliers":
+        vals = torch.round(W.uniform_f32(3, 4, n) * 64) / 8
+        vals[5] = 3.0e20
+        vals[77] = 1.0e-30
+        vals[1000] = float("inf")
+        vals[2000:2100] = 7.0e5
+    else:
+        keys = torch.zeros(n, dtype=torch.int32)
+        vals = torch.full((n,), 262143.0)
+    inputs = {0: keys, 1: defaults, 2: vals}
+    ref = oracle_run(prog, np_inputs(inputs))
+    for pi in ([-1, -1, -1, 0, 1], [-1, -1, -1, 0, 0]):
+        got, _ = gpu_run(prog, inputs, pi, B.FUSED)
+        with np.errstate(invalid="ignore"):
+            compare_hist(prog, ref, got, flavour)
+
+
+def compare_hist(prog, ref, got, what):
+    exact, scale, a = ref.exact[4], ref.abs_sum[4], got[4].astype(np.float64)
+    finite = np.isfinite(exact)
+    assert np.array_equal(np.isfinite(a), finite), what
+    assert np.array_equal(a[~finite], exact[~finite]) or np.all(np.isnan(exact[~finite]) == np.isnan(a[~finite])), what
+    bound = 1e-5 * scale[finite] + np.abs(exact[finite]) * 2.0 ** -24 + 1e-30
+    assert np.all(np.abs(a[finite] - exact[finite]) <= bound), what
+    assert 3 not in got or np.array_equal(got[3], ref.values[3]), what
