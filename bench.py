@@ -31,6 +31,14 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
 
+def scaled(sizes, shrink):
+    """Sizes with every element count divided by 2^shrink (square arrays shrink by 2^(shrink/2) per side)."""
+    out = {}
+    for k, v in sizes.items():
+        out[k] = max(4, v >> shrink) if k == "n" else max(4, v >> (shrink // 2))
+    return out
+
+
 def count_of(nd):
     c = 1
     for e in nd.shape:
@@ -229,7 +237,8 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    loads = [Workload(cfg, FULL[cfg], device) for cfg in ORDER]
+    order = [c for c in ORDER if c in args.configs]
+    loads = [Workload(cfg, scaled(FULL[cfg], args.shrink), device, host=not args.fused_only) for cfg in order]
     step_bytes = sum(w.bytes for w in loads)
 
     def step():
@@ -254,6 +263,15 @@ def run_ours(args):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         ms_step = float(t.item())
     value = world * step_bytes / (ms_step * 1e-3) / 1e9
+    if args.fused_only:
+        # profiling aid: only the fused steps above, no unfused / end-to-end / CPU legs
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": value, "unit": "GB/s", "ms_per_step": ms_step,
+                              "config": {"workload": "configs %s, sizes / 2^%d" % (order, args.shrink)},
+                              "gpu_launches": launches * args.steps}))
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     # per program: fused and unfused executors side by side (rank 0's GPU)
     per = {}
@@ -355,7 +373,11 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--configs", default="1,2,3,4,5", help="programs to include (profiling aid)")
+    ap.add_argument("--shrink", type=int, default=0, help="divide every element count by 2^SHRINK (profiling aid)")
+    ap.add_argument("--fused-only", action="store_true", help="time the fused steps only (profiling aid)")
     args = ap.parse_args()
+    args.configs = [int(c) for c in args.configs.split(",")]
     if args.impl == "reference":
         run_reference(args)
     else:

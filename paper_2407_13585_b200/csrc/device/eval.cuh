@@ -288,6 +288,15 @@ __device__ __forceinline__ val_of<IX> eval(const A& a, const IX& ix) {
     if constexpr (std::is_same<IX, IxS4>::value) {
 #pragma unroll
       for (int j = 0; j < 4; ++j) out.v[j] = generate1<nd.fn, nd.dtype>(a.n[I], lane_clamped(ix, j, a.n[I].C), f0);
+    } else if constexpr (std::is_same<IX, Ix4>::value && nd.fn == ACC_FN_IMOD_TO_F32) {
+      // one division for four consecutive indices: the remainders follow by stepping
+      const uint32_t m = (uint32_t)a.n[I].ip0;
+      uint32_t r = (uint32_t)(ix.r * a.n[I].C + ix.c) % m;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        out.v[j] = u_((float)r);
+        r = r + 1 == m ? 0u : r + 1;
+      }
     } else {
 #pragma unroll
       for (int j = 0; j < 4; ++j) out.v[j] = generate1<nd.fn, nd.dtype>(a.n[I], lane(ix, j), f0);

@@ -1,26 +1,29 @@
 // k_hist: the skeleton for a cluster whose permute is an fp32 '+' scatter into few enough
 // bins to keep them on chip.
 //
-// Measured on B200: shared-memory integer atomics sustain about 1000 G updates/s on a
-// Zipf-skewed key stream, fp32 shared-memory atomics about 56 G/s (they retry on every
-// collision, and a hot bin collides all the time), atomics into a partner CTA's shared
-// memory 140 G/s.  So the bins are 32-bit *integers* in the CTA's own shared memory:
+// Measured on B200 (2^27 Zipf-skewed keys): shared-memory integer atomics sustain about
+// 1000 G updates/s, fp32 shared-memory atomics about 56 G/s (they retry on every collision,
+// and a hot bin collides all the time), atomics into a partner CTA's shared memory 140 G/s.
+// So the bins are 32-bit *integers* in the CTA's own shared memory:
 //
-//  * a value x is added as the integer x * 2^S when that product is an integer below 2^19
-//    in magnitude -- exact, one native atomic.  S is picked per CTA from the largest
-//    magnitude among the first elements it sees;
+//  * a value x is added as the integer x * 2^S when that product is an integer of magnitude
+//    below `cap` -- exact, one fire-and-forget native atomic.  `cap` is 2^31 divided by the
+//    number of elements the CTA can meet, so a bin cannot overflow; S is picked per CTA from
+//    the largest magnitude among the first elements it sees;
 //  * any other value (not a multiple of 2^-S, too large, not finite) is added to the global
 //    fp64 accumulator of its bin directly -- exact as well, slower;
-//  * a bin that reaches 2^29 in magnitude is emptied into its fp64 accumulator by the thread
-//    that crossed the line, so bins never overflow;
 //  * at the end every CTA adds its bins into the fp64 accumulators, and the block that
 //    finishes last turns those into the fp32 result on top of the defaults.
 //
 // Every partial sum is exact, so the result is the fp32 rounding of the exact fp64-combined
-// sum whatever the order of arrival.  When the bins of one scatter exceed one CTA's shared
-// memory, a group of G = 2, 4 or 8 neighbouring CTAs splits them: all CTAs of a group walk
-// the same elements (the second reader hits L2) and each updates only the bins it owns.
-// Store roots and whole-array folds of an element are handled by one CTA of the group.
+// sum whatever the order of arrival.
+//
+// Bins beyond one CTA's shared memory: up to kHistOverflowBins more live in a private slice
+// of global memory per CTA (integer atomics again; private, so a hot bin is not shared
+// between SMs).  Beyond that a group of G = 2, 4 or 8 neighbouring CTAs splits the bins:
+// all CTAs of a group walk the same elements (the later readers hit L2) and each updates
+// only the bins it owns; store roots and whole-array folds of an element are handled by one
+// CTA of the group.
 #pragma once
 #include "skeletons.cuh"
 
@@ -29,9 +32,32 @@ namespace dev {
 
 constexpr int kHistBlock = 1024;
 constexpr int kHistMaxBinsPerCta = 56 * 1024;   // 224 KiB of 32-bit bins per CTA
+constexpr int kHistOverflowBins = 16 * 1024;    // further bins kept per CTA in global memory
 constexpr int kHistUnroll = 2;                  // independent chunks in flight per thread
-constexpr int kHistElementCap = 1 << 19;        // largest |x * 2^S| taken on the integer path
-constexpr int kHistSpillAt = 1 << 29;           // a bin is emptied once it reaches this magnitude
+
+struct HistPlan {
+  int group;        // CTAs that split the bins
+  int per_cta;      // bins in each CTA's shared memory
+  int shift;        // log2(per_cta) when it is a power of two and group > 1, else -1
+  int overflow;     // bins per CTA kept in global memory (group == 1 only)
+};
+
+// How the bins are laid out, or false when they do not fit eight CTAs.
+inline bool hist_plan(int64_t bins, int sms, HistPlan& p) {
+  p = HistPlan{1, 0, -1, 0};
+  if (bins <= 0) return false;
+  if (bins <= kHistMaxBinsPerCta + kHistOverflowBins) {
+    p.per_cta = (int)std::min<int64_t>(bins, kHistMaxBinsPerCta);
+    p.overflow = (int)(bins - p.per_cta);
+    return true;
+  }
+  while (p.group <= 8 && (bins + p.group - 1) / p.group > kHistMaxBinsPerCta) p.group *= 2;
+  if (p.group > 8 || p.group > sms) return false;
+  p.per_cta = (int)((bins + p.group - 1) / p.group);
+  if ((p.per_cta & (p.per_cta - 1)) == 0)
+    for (p.shift = 0; (1 << p.shift) < p.per_cta; ++p.shift) {}
+  return true;
+}
 
 template <class CL> constexpr int the_f32_add_permute() {
   for (int i = 0; i < CL::c.n; ++i)
@@ -41,7 +67,7 @@ template <class CL> constexpr int the_f32_add_permute() {
 
 template <class CL, bool VEC>
 __global__ void __launch_bounds__(kHistBlock, 1)
-k_hist(const __grid_constant__ Args<CL::c.n> a, int per_cta, int per_cta_shift, int group) {
+k_hist(const __grid_constant__ Args<CL::c.n> a, const HistPlan plan, int* overflow_base) {
   constexpr int N = CL::c.n;
   constexpr int W = VEC ? 4 : 1;
   constexpr int U = kHistUnroll;
@@ -57,9 +83,12 @@ k_hist(const __grid_constant__ Args<CL::c.n> a, int per_cta, int per_cta_shift, 
   __shared__ bool last_block;
   __shared__ float sample_max;
 
-  const uint32_t rank = blockIdx.x % (uint32_t)group;          // which slice of the bins this CTA owns
-  const uint32_t team = blockIdx.x / (uint32_t)group;          // which share of the elements its group walks
-  const uint32_t n_teams = gridDim.x / (uint32_t)group;
+  const int per_cta = plan.per_cta;
+  const uint32_t group = (uint32_t)plan.group;
+  const uint32_t rank = blockIdx.x % group;                    // which slice of the bins this CTA owns
+  const uint32_t team = blockIdx.x / group;                    // which share of the elements its group walks
+  const uint32_t n_teams = gridDim.x / group;
+  int* const spill = overflow_base + (size_t)blockIdx.x * plan.overflow;   // zeroed by the host with the scratch
   for (int i = threadIdx.x; i < per_cta; i += kHistBlock) bins_smem[i] = 0;
 
   uint32_t acc[N];
@@ -99,33 +128,34 @@ k_hist(const __grid_constant__ Args<CL::c.n> a, int per_cta, int per_cta_shift, 
     if (threadIdx.x == 0) sample_max = f_(top);
   }
   __syncthreads();
+  // a bin receives at most `mine` addends of magnitude < cap each: |sum| < 2^31
+  const uint32_t mine = ((total + n_teams - 1) / n_teams + 1) * W;
+  const int cap_log2 = 30 - (32 - __clz(mine));                // 2^cap_log2 * mine < 2^30
   int S = 0;
   if (sample_max > 0.0f) {
     int e;
     frexpf(sample_max, &e);                                    // sample_max = f * 2^e, f in [0.5, 1)
-    S = min(max(18 - e, -100), 100);                           // sample_max * 2^S in [2^17, 2^18)
+    S = min(max(cap_log2 - 1 - e, -100), 100);                 // sample_max * 2^S < cap / 2
   }
+  const float cap = exp2f((float)cap_log2);
   const float up = exp2f((float)S);
   const double down = exp2((double)-S);
 
   auto scatter_one = [&](uint32_t k, uint32_t xbits) {
     if (k >= n_bins) { atomicOr(a.status, kStatusIndex); return; }
-    const uint32_t owner = per_cta_shift >= 0 ? (k >> per_cta_shift) : (k / (uint32_t)per_cta);
-    if (owner != rank) return;
+    int* slot;
+    if (group == 1) {
+      slot = k < (uint32_t)per_cta ? bins_smem + k : spill + (k - (uint32_t)per_cta);
+    } else {
+      const uint32_t owner = plan.shift >= 0 ? (k >> plan.shift) : (k / (uint32_t)per_cta);
+      if (owner != rank) return;
+      slot = bins_smem + (k - owner * (uint32_t)per_cta);
+    }
     const float x = f_(xbits);
     if (x == 0.0f) return;
     const float t = __fmul_rn(x, up);                          // exact whenever |t| >= 1 (no underflow)
-    if (fabsf(t) >= 1.0f && fabsf(t) < (float)kHistElementCap && t == rintf(t)) {
-      const int v = (int)t;
-      int* slot = bins_smem + (k - owner * (uint32_t)per_cta);
-      const int old = atomicAdd(slot, v);
-      if (abs(old + v) >= kHistSpillAt && abs(old) < kHistSpillAt) {
-        const int taken = atomicExch(slot, 0);
-        atomicAdd(acc64 + k, (double)taken * down);
-      }
-    } else {
-      atomicAdd(acc64 + k, (double)x);
-    }
+    if (fabsf(t) >= 1.0f && fabsf(t) < cap && t == rintf(t)) atomicAdd(slot, (int)t);
+    else atomicAdd(acc64 + k, (double)x);
   };
 
   uint32_t it = 0;
@@ -146,7 +176,7 @@ k_hist(const __grid_constant__ Args<CL::c.n> a, int per_cta, int per_cta_shift, 
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       if (!live[u]) continue;
-      if ((it + u) % (uint32_t)group == rank) {                // this CTA's turn for the element-wise side
+      if (group == 1 || (it + u) % group == rank) {            // this CTA's turn for the element-wise side
         const IX ix = index_of(q0 + u * stride);
         static_for<0, N>([&](auto ic) {
           constexpr int i = decltype(ic)::value;
@@ -178,6 +208,10 @@ k_hist(const __grid_constant__ Args<CL::c.n> a, int per_cta, int per_cta_shift, 
     const int v = bins_smem[i];
     const uint32_t bin = rank * (uint32_t)per_cta + i;
     if (v != 0 && bin < n_bins) atomicAdd(acc64 + bin, (double)v * down);
+  }
+  for (int i = threadIdx.x; i < plan.overflow; i += kHistBlock) {
+    const int v = *reinterpret_cast<volatile int*>(spill + i);
+    if (v != 0) atomicAdd(acc64 + per_cta + i, (double)v * down);
   }
 
   static_for<0, N>([&](auto ic) {

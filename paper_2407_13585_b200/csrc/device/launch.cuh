@@ -82,6 +82,8 @@ struct Launcher {
     int64_t words = dev::stream_acc64_off(kScalarFolds, sm_count() * 8);
     for (int i = 0; i < N; ++i)
       if (dev::is_f32_add_permute(CL::c.nodes[i])) words += 2 * (int64_t)L.nodes[i].R * L.nodes[i].C;
+    dev::HistPlan plan;
+    if (use_hist(L, R, C, plan)) words += (int64_t)sm_count() * plan.overflow;   // private overflow bins per CTA
     return words * 4;
   }
 
@@ -96,6 +98,19 @@ struct Launcher {
   }
 
   static int launch_hist(const ClusterLaunch& L, dev::Args<N>& a, int R, int C, bool vec);
+
+  // Whether the scatter's bins go on chip: they must fit (see hist_plan) and there must be
+  // enough elements per bin to repay clearing and flushing them.
+  static bool use_hist(const ClusterLaunch& L, int R, int C, dev::HistPlan& plan) {
+    if constexpr (kHistShape) {
+      constexpr int P = dev::the_f32_add_permute<CL>();
+      const int64_t bins = (int64_t)L.nodes[P].R * L.nodes[P].C;
+      if (bins <= 0 || (int64_t)R * C < 8 * bins) return false;
+      return dev::hist_plan(bins, sm_count(), plan);
+    } else {
+      return false;
+    }
+  }
 
   static int launch(const ClusterLaunch& L) {
     int R, C;
@@ -143,33 +158,25 @@ struct Launcher {
 };
 
 // On-chip histogram path.  Returns ACC_OK after a launch, an error, or 1 when the generic
-// streaming kernel should run instead (more bins than eight CTAs' shared memory holds, or too
-// few elements per bin to repay clearing and flushing the on-chip bins).
+// streaming kernel should run instead.
 template <class CL>
 int Launcher<CL>::launch_hist(const ClusterLaunch& L, dev::Args<N>& a, int R, int C, bool vec) {
   if constexpr (kHistShape) {
+    dev::HistPlan plan;
+    if (!use_hist(L, R, C, plan)) return 1;
     constexpr int P = dev::the_f32_add_permute<CL>();
     const int64_t bins = (int64_t)L.nodes[P].R * L.nodes[P].C;
-    const int64_t total = (int64_t)R * C;
-    if (bins <= 0 || total < 8 * bins) return 1;
-    int group = 1;
-    while (group <= 8 && (bins + group - 1) / group > dev::kHistMaxBinsPerCta) group *= 2;
-    if (group > 8 || group > sm_count()) return 1;
-    const int per_cta = (int)((bins + group - 1) / group);
-    int shift = -1;
-    if ((per_cta & (per_cta - 1)) == 0)
-      for (shift = 0; (1 << shift) < per_cta; ++shift) {}
     auto kern = vec ? dev::k_hist<CL, true> : dev::k_hist<CL, false>;
-    const size_t smem = (size_t)per_cta * 4;
+    const size_t smem = (size_t)plan.per_cta * 4;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return set_error(ACC_ERR_CUDA, "shared-memory opt-in failed: %s", cudaGetErrorString(cudaGetLastError()));
-    const int64_t chunks = total / (vec ? 4 : 1);
+    const int64_t chunks = (int64_t)R * C / (vec ? 4 : 1);
     const int64_t per_team = (int64_t)dev::kHistBlock * dev::kHistUnroll;
     const int64_t want = (chunks + per_team - 1) / per_team;
-    const int teams = (int)std::max<int64_t>(1, std::min<int64_t>(want, sm_count() / group));
-    const int grid = teams * group;                       // one CTA per SM: all of them are resident together
-    if (grid > a.grid) return 1;
-    kern<<<grid, dev::kHistBlock, smem, L.stream>>>(a, per_cta, shift, group);
+    const int teams = (int)std::max<int64_t>(1, std::min<int64_t>(want, sm_count() / plan.group));
+    const int grid = teams * plan.group;                  // one CTA per SM: all of them are resident together
+    int* overflow = reinterpret_cast<int*>(L.scratch + dev::stream_acc64_off(kScalarFolds, a.grid) + 2 * bins);
+    kern<<<grid, dev::kHistBlock, smem, L.stream>>>(a, plan, overflow);
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return set_error(ACC_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
     return ACC_OK;

@@ -76,10 +76,11 @@ def test_config4_four_iterations_planned():
         check_program(prog, [pi])
 
 
-# few elements per bin: atomics on global accumulators; many: bins in shared memory, of one CTA
-# (up to 48 Ki bins) or split over a cluster of CTAs (2^16 bins over two, 3 * 2^16 over eight)
+# few elements per bin: atomics on global accumulators; many: bins in one CTA's shared memory
+# (up to 56 Ki), with a private overflow slice in global memory (2^16 bins), or split over a
+# group of two (100000 bins) or four (3 * 2^16 bins) CTAs
 @pytest.mark.parametrize("n,bins", [(1, 1), (7, 4), (1000, 16), (4096, 256), (100003, 1 << 10), (1 << 18, 1 << 16),
-                                    (1 << 20, 1 << 16), (3 << 19, 50000), (3 << 20, 3 << 16)])
+                                    (1 << 20, 1 << 16), (3 << 19, 50000), (1 << 20, 100000), (3 << 20, 3 << 16)])
 def test_config5_all_partitions(n, bins):
     assert check_program(W.config5(n, bins)) == 10
 
