@@ -220,6 +220,13 @@ __device__ __forceinline__ Ix gather1(uint32_t k, const NodeArg& src) {
 template <class CL, int I, class A, class IX>
 __device__ __forceinline__ val_of<IX> eval(const A& a, const IX& ix);
 
+// Read of external I at an index.  Skeletons that stage externals on chip overload this for
+// their own index kinds.
+template <class CL, int I, class A, class IX>
+__device__ __forceinline__ val_of<IX> ld_ext(const A& a, const IX& ix) {
+  return ld(reinterpret_cast<const uint32_t*>(a.n[I].ptr), a.n[I].C, ix);
+}
+
 template <class CL, int I, class A>
 __device__ __forceinline__ uint32_t free_of(const A& a) {
   constexpr CNode nd = CL::c.nodes[I];
@@ -249,7 +256,7 @@ __device__ __forceinline__ val_of<IX> eval(const A& a, const IX& ix) {
   constexpr CNode nd = CL::c.nodes[I];
   constexpr int W = width_of<IX>::value;
   if constexpr (!nd.member) {
-    return ld(reinterpret_cast<const uint32_t*>(a.n[I].ptr), a.n[I].C, ix);
+    return ld_ext<CL, I>(a, ix);
   } else if constexpr (nd.kind == ACC_BACKPERMUTE) {
     return eval<CL, nd.in[0]>(a, map_index<nd.idxfn>(ix, a.n[I], a.n[nd.in[0]]));
   } else if constexpr (nd.kind == ACC_GATHER) {

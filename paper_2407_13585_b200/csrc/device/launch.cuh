@@ -8,6 +8,7 @@
 #include "../registry.h"
 #include "hist.cuh"
 #include "skeletons.cuh"
+#include "tile.cuh"
 
 namespace acc {
 
@@ -74,9 +75,30 @@ struct Launcher {
     return (int)std::max<int64_t>(1, std::min<int64_t>(want, (int64_t)sm_count() * 8));
   }
 
+  // transposes staged through shared-memory tile pairs (k_tile_pair)
+  static constexpr bool kTileShape = dev::tile_eligible<CL>();
+  static constexpr int kRowFolds = dev::count_if<CL>(dev::is_row_fold);
+
+  // The tile-pair kernel wants a square domain of at least one tile, and every staged
+  // external of that same shape.
+  static bool use_tiles(const ClusterLaunch& L, int R, int C) {
+    if constexpr (kTileShape) {
+      if (R != C || R < dev::kTile) return false;
+      for (int i = 0; i < N; ++i)
+        if (dev::is_staged_external<CL>(i) && (L.nodes[i].R != R || L.nodes[i].C != C)) return false;
+      return true;
+    } else {
+      return false;
+    }
+  }
+
   static int64_t scratch_bytes(const ClusterLaunch& L) {
     int R, C;
     if (!domain(L, R, C)) return ACC_ERR_NO_KERNEL;
+    if (use_tiles(L, R, C)) {
+      const int blocks = (R + dev::kTile - 1) / dev::kTile;
+      return (dev::tile_partials_off(blocks) + (int64_t)kRowFolds * blocks * R) * 4;
+    }
     if (kHasScan) return 16 + (int64_t)(((int64_t)R * C + kScanTile - 1) / kScanTile) * 8;
     if (kHasRowFold) return 0;
     int64_t words = dev::stream_acc64_off(kScalarFolds, sm_count() * 8);
@@ -129,6 +151,19 @@ struct Launcher {
     }
     dev::Args<N> a;
     fill(L, a, R, C);
+    if (use_tiles(L, R, C)) {
+      if constexpr (kTileShape) {
+        auto kern = vec ? dev::k_tile_pair<CL, true> : dev::k_tile_pair<CL, false>;
+        const size_t smem = (size_t)dev::staged_externals<CL>() * 2 * dev::kTileWords * 4;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+          return set_error(ACC_ERR_CUDA, "shared-memory opt-in failed: %s", cudaGetErrorString(cudaGetLastError()));
+        const int blocks = (R + dev::kTile - 1) / dev::kTile;
+        kern<<<dim3(blocks, blocks), dev::kBlock, smem, L.stream>>>(a);
+        const cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return set_error(ACC_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+      }
+      return ACC_OK;
+    }
     if constexpr (kHasScan) {
       if (R != 1) return set_error(ACC_ERR_NO_KERNEL, "scans of rank-2 arrays are not instantiated");
       if (C == 0) return ACC_OK;

@@ -35,7 +35,9 @@ def test_config1_all_partitions(n):
     assert check_program(W.config1(n)) == 8
 
 
-@pytest.mark.parametrize("rows", [1, 4, 33, 100, 256])
+# below one 64 x 64 tile: generic kernels; from 64 rows on: shared-memory tile pairs, with ragged
+# edge tiles (100, 130), without 128-bit accesses (130, 67) and on whole tiles (64, 256)
+@pytest.mark.parametrize("rows", [1, 4, 33, 64, 67, 100, 130, 256])
 def test_config2_all_partitions(rows):
     assert check_program(W.config2(rows)) == 4
 
