@@ -121,7 +121,6 @@ __host__ __device__ inline int64_t tile_partials_off(int row_blocks) { return (r
 template <class CL, bool VEC>
 __global__ void __launch_bounds__(kBlock) k_tile_pair(const __grid_constant__ Args<CL::c.n> a) {
   constexpr int N = CL::c.n;
-  constexpr int E = staged_externals<CL>();
   constexpr int NRF = count_if<CL>(is_row_fold);
   extern __shared__ uint32_t tiles[];
   __shared__ bool finishing[2];
@@ -129,7 +128,10 @@ __global__ void __launch_bounds__(kBlock) k_tile_pair(const __grid_constant__ Ar
   if (I > J) return;                                        // the pair {(I,J),(J,I)} belongs to the CTA with I <= J
   const int n = a.R;                                        // square domain: n x n
   const int blocks = (n + kTile - 1) / kTile;
-  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;   // 16 chunks of four columns x 16 rows per pass
+  // A warp covers 4 rows x 8 chunks of four columns.  With the odd row stride of the staged
+  // tiles, its 32 lanes then fall into 32 different banks both for reads along rows
+  // (bank = row + 4*chunk + j) and for transposed reads (bank = 4*chunk + j + row).
+  const int tx = threadIdx.x & 7, ty = threadIdx.x >> 3;    // chunk 0..7 (32 columns), row 0..31, four passes
 
   // ---- stage source tiles [I,J] (buffer 0) and [J,I] (buffer 1) of every external ----------
   static_for<0, N>([&](auto ic) {
@@ -143,8 +145,8 @@ __global__ void __launch_bounds__(kBlock) k_tile_pair(const __grid_constant__ Ar
         const int row0 = (b == 0 ? I : J) * kTile, col0 = (b == 0 ? J : I) * kTile;
         uint32_t* dst = tiles + (slot * 2 + b) * kTileWords;
 #pragma unroll
-        for (int p = 0; p < kTile / 16; ++p) {
-          const int r = ty + 16 * p, gr = row0 + r, gc = col0 + 4 * tx;
+        for (int p = 0; p < 4; ++p) {
+          const int r = ty + 32 * (p >> 1), c = 32 * (p & 1) + 4 * tx, gr = row0 + r, gc = col0 + c;
           uint32_t v[4] = {0u, 0u, 0u, 0u};
           if (gr < n) {
             if constexpr (VEC) {
@@ -159,7 +161,7 @@ __global__ void __launch_bounds__(kBlock) k_tile_pair(const __grid_constant__ Ar
             }
           }
 #pragma unroll
-          for (int j = 0; j < 4; ++j) dst[r * kTileStride + 4 * tx + j] = v[j];
+          for (int j = 0; j < 4; ++j) dst[r * kTileStride + c + j] = v[j];
         }
       }
     }
@@ -179,54 +181,61 @@ __global__ void __launch_bounds__(kBlock) k_tile_pair(const __grid_constant__ Ar
     ctx.trans = (I == J) ? 0 : 1 - o;
     const int col_tile = o == 0 ? J : I;
 #pragma unroll
-    for (int p = 0; p < kTile / 16; ++p) {
-      const int r = ctx.r0 + ty + 16 * p, c = ctx.c0 + 4 * tx;
-      const bool live = r < n && c < n;                     // VEC: n % 4 == 0, so a live chunk is whole
-      const IxP4 ix{r, c, &ctx};
+    for (int rh = 0; rh < 2; ++rh) {
+      const int r = ctx.r0 + ty + 32 * rh;
       uint32_t row_part[N];
       static_for<0, N>([&](auto ic) {
         constexpr int i = decltype(ic)::value;
         constexpr CNode nd = CL::c.nodes[i];
-        if constexpr (is_store_root(nd)) {
-          if (live) {
-            const V4 v = eval<CL, i>(a, ix);
-            uint32_t* out = reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr));
-            if constexpr (VEC) {
-              st(out, n, Ix4{r, c}, v);
-            } else {
+        if constexpr (is_row_fold(nd)) row_part[i] = identity_of<nd.fn, nd.dtype>();
+      });
+#pragma unroll
+      for (int ch = 0; ch < 2; ++ch) {
+        const int c = ctx.c0 + 32 * ch + 4 * tx;
+        const bool live = r < n && c < n;                   // VEC: n % 4 == 0, so a live chunk is whole
+        const IxP4 ix{r, c, &ctx};
+        static_for<0, N>([&](auto ic) {
+          constexpr int i = decltype(ic)::value;
+          constexpr CNode nd = CL::c.nodes[i];
+          if constexpr (is_store_root(nd)) {
+            if (live) {
+              const V4 v = eval<CL, i>(a, ix);
+              uint32_t* out = reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr));
+              if constexpr (VEC) {
+                st(out, n, Ix4{r, c}, v);
+              } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                  if (c + j < n) out[(size_t)r * n + c + j] = v.v[j];
+              }
+            }
+          } else if constexpr (is_row_fold(nd)) {
+            if (live) {
+              const V4 v = eval<CL, nd.in[0]>(a, ix);
 #pragma unroll
               for (int j = 0; j < 4; ++j)
-                if (c + j < n) out[(size_t)r * n + c + j] = v.v[j];
+                if (VEC || c + j < n) row_part[i] = combine<nd.fn, nd.dtype>(row_part[i], v.v[j]);
             }
           }
-        } else if constexpr (is_row_fold(nd)) {
-          uint32_t s = identity_of<nd.fn, nd.dtype>();
-          if (live) {
-            const V4 v = eval<CL, nd.in[0]>(a, ix);
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-              if (VEC || c + j < n) s = combine<nd.fn, nd.dtype>(s, v.v[j]);
-          }
-#pragma unroll
-          for (int w = 8; w > 0; w >>= 1) s = combine<nd.fn, nd.dtype>(s, __shfl_xor_sync(0xFFFFFFFFu, s, w));
-          row_part[i] = s;
-        }
-      });
+        });
+      }
       if constexpr (NRF > 0) {
-        if (tx == 0 && r < n) {
-          static_for<0, N>([&](auto ic) {
-            constexpr int i = decltype(ic)::value;
-            if constexpr (is_row_fold(CL::c.nodes[i])) {
-              constexpr int ord = count_if<CL>(is_row_fold, i);
-              partials[((size_t)ord * blocks + col_tile) * n + r] = row_part[i];
-            }
-          });
-        }
+        static_for<0, N>([&](auto ic) {
+          constexpr int i = decltype(ic)::value;
+          constexpr CNode nd = CL::c.nodes[i];
+          if constexpr (is_row_fold(nd)) {
+            constexpr int ord = count_if<CL>(is_row_fold, i);
+            uint32_t s = row_part[i];
+#pragma unroll
+            for (int w = 4; w > 0; w >>= 1) s = combine<nd.fn, nd.dtype>(s, __shfl_xor_sync(0xFFFFFFFFu, s, w));
+            if (tx == 0 && r < n) partials[((size_t)ord * blocks + col_tile) * n + r] = s;
+          }
+        });
       }
     }
     if constexpr (NRF > 0) {
       const int row_block = o == 0 ? I : J;
-      __threadfence();
+      if (tx == 0) __threadfence();                         // the writers publish their partials
       __syncthreads();
       if (threadIdx.x == 0) finishing[o] = atomicAdd(counters + row_block, 1u) == (uint32_t)blocks - 1;
       __syncthreads();
