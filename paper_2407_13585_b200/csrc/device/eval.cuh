@@ -299,9 +299,10 @@ __device__ __forceinline__ val_of<IX> eval(const A& a, const IX& ix) {
       // one division for four consecutive indices: the remainders follow by stepping
       const uint32_t m = (uint32_t)a.n[I].ip0;
       uint32_t r = (uint32_t)(ix.r * a.n[I].C + ix.c) % m;
+      const bool small = m <= (1u << 23);      // then float(r) = bits(2^23 + r) - 2^23, no conversion unit
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        out.v[j] = u_((float)r);
+        out.v[j] = small ? u_(__fadd_rn(__uint_as_float(0x4B000000u | r), -8388608.0f)) : u_((float)r);
         r = r + 1 == m ? 0u : r + 1;
       }
     } else {
