@@ -70,10 +70,11 @@ struct Launcher {
   }
 
   static int stream_grid(int R, int C, bool vec) {
-    const int64_t chunks = (int64_t)R * (C / (vec ? 4 : 1));
-    const int64_t per_block = (int64_t)dev::kBlock * dev::kStreamUnroll;
-    const int64_t want = (chunks + per_block - 1) / per_block;
-    return (int)std::max<int64_t>(1, std::min<int64_t>(want, (int64_t)sm_count() * 8));
+    const int64_t per_row = C / (vec ? 4 : 1);
+    const int64_t trips = dev::domain_rank<CL>() <= 1
+                              ? (per_row + dev::kBlock - 1) / dev::kBlock
+                              : ((per_row + 31) / 32) * ((R + dev::kStreamTileRows - 1) / dev::kStreamTileRows);
+    return (int)std::max<int64_t>(1, std::min<int64_t>(trips, (int64_t)sm_count() * 8));
   }
 
   // transposes staged through shared-memory tile pairs (k_tile_pair)

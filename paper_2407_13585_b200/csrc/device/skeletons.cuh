@@ -19,9 +19,7 @@ namespace acc {
 namespace dev {
 
 constexpr int kBlock = 256;
-// Chunks a k_stream thread evaluates per trip.  Measured on the Jacobi iteration (8192^2):
-// 1 -> 0.103 ms, 2 -> 0.147 ms, 4 -> 0.143 ms per kernel; on the 1-D chain no gain either.
-constexpr int kStreamUnroll = 1;
+constexpr int kStreamTileRows = kBlock / 32;   // rows of a rank-2 tile of k_stream (one warp each)
 constexpr uint32_t kStatusTimeout = 1u;
 constexpr uint32_t kStatusIndex = 2u;
 
@@ -135,82 +133,58 @@ __global__ void __launch_bounds__(kBlock) k_stream(const __grid_constant__ Args<
   });
   double* acc64_base = reinterpret_cast<double*>(a.scratch + stream_acc64_off(NF, a.grid));
 
-  // A thread takes U chunks per trip.  Rank 1: U chunks a grid stride apart.  Rank 2: the same
-  // four columns of U consecutive rows, so that what one row's evaluation loads of its
-  // neighbours (shifted reads of a stencil) is what the next row's evaluation loads of itself:
-  // identical loads in straight-line code are issued once.  The rows are clamped to the last
-  // one instead of being skipped, which keeps that code straight-line; only the stores,
-  // accumulations and scatters of a clamped duplicate are suppressed.
-  constexpr int U = kStreamUnroll;
+  // Rank 1: a grid-stride walk over chunks.  Rank 2: a grid-stride walk over tiles of
+  // kStreamTileRows rows x 32 chunks, one warp per row segment (512 contiguous bytes), so that
+  // the rows a stencil reads above and below its own are rows the same block touches anyway.
+  // (Measured on the 8192^2 Jacobi iteration this walk and a plain row-major walk run at the
+  // same speed, 0.103 ms: the kernel is held by the load/store unit, not by L2.)
   const uint32_t per_row = (uint32_t)a.C / W;
-  const uint32_t row_groups = DR <= 1 ? 1u : ((uint32_t)a.R + U - 1) / U;
-  const uint32_t total = DR <= 1 ? per_row : row_groups * per_row;
-  const uint32_t stride = gridDim.x * kBlock;
-  using VAL = val_of<IX>;
-  for (uint32_t q0 = blockIdx.x * kBlock + threadIdx.x; q0 < total; q0 += DR <= 1 ? stride * U : stride) {
-    VAL val[U][N], key[U][N];
-    IX ixs[U];
-    bool live[U];
+  const uint32_t tiles_x = (per_row + 31) / 32;
+  const uint32_t trips = DR <= 1 ? (per_row + kBlock - 1) / kBlock
+                                 : tiles_x * (((uint32_t)a.R + kStreamTileRows - 1) / kStreamTileRows);
+  for (uint32_t t = blockIdx.x; t < trips; t += gridDim.x) {
+    IX ix;
+    bool live;
+    if constexpr (DR <= 1) {
+      const uint32_t q = t * kBlock + threadIdx.x;
+      live = q < per_row;
+      ix.r = 0;
+      ix.c = (int)(q * W);
+    } else {
+      const uint32_t ty = t / tiles_x, tx = t - ty * tiles_x;
+      const uint32_t r = ty * kStreamTileRows + (threadIdx.x >> 5), q = tx * 32 + (threadIdx.x & 31);
+      live = r < (uint32_t)a.R && q < per_row;
+      ix.r = (int)r;
+      ix.c = (int)(q * W);
+    }
+    if (!live) continue;
+    static_for<0, N>([&](auto ic) {
+      constexpr int i = decltype(ic)::value;
+      constexpr CNode nd = CL::c.nodes[i];
+      if constexpr (is_store_root(nd)) {
+        st(reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr)), a.n[i].C, ix, eval<CL, i>(a, ix));
+      } else if constexpr (is_scalar_fold(nd)) {
+        const auto v = eval<CL, nd.in[0]>(a, ix);
+        if constexpr (VEC) {
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-      IX ix;
-      if constexpr (DR <= 1) {
-        const uint32_t q = q0 + u * stride;
-        live[u] = q < total;
-        if (!live[u]) continue;
-        ix.r = 0;
-        ix.c = (int)(q * W);
-      } else {
-        const uint32_t g = q0 / per_row, r = g * U + u;
-        live[u] = r < (uint32_t)a.R;
-        ix.r = (int)min(r, (uint32_t)a.R - 1);
-        ix.c = (int)((q0 - g * per_row) * W);
+          for (int j = 0; j < 4; ++j) acc[i] = combine<nd.fn, nd.dtype>(acc[i], v.v[j]);
+        } else {
+          acc[i] = combine<nd.fn, nd.dtype>(acc[i], v);
+        }
+      } else if constexpr (is_permute_root(nd)) {
+        const auto k = eval<CL, nd.in[1]>(a, ix);
+        const auto x = eval<CL, nd.in[2]>(a, ix);
+        uint32_t* out = reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr));
+        const uint32_t bins = (uint32_t)(a.n[i].R * a.n[i].C);
+        double* acc64 = acc64_of<CL, i>(a, acc64_base);
+        if constexpr (VEC) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) permute_update<nd.fn, nd.dtype>(out, acc64, bins, k.v[j], x.v[j], a.status);
+        } else {
+          permute_update<nd.fn, nd.dtype>(out, acc64, bins, k, x, a.status);
+        }
       }
-      ixs[u] = ix;
-      static_for<0, N>([&](auto ic) {
-        constexpr int i = decltype(ic)::value;
-        constexpr CNode nd = CL::c.nodes[i];
-        if constexpr (is_store_root(nd)) {
-          val[u][i] = eval<CL, i>(a, ix);
-        } else if constexpr (is_scalar_fold(nd)) {
-          val[u][i] = eval<CL, nd.in[0]>(a, ix);
-        } else if constexpr (is_permute_root(nd)) {
-          key[u][i] = eval<CL, nd.in[1]>(a, ix);
-          val[u][i] = eval<CL, nd.in[2]>(a, ix);
-        }
-      });
-    }
-    // ... then store, accumulate and scatter them
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-      if (!live[u]) continue;
-      const IX ix = ixs[u];
-      static_for<0, N>([&](auto ic) {
-        constexpr int i = decltype(ic)::value;
-        constexpr CNode nd = CL::c.nodes[i];
-        if constexpr (is_store_root(nd)) {
-          st(reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr)), a.n[i].C, ix, val[u][i]);
-        } else if constexpr (is_scalar_fold(nd)) {
-          if constexpr (VEC) {
-#pragma unroll
-            for (int j = 0; j < 4; ++j) acc[i] = combine<nd.fn, nd.dtype>(acc[i], val[u][i].v[j]);
-          } else {
-            acc[i] = combine<nd.fn, nd.dtype>(acc[i], val[u][i]);
-          }
-        } else if constexpr (is_permute_root(nd)) {
-          uint32_t* out = reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr));
-          const uint32_t bins = (uint32_t)(a.n[i].R * a.n[i].C);
-          double* acc64 = acc64_of<CL, i>(a, acc64_base);
-          if constexpr (VEC) {
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-              permute_update<nd.fn, nd.dtype>(out, acc64, bins, key[u][i].v[j], val[u][i].v[j], a.status);
-          } else {
-            permute_update<nd.fn, nd.dtype>(out, acc64, bins, key[u][i], val[u][i], a.status);
-          }
-        }
-      });
-    }
+    });
   }
 
   if constexpr (NF > 0 || NP64 > 0) {
