@@ -334,10 +334,15 @@ def run_ours(args):
     wtop = [w for w in loads if w.cfg == top][0]
     peak, peak_kind = measured_peak()
     achieved = kernel_bytes[top](wtop) / (per[top]["ms_fused"] / kernel_launches[top]) / 1e6
-    names = {2: "k_rowfold<transpose+zip+fold>", 3: "k_scan<hash+gather+mask+scan>", 4: "k_stream<jacobi iteration>",
-             5: "k_stream<hash+generate+permute+fold>", 1: "k_stream<chain>"}
+    names = {2: "k_tile_pair<transpose+zip+fold>", 3: "k_scan<hash+gather+mask+scan>", 4: "k_stream<jacobi iteration>",
+             5: "k_hist<hash+generate+permute+fold>", 1: "k_stream<chain>"}
+    # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
+    # summarised under profiles/, taken at these sizes; null for a kernel without a capture
+    ncu_traffic = {3: 6.267e9 + 0.258e9, 4: 268.4e6 + 226.8e6, 2: 269.4e6 + 6.2e6, 5: 542.6e6 + 3.9e6}
+    traffic = ncu_traffic.get(top) if args.shrink == 0 else None
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None, "kernel": names[top], "of": peak_kind,
+                "traffic": traffic, "kernel": names[top], "of": peak_kind,
+                "dram_rate": None if traffic is None else traffic / (per[top]["ms_fused"] / kernel_launches[top]) / 1e6,
                 "bytes_per_launch": kernel_bytes[top](wtop), "launches_per_step": kernel_launches[top]}
 
     cpu = None
@@ -370,7 +375,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--configs", default="1,2,3,4,5", help="programs to include (profiling aid)")
