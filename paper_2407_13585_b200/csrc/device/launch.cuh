@@ -160,7 +160,7 @@ struct Launcher {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
           return set_error(ACC_ERR_CUDA, "shared-memory opt-in failed: %s", cudaGetErrorString(cudaGetLastError()));
         const int blocks = (R + dev::kTile - 1) / dev::kTile;
-        kern<<<dim3(blocks, blocks), dev::kBlock, smem, L.stream>>>(a);
+        kern<<<blocks * (blocks + 1) / 2, dev::kBlock, smem, L.stream>>>(a);
         const cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return set_error(ACC_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
       }

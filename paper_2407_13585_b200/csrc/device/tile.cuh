@@ -118,16 +118,28 @@ __device__ __forceinline__ V4 ld_ext(const A&, const IxQ4& ix) { return ld_tile(
 // one partial per (row fold, column tile, row).
 __host__ __device__ inline int64_t tile_partials_off(int row_blocks) { return (row_blocks + 3) & ~3; }
 
+// Pair number p -> (I, J) with I <= J, rows of the upper triangle one after the other.
+__device__ __forceinline__ void pair_of(uint32_t p, int T, int& I, int& J) {
+  auto first = [T](int k) { return (uint32_t)k * (uint32_t)T - (uint32_t)(k * (k - 1) / 2); };   // first pair of row k
+  const float w = (float)(2 * T + 1);
+  int i = (int)((w - sqrtf(fmaxf(w * w - 8.0f * (float)p, 0.0f))) * 0.5f);
+  i = max(0, min(i, T - 1));
+  for (int guard = 0; guard < 4 && i > 0 && first(i) > p; ++guard) --i;
+  for (int guard = 0; guard < 4 && i + 1 < T && first(i + 1) <= p; ++guard) ++i;
+  I = i;
+  J = min(i + (int)(p - first(i)), T - 1);
+}
+
 template <class CL, bool VEC>
 __global__ void __launch_bounds__(kBlock) k_tile_pair(const __grid_constant__ Args<CL::c.n> a) {
   constexpr int N = CL::c.n;
   constexpr int NRF = count_if<CL>(is_row_fold);
   extern __shared__ uint32_t tiles[];
   __shared__ bool finishing[2];
-  const int I = blockIdx.y, J = blockIdx.x;
-  if (I > J) return;                                        // the pair {(I,J),(J,I)} belongs to the CTA with I <= J
   const int n = a.R;                                        // square domain: n x n
   const int blocks = (n + kTile - 1) / kTile;
+  int I, J;
+  pair_of(blockIdx.x, blocks, I, J);                        // one CTA per pair {(I,J),(J,I)}, I <= J
   // A warp covers 4 rows x 8 chunks of four columns.  With the odd row stride of the staged
   // tiles, its 32 lanes then fall into 32 different banks both for reads along rows
   // (bank = row + 4*chunk + j) and for transposed reads (bank = 4*chunk + j + row).
