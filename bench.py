@@ -221,6 +221,7 @@ def run_ours(args):
     import torch
     import torch.distributed as dist
     from paper_2407_13585_b200 import binding as B
+    from paper_2407_13585_b200.replicas import combine_replicas, effective_gbs
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -258,11 +259,8 @@ def run_ours(args):
     launches = sum(w.g.launch_count() for w in loads)
     for w in loads:
         w.finish()
-    if world > 1:
-        t = torch.tensor([ms_step], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_step = float(t.item())
-    value = world * step_bytes / (ms_step * 1e-3) / 1e9
+    ms_step, job_bytes = combine_replicas(ms_step, step_bytes, dist if world > 1 else None, device)
+    value = effective_gbs(job_bytes, ms_step)
     if args.fused_only:
         # profiling aid: only the fused steps above, no unfused / end-to-end / CPU legs
         if rank == 0:
@@ -317,10 +315,7 @@ def run_ours(args):
     t1.record()
     torch.cuda.synchronize()
     ms_e2e = t0.elapsed_time(t1) / e2e_reps
-    if world > 1:
-        t = torch.tensor([ms_e2e], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
+    ms_e2e, _ = combine_replicas(ms_e2e, step_bytes, dist if world > 1 else None, device)
 
     if rank != 0:
         if world > 1:
