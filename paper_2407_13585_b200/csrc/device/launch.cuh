@@ -8,6 +8,7 @@
 #include "../registry.h"
 #include "hist.cuh"
 #include "skeletons.cuh"
+#include "stencil.cuh"
 #include "tile.cuh"
 
 namespace acc {
@@ -123,6 +124,41 @@ struct Launcher {
 
   static int launch_hist(const ClusterLaunch& L, dev::Args<N>& a, int R, int C, bool vec);
 
+  // clamped shifts served from halo tiles copied by cp.async.bulk.tensor (k_stencil)
+  static constexpr bool kStencilShape = dev::stencil_eligible<CL>();
+
+  // Returns ACC_OK after a launch, an error, or 1 when k_stream should run instead: no
+  // 128-bit rows, an external of another shape, a shift by more than one, or a domain too
+  // small to fill the machine with tiles.
+  static int launch_stencil(const ClusterLaunch& L, dev::Args<N>& a, int R, int C, bool vec) {
+    if constexpr (kStencilShape) {
+      if (!vec || R < 1 || (int64_t)R * C < (int64_t)dev::kStRows * dev::kStCols * sm_count()) return 1;
+      dev::StencilMaps maps;
+      for (int i = 0; i < N; ++i) {
+        const CNode& n = CL::c.nodes[i];
+        if (n.member && n.kind == ACC_BACKPERMUTE && n.idxfn == ACC_IDX_SHIFT_CLAMP &&
+            (L.nodes[i].ip0 < -1 || L.nodes[i].ip0 > 1 || L.nodes[i].ip1 < -1 || L.nodes[i].ip1 > 1))
+          return 1;
+        if (dev::is_staged_external<CL>(i)) {
+          if (L.nodes[i].R != R || L.nodes[i].C != C) return 1;
+          if (!make_tensor_map_2d(&maps.m[dev::tile_slot<CL>(i)], L.nodes[i].ptr, R, C, dev::kStBoxRows, dev::kStBoxCols)) return 1;
+        }
+      }
+      auto kern = dev::k_stencil<CL>;
+      const size_t smem = (size_t)dev::kStStages * dev::staged_externals<CL>() * dev::kStBoxStride * 4;
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return set_error(ACC_ERR_CUDA, "shared-memory opt-in failed: %s", cudaGetErrorString(cudaGetLastError()));
+      const int64_t tiles = (int64_t)((C + dev::kStCols - 1) / dev::kStCols) * ((R + dev::kStRows - 1) / dev::kStRows);
+      const int grid = (int)std::min<int64_t>(tiles, (int64_t)sm_count() * 6);
+      kern<<<grid, dev::kBlock, smem, L.stream>>>(a, maps);
+      const cudaError_t e = cudaGetLastError();
+      if (e != cudaSuccess) return set_error(ACC_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+      return ACC_OK;
+    } else {
+      return 1;
+    }
+  }
+
   // Whether the scatter's bins go on chip: they must fit (see hist_plan) and there must be
   // enough elements per bin to repay clearing and flushing them.
   static bool use_hist(const ClusterLaunch& L, int R, int C, dev::HistPlan& plan) {
@@ -165,6 +201,10 @@ struct Launcher {
         if (e != cudaSuccess) return set_error(ACC_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
       }
       return ACC_OK;
+    }
+    if constexpr (kStencilShape) {
+      const int rc = launch_stencil(L, a, R, C, vec);
+      if (rc != 1) return rc;                            // 1 = shapes or shifts it does not cover: stream instead
     }
     if constexpr (kHasScan) {
       if (R != 1) return set_error(ACC_ERR_NO_KERNEL, "scans of rank-2 arrays are not instantiated");

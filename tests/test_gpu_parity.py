@@ -56,7 +56,9 @@ def test_config3_ragged_lengths():
         check_program(prog)
 
 
-@pytest.mark.parametrize("rows,cols", [(1, 4), (3, 5), (8, 8), (33, 64), (64, 33), (130, 260)])
+# small domains run the streaming kernel; from about 600k cells on, clusters of clamped shifts run on
+# halo tiles copied by the tensor-copy engine: whole tiles (1024^2) and ragged ones (1000 x 1028)
+@pytest.mark.parametrize("rows,cols", [(1, 4), (3, 5), (8, 8), (33, 64), (64, 33), (130, 260), (1024, 1024), (1000, 1028)])
 def test_config4_iteration_cuts(rows, cols):
     prog = W.config4(rows, cols, iters=2)
     per_iter = [-1] + [0] * 9 + [1] * 9
