@@ -132,7 +132,7 @@ struct Launcher {
   // small to fill the machine with tiles.
   static int launch_stencil(const ClusterLaunch& L, dev::Args<N>& a, int R, int C, bool vec) {
     if constexpr (kStencilShape) {
-      if (!vec || R < 1 || (int64_t)R * C < (int64_t)dev::kStRows * dev::kStCols * sm_count()) return 1;
+      if (!vec || R < 1 || (int64_t)R * C < (int64_t)dev::kStRows * dev::kStCols * 64) return 1;
       dev::StencilMaps maps;
       for (int i = 0; i < N; ++i) {
         const CNode& n = CL::c.nodes[i];
@@ -149,7 +149,7 @@ struct Launcher {
       if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return set_error(ACC_ERR_CUDA, "shared-memory opt-in failed: %s", cudaGetErrorString(cudaGetLastError()));
       const int64_t tiles = (int64_t)((C + dev::kStCols - 1) / dev::kStCols) * ((R + dev::kStRows - 1) / dev::kStRows);
-      const int grid = (int)std::min<int64_t>(tiles, (int64_t)sm_count() * 6);
+      const int grid = (int)std::min<int64_t>(tiles, (int64_t)sm_count() * 3);
       kern<<<grid, dev::kBlock, smem, L.stream>>>(a, maps);
       const cudaError_t e = cudaGetLastError();
       if (e != cudaSuccess) return set_error(ACC_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));

@@ -22,7 +22,7 @@
 namespace acc {
 namespace dev {
 
-constexpr int kStRows = 32, kStCols = 128;            // output tile
+constexpr int kStRows = 64, kStCols = 128;            // output tile
 constexpr int kStBoxRows = kStRows + 2;               // + halo rows
 constexpr int kStBoxCols = kStCols + 8;               // + halo columns (4 each side: 16-byte alignment)
 constexpr int kStBoxWords = kStBoxRows * kStBoxCols;  // 4624 words = 18496 bytes per copy
