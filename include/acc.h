@@ -45,7 +45,9 @@ enum acc_kind {
   ACC_GATHER,      /* ys[j] = src[idx[j]] (linear index)     slots {idx, src}     */
   ACC_PERMUTE,     /* out = defaults; out[idx[j]] op= vals[j] slots {defaults, idx, vals} */
   ACC_FOLD,        /* reduce the innermost extent, no seed   slots {xs}           */
-  ACC_FOLDSEG,     /* reserved: segmented fold (not built; acc_add_node rejects it) */
+  ACC_FOLDSEG,     /* ys[s] = fold of xs[off[s] .. off[s+1]), rank-1 xs   slots {xs, off}: n_array_inputs = 1,
+                      off is S+1 increasing int offsets read by index (the paper names foldSeg in a keyword
+                      list only; segments must be non-empty since a fold has no seed)          */
   ACC_SCANL,       /* inclusive left-to-right scan per innermost row  slots {xs}  */
   ACC_SCANR        /* inclusive right-to-left scan per innermost row  slots {xs}  */
 };

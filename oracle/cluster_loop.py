@@ -72,6 +72,9 @@ class _Cluster:
             return self.pull(nd.inputs[1], i)
         if k == "fold":
             return self.fold_at(a, j)[0]
+        if k == "foldseg":
+            off = self.mem[nd.inputs[1]].reshape(-1)
+            return self.reduce_range(a, nd.inputs[0], int(off[j]), int(off[j + 1]))
         if k in ("scanl", "scanr"):
             return self.scan_row(a, j)
         raise ValueError(f"{k} cannot be pulled through")
@@ -90,6 +93,21 @@ class _Cluster:
         for t in range(1, inner):
             acc = self._icombine(nd, acc, self.pull(src, base + t))
         return U32(acc), None
+
+    def reduce_range(self, a, src, lo, hi):
+        """fold(op) of src[lo:hi], left to right, fp32 data carried in fp64."""
+        nd = self.nodes[a]
+        if hi <= lo:
+            raise ValueError("an empty segment has no value")
+        if nd.dtype == "f32":
+            acc = float(self.pull(src, lo))
+            for t in range(lo + 1, hi):
+                acc = float(fns.combine(nd.fn, F64(acc), F64(self.pull(src, t))))
+            return F32(acc)
+        acc = self.pull(src, lo)
+        for t in range(lo + 1, hi):
+            acc = self._icombine(nd, acc, self.pull(src, t))
+        return U32(acc)
 
     def _icombine(self, nd, a, b):
         if nd.fn in ("min", "max") and nd.dtype == "i32":

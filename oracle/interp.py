@@ -108,6 +108,8 @@ def run(nodes, inputs, stop_after=None):
             if src.ndim < 1 or src.shape[-1] == 0:
                 raise ValueError(f"node {i}: fold over an empty extent has no value")
             out = _fold(res, i, nd, src).reshape(shape)
+        elif k == "foldseg":
+            out = _foldseg(res, i, nd, val[nd.inputs[0]], val[nd.inputs[1]])
         elif k in ("scanl", "scanr"):
             src = val[nd.inputs[0]]
             out = _scan(res, i, nd, src, k == "scanr")
@@ -144,6 +146,41 @@ def _fold(res, i, nd, src):
         else:
             out = (s.min(axis=-1) if op == "min" else s.max(axis=-1)).view(U32)
     return np.asarray(out, dtype=U32)
+
+
+def _foldseg(res, i, nd, src, offsets):
+    """ys[s] = fold(op) of src[offsets[s] : offsets[s+1]] (rank-1 source, no seed: segments must be non-empty).
+    The paper only names foldSeg; this is the reading the library documents."""
+    off = offsets.reshape(-1).astype(np.int64)
+    flat = src.reshape(-1)
+    S = off.size - 1
+    if S != int(np.prod(nd.shape, dtype=np.int64)):
+        raise ValueError(f"node {i}: {S} segments for a result of shape {tuple(nd.shape)}")
+    if off[0] < 0 or off[-1] > flat.size:
+        raise IndexError(f"node {i}: segment offsets leave the source")
+    if np.any(off[1:] <= off[:-1]):
+        raise ValueError(f"node {i}: an empty segment has no value (offsets must increase)")
+    op = nd.fn
+    if nd.dtype == "f32":
+        ex, ab = np.empty(S, F64), np.empty(S, F64)
+        red = {"add": np.sum, "mul": np.prod, "min": np.min, "max": np.max}[op]
+        for s in range(S):
+            seg = flat[off[s]:off[s + 1]].astype(F64)
+            ex[s], ab[s] = red(seg), np.abs(seg).sum()
+        res.exact[i], res.abs_sum[i] = ex, ab
+        return ex.astype(F32)
+    out = np.empty(S, U32)
+    view = _signed_view(flat, nd.dtype)
+    with np.errstate(over="ignore"):
+        for s in range(S):
+            if op == "add":
+                out[s] = np.add.reduce(flat[off[s]:off[s + 1]], dtype=U32)
+            elif op == "mul":
+                out[s] = np.multiply.reduce(flat[off[s]:off[s + 1]], dtype=U32)
+            else:
+                seg = view[off[s]:off[s + 1]]
+                out[s] = np.asarray(seg.min() if op == "min" else seg.max()).astype(view.dtype).view(U32)
+    return out
 
 
 def _scan(res, i, nd, src, right):

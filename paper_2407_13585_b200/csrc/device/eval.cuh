@@ -287,6 +287,25 @@ __device__ __forceinline__ val_of<IX> eval(const A& a, const IX& ix) {
     } else {
       return V4{{row_value(lane(ix, 0)), row_value(lane(ix, 1)), row_value(lane(ix, 2)), row_value(lane(ix, 3))}};
     }
+  } else if constexpr (nd.kind == ACC_FOLDSEG) {
+    // a segmented fold pulled through: the requested element names a segment, an inner loop
+    // walks it (offsets are clamped to the source so that a bad offset cannot leave it)
+    const NodeArg& s = a.n[nd.in[0]];
+    const int32_t* off = reinterpret_cast<const int32_t*>(a.n[nd.in[1]].ptr);
+    auto seg_value = [&](const Ix& o) {
+      const int lo = max(__ldg(off + o.c), 0), hi = min(__ldg(off + o.c + 1), s.R * s.C);
+      uint32_t acc = identity_of<nd.fn, nd.dtype>();
+      for (int j = lo; j < hi; ++j) acc = combine<nd.fn, nd.dtype>(acc, eval<CL, nd.in[0]>(a, Ix{0, j}));
+      return acc;
+    };
+    if constexpr (W == 1) {
+      return seg_value(ix);
+    } else if constexpr (std::is_same<IX, IxS4>::value) {
+      return V4{{seg_value(lane_clamped(ix, 0, a.n[I].C)), seg_value(lane_clamped(ix, 1, a.n[I].C)),
+                 seg_value(lane_clamped(ix, 2, a.n[I].C)), seg_value(lane_clamped(ix, 3, a.n[I].C))}};
+    } else {
+      return V4{{seg_value(lane(ix, 0)), seg_value(lane(ix, 1)), seg_value(lane(ix, 2)), seg_value(lane(ix, 3))}};
+    }
   } else if constexpr (W == 1) {
     return eval_member1<CL, I>(a, ix);
   } else if constexpr (nd.kind == ACC_GENERATE) {
@@ -341,6 +360,7 @@ constexpr bool is_elementwise(int kind) {
 }
 constexpr bool is_store_root(const CNode& n) { return n.member && n.manifest && is_elementwise(n.kind); }
 constexpr bool is_fold_root(const CNode& n) { return n.member && n.manifest && n.kind == ACC_FOLD; }
+constexpr bool is_segfold_root(const CNode& n) { return n.member && n.manifest && n.kind == ACC_FOLDSEG; }
 constexpr bool is_scan_root(const CNode& n) { return n.member && (n.kind == ACC_SCANL || n.kind == ACC_SCANR); }
 constexpr bool is_permute_root(const CNode& n) { return n.member && n.kind == ACC_PERMUTE; }
 

@@ -7,6 +7,7 @@
 #include "../graph.h"
 #include "../registry.h"
 #include "hist.cuh"
+#include "segfold.cuh"
 #include "skeletons.cuh"
 #include "stencil.cuh"
 #include "tile.cuh"
@@ -20,6 +21,7 @@ struct Launcher {
   static constexpr bool kHasRowFold = dev::count_if<CL>(dev::is_row_fold) > 0;
   static constexpr int kScalarFolds = dev::count_if<CL>(dev::is_scalar_fold);
   static constexpr int kScanTile = dev::kBlock * 16;
+  static constexpr bool kHasSegFold = dev::count_if<CL>(dev::is_segfold_root) > 0;
   // exactly one scatter, fp32 '+': its bins can live in shared memory (k_hist)
   static constexpr bool kHistShape = !kHasScan && !kHasRowFold && dev::count_if<CL>(dev::is_permute_root) == 1 &&
                                      dev::count_if<CL>(dev::is_f32_add_permute) == 1;
@@ -27,7 +29,7 @@ struct Launcher {
   // Local id of the array whose index space root `i` iterates over, -1 if i is no root.
   static int domain_of(int i) {
     const CNode& n = CL::c.nodes[i];
-    if (dev::is_store_root(n) || dev::is_scan_root(n)) return i;
+    if (dev::is_store_root(n) || dev::is_scan_root(n) || dev::is_segfold_root(n)) return i;
     if (dev::is_fold_root(n)) return n.in[0];
     if (dev::is_permute_root(n)) return n.in[1];
     return -1;
@@ -103,7 +105,7 @@ struct Launcher {
       return (dev::tile_partials_off(blocks) + (int64_t)kRowFolds * blocks * R) * 4;
     }
     if (kHasScan) return 16 + (int64_t)(((int64_t)R * C + kScanTile - 1) / kScanTile) * 8;
-    if (kHasRowFold) return 0;
+    if (kHasRowFold || kHasSegFold) return 0;
     int64_t words = dev::stream_acc64_off(kScalarFolds, sm_count() * 8);
     for (int i = 0; i < N; ++i)
       if (dev::is_f32_add_permute(CL::c.nodes[i])) words += 2 * (int64_t)L.nodes[i].R * L.nodes[i].C;
@@ -201,6 +203,18 @@ struct Launcher {
         if (e != cudaSuccess) return set_error(ACC_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
       }
       return ACC_OK;
+    }
+    if constexpr (kHasSegFold) {
+      if constexpr (dev::segfold_eligible<CL>()) {
+        if (C == 0) return ACC_OK;
+        const int grid = std::min((C + dev::kBlock / 32 - 1) / (dev::kBlock / 32), sm_count() * 8);
+        dev::k_segfold<CL><<<grid, dev::kBlock, 0, L.stream>>>(a);
+        const cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return set_error(ACC_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+        return ACC_OK;
+      } else {
+        return set_error(ACC_ERR_NO_KERNEL, "segmented folds share a kernel only with each other and over one offsets array");
+      }
     }
     if constexpr (kStencilShape) {
       const int rc = launch_stencil(L, a, R, C, vec);

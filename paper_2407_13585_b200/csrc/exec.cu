@@ -169,7 +169,8 @@ int finish(Graph& g, void* workspace, cudaStream_t stream) {
   if (e != cudaSuccess) return set_error(ACC_ERR_CUDA, "stream failed: %s", cudaGetErrorString(e));
   g.host_status = status;
   if (status & 1u) return set_error(ACC_ERR_DEVICE_TIMEOUT, "a device-side wait ran out of iterations");
-  if (status & 2u) return set_error(ACC_ERR_INDEX_RANGE, "a scatter index fell outside its destination");
+  if (status & 2u) return set_error(ACC_ERR_INDEX_RANGE, "a scatter index or a segment offset fell outside its array");
+  if (status & 4u) return set_error(ACC_ERR_SHAPE, "an empty segment has no value: segment offsets must increase");
   return ACC_OK;
 }
 

@@ -51,7 +51,6 @@ static int fn_arity(int fn, int* free_slots) {
 int add_node(Graph& g, const acc_node_desc& d) {
   const int id = (int)g.nodes.size();
   if (d.kind < ACC_INPUT || d.kind > ACC_SCANR) return set_error(ACC_ERR_ARG, "node %d: unknown kind %d", id, d.kind);
-  if (d.kind == ACC_FOLDSEG) return set_error(ACC_ERR_UNSUPPORTED, "node %d: segmented fold is not built", id);
   if (d.dtype < ACC_F32 || d.dtype > ACC_U32) return set_error(ACC_ERR_DTYPE, "node %d: unknown dtype %d", id, d.dtype);
   if (d.rank < 0 || d.rank > 2) return set_error(ACC_ERR_SHAPE, "node %d: rank %d outside 0..2", id, d.rank);
   int64_t count = 1;
@@ -148,6 +147,17 @@ int add_node(Graph& g, const acc_node_desc& d) {
       for (int i = 0; i < d.rank; ++i)
         if (d.shape[i] != s.shape[i]) return set_error(ACC_ERR_SHAPE, "node %d: outer extents differ from the source", id);
       if (s.shape[s.rank - 1] <= 0) return set_error(ACC_ERR_SHAPE, "node %d: fold over an empty extent has no value", id);
+      if (s.dtype != d.dtype) return set_error(ACC_ERR_DTYPE, "node %d: dtype differs from its source", id);
+      break;
+    }
+    case ACC_FOLDSEG: {
+      if (d.n_inputs != 2 || d.n_array_inputs != 1) return set_error(ACC_ERR_ARG, "node %d: foldSeg takes {xs, offsets} with one array slot", id);
+      if (!is_combine(d.fn_id)) return set_error(ACC_ERR_ARG, "node %d: %d is not a combine operator", id, d.fn_id);
+      const acc_node_desc& s = in(0);
+      const acc_node_desc& o = in(1);
+      if (s.rank != 1 || d.rank != 1) return set_error(ACC_ERR_SHAPE, "node %d: foldSeg reduces a rank-1 array to a rank-1 array", id);
+      if (o.rank != 1 || o.shape[0] != d.shape[0] + 1) return set_error(ACC_ERR_SHAPE, "node %d: S segments need S+1 offsets", id);
+      if (!is_int(o.dtype)) return set_error(ACC_ERR_DTYPE, "node %d: offsets must be integer", id);
       if (s.dtype != d.dtype) return set_error(ACC_ERR_DTYPE, "node %d: dtype differs from its source", id);
       break;
     }

@@ -12,7 +12,7 @@ def oracle_run(prog, inputs_np):
 
 
 def accumulating(nd):
-    return nd.kind in ("fold", "scanl", "scanr", "permute") and nd.dtype == "f32"
+    return nd.kind in ("fold", "foldseg", "scanl", "scanr", "permute") and nd.dtype == "f32"
 
 
 def count_of(nd):

@@ -182,3 +182,32 @@ def compare_hist(prog, ref, got, what):
     bound = 1e-5 * scale[finite] + np.abs(exact[finite]) * 2.0 ** -24 + 1e-30
     assert np.all(np.abs(a[finite] - exact[finite]) <= bound), what
     assert 3 not in got or np.array_equal(got[3], ref.values[3]), what
+
+
+@pytest.mark.parametrize("n,segments", [(5, 1), (64, 5), (1000, 16), (100000, 300), (1 << 20, 1 << 12), (1 << 20, 6)])
+def test_segmented_fold(n, segments):
+    # warp-per-segment walk, segments longer than 2^14 elements by the whole block (the last two shapes),
+    # a sum fed by a fused map and a maximum sharing the same walk
+    from paper_2407_13585_b200 import binding as B
+    prog = W.segmented_sums(n, segments)
+    runnable = [pi for pi in all_partitions(prog) if pi != [-1, -1, 0, 1, 0]]
+    assert check_program(prog, runnable) == 3
+    # {m, maxes} is legal (they share the read of xs) but mixes an element-wise store with a segmented fold
+    g = B.Graph(prog.nodes, prog.outputs)
+    g.set_partition([-1, -1, 0, 1, 0])
+    inputs = W.make_inputs(prog)
+    with pytest.raises(B.AccError) as e:
+        gpu_run(prog, inputs, [-1, -1, 0, 1, 0], B.FUSED)
+    assert e.value.status == "ACC_ERR_NO_KERNEL"
+
+
+def test_segmented_fold_reports_bad_offsets():
+    import torch
+    from paper_2407_13585_b200 import binding as B
+    prog = W.segmented_sums(1000, 4)
+    for offsets, status in (([0, 10, 10, 500, 1000], "ACC_ERR_SHAPE"), ([0, 10, 20, 500, 1001], "ACC_ERR_INDEX_RANGE")):
+        inputs = W.make_inputs(prog)
+        inputs[1] = torch.tensor(offsets, dtype=torch.int32)
+        with pytest.raises(B.AccError) as e:
+            gpu_run(prog, inputs, [-1, -1, 0, 0, 0], B.FUSED)
+        assert e.value.status == status

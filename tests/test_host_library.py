@@ -33,7 +33,8 @@ def test_library_exports_every_declared_symbol():
 
 PROGRAMS = [W.config1(64), W.config2(8), W.config3(64), W.config4(8, 8, iters=1), W.config5(256, 16),
             W.scatter_example(16), W.scatter_example_paper_graph(), W.single_loop(16), W.simple1(), W.simple2(),
-            W.simple3(), W.simple4(), W.simple5(), W.greedy_bottom_up_bad(4, 5), W.greedy_top_down_bad(16)]
+            W.simple3(), W.simple4(), W.simple5(), W.greedy_bottom_up_bad(4, 5), W.greedy_top_down_bad(16),
+            W.segmented_sums(64, 5)]
 
 
 @pytest.mark.parametrize("prog", PROGRAMS, ids=lambda p: p.name)
@@ -136,12 +137,16 @@ def test_add_node_validation():
     with pytest.raises(B.AccError) as e:
         g.add_node(Node("fold", "f32", (3,), (empty,), 1, fn="add"))              # fold without a seed over nothing
     assert e.value.status == "ACC_ERR_SHAPE"
-    d = B.make_desc(Node("map", "f32", (4, 6), (x,), 1, fn="affine"))
-    d.kind = B.KIND["foldseg"]
-    with pytest.raises(B.AccError) as e:
-        g.add_node(d)
-    assert e.value.status == "ACC_ERR_UNSUPPORTED"
-    assert g.n == 2
+    flat = g.add_node(_inp("flat", "f32", (24,)))
+    offs = g.add_node(_inp("offs", "i32", (5,)))
+    for nd in (Node("foldseg", "f32", (5,), (flat, offs), 1, fn="add"),        # 5 segments need 6 offsets
+               Node("foldseg", "f32", (4,), (x, offs), 1, fn="add"),           # rank-2 source
+               Node("foldseg", "f32", (4,), (flat, flat), 1, fn="add"),        # float offsets
+               Node("foldseg", "f32", (4,), (flat, offs), 2, fn="add")):       # offsets are read by index, not traversed
+        with pytest.raises(B.AccError):
+            g.add_node(nd)
+    assert g.add_node(Node("foldseg", "f32", (4,), (flat, offs), 1, fn="add")) == 4
+    assert g.n == 5
 
 
 def test_planner_enumerate_finds_the_paper_optima():

@@ -264,3 +264,35 @@ def test_shape_mismatch_rejected():
     nodes = [_inp("a", "f32", (3,)), _inp("b", "f32", (4,)), Node("zipwith", "f32", (3,), (0, 1), 2, fn="add")]
     with pytest.raises(ValueError):
         run(nodes, {0: np.zeros(3, F32), 1: np.zeros(4, F32)})
+
+
+def test_foldseg_worked_and_reductions_to_fold():
+    # foldSeg(+) [1,2,3,4,5] with offsets [0,2,5] = [1+2, 3+4+5]; elements outside [off[0], off[-1]) are ignored
+    nodes = [_inp("x", "f32", (5,)), _inp("off", "i32", (3,)),
+             Node("foldseg", "f32", (2,), (0, 1), 1, fn="add"), Node("foldseg", "f32", (2,), (0, 1), 1, fn="max")]
+    v = run(nodes, {0: np.array([1, 2, 3, 4, 5], F32), 1: np.array([0, 2, 5], I32)})
+    assert v[2].tolist() == [3.0, 12.0] and v[3].tolist() == [2.0, 5.0]
+    v = run(nodes, {0: np.array([1, 2, 3, 4, 5], F32), 1: np.array([1, 2, 4], I32)})
+    assert v[2].tolist() == [2.0, 7.0]
+    # one segment over everything is fold; equal segments are the row fold of the reshaped array
+    n, m = 12, 7
+    x = W.uniform_f32(0, 0, n * m).numpy()
+    nodes = [_inp("x", "f32", (n * m,)), _inp("off", "i32", (n + 1,)), Node("foldseg", "f32", (n,), (0, 1), 1, fn="add"),
+             _inp("x2", "f32", (n, m)), Node("fold", "f32", (n,), (3,), 1, fn="add"),
+             _inp("one", "i32", (2,)), Node("foldseg", "f32", (1,), (0, 5), 1, fn="add"),
+             Node("fold", "f32", (), (0,), 1, fn="add")]
+    r = interp.run(nodes, {0: x, 1: np.arange(0, n * m + 1, m, dtype=I32), 3: x.reshape(n, m), 5: np.array([0, n * m], I32)})
+    assert np.array_equal(r.exact[2], r.exact[4])
+    assert abs(r.exact[6][0] - r.exact[7]) < 1e-12 and abs(r.exact[2].sum() - r.exact[7]) < 1e-9
+    # integers wrap like every other integer fold
+    nodes = [_inp("x", "i32", (3,)), _inp("off", "i32", (2,)), Node("foldseg", "i32", (1,), (0, 1), 1, fn="add")]
+    out = interp.to_external(run(nodes, {0: np.array([2**31 - 1, 1, 5], I32), 1: np.array([0, 3], I32)})[2], "i32")
+    assert out.tolist() == [-2**31 + 5]
+
+
+def test_foldseg_rejects_empty_and_stray_segments():
+    nodes = [_inp("x", "f32", (5,)), _inp("off", "i32", (3,)), Node("foldseg", "f32", (2,), (0, 1), 1, fn="add")]
+    with pytest.raises(ValueError):
+        run(nodes, {0: np.zeros(5, F32), 1: np.array([0, 2, 2], I32)})       # no seed: an empty segment has no value
+    with pytest.raises(IndexError):
+        run(nodes, {0: np.zeros(5, F32), 1: np.array([0, 2, 6], I32)})

@@ -90,6 +90,21 @@ def zipf_keys(seed, stream, n, ids=1 << 20, s=1.1, device="cpu"):
     return out
 
 
+def segment_offsets(seed, stream, n, segments, s=1.1, device="cpu"):
+    """segments+1 int32 offsets over n elements: every segment non-empty, the lengths beyond one
+    element shared out in proportion to r**-s over a seeded shuffle of the ranks r = 1..segments."""
+    assert 1 <= segments <= n
+    order = torch.argsort(counter_bits(seed, stream, segments, device))       # a seeded permutation
+    w = torch.empty(segments, dtype=torch.float64, device=device)
+    w[order] = torch.arange(1, segments + 1, dtype=torch.float64, device=device).pow(-s)
+    extra = torch.floor(w / w.sum() * (n - segments)).to(torch.int64)
+    lengths = extra + 1
+    lengths[order[0]] += n - int(lengths.sum())                                # the remainder goes to the longest
+    off = torch.zeros(segments + 1, dtype=torch.int64, device=device)
+    off[1:] = torch.cumsum(lengths, 0)
+    return off.to(torch.int32)
+
+
 def make_inputs(program, seed=0, device="cpu"):
     """Input tensors of a benchmark or fixture program, keyed by node id.
 
@@ -109,6 +124,8 @@ def make_inputs(program, seed=0, device="cpu"):
         elif name == "config3" and nd.name == "idx":
             assert cnt & (cnt - 1) == 0, "config 3 sizes are powers of two"
             t = uniform_int(seed, st, cnt, cnt, device=device)
+        elif name == "segmented_sums" and nd.name == "offsets":
+            t = segment_offsets(seed, st, nodes[program.id("xs")].shape[0], cnt - 1, device=device)
         elif name == "config4":
             t = normal_f32(seed, st, cnt, device=device)
         elif name == "config5" and nd.name == "keys":

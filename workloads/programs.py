@@ -12,9 +12,10 @@ inputs, so every list is a DAG in topological order.  Slot layout by kind:
   permute      [defaults, idx, vals]           combine op named by fn
   fold         [src]                           reduces the innermost extent
   scanl/scanr  [src]                           inclusive, per innermost row
+  foldseg      [src, offsets]                  n_array = 1; ys[s] = fold of src[offsets[s] .. offsets[s+1])
 
 Slots at positions >= n_array are "free variable" reads (element-level
-indexing, always of element 0 here).  Function names are interpreted by each
+indexing: element 0, except the offsets of a foldseg, which are read at s and s+1).  Function names are interpreted by each
 executor's own table; this file only spells them.
 """
 from dataclasses import dataclass, field
@@ -244,6 +245,18 @@ def greedy_top_down_bad(n=4096):
         Node("fold", "f32", (), (4,), 1, fn="add", name="result"),
     ]
     return Program("greedy_top_down_bad", nodes, [5])
+
+
+def segmented_sums(n=1 << 20, segments=1 << 12):
+    """Segmented fold fed by a fused map: m = map(a*x+b) xs; sums = foldSeg(+) m offsets; maxes = foldSeg(max) xs offsets."""
+    nodes = [
+        _inp("xs", "f32", (n,)),
+        _inp("offsets", "i32", (segments + 1,)),
+        Node("map", "f32", (n,), (0,), 1, fn="affine", fparam=(0.5, 0.25), name="m"),
+        Node("foldseg", "f32", (segments,), (2, 1), 1, fn="add", name="sums"),
+        Node("foldseg", "f32", (segments,), (0, 1), 1, fn="max", name="maxes"),
+    ]
+    return Program("segmented_sums", nodes, [3, 4])
 
 
 CONFIGS = {1: config1, 2: config2, 3: config3, 4: config4, 5: config5}
