@@ -50,8 +50,9 @@ __global__ void __launch_bounds__(kBlock) k_segfold(const __grid_constant__ Args
   __shared__ int n_long;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int S = a.C;                                               // segments
-  const int32_t* off = reinterpret_cast<const int32_t*>(a.n[CL::c.nodes[F].in[1]].ptr);
-  const int n_src = a.n[CL::c.nodes[F].in[0]].R * a.n[CL::c.nodes[F].in[0]].C;
+  constexpr int OFF = CL::c.nodes[F].in[1], SRC = CL::c.nodes[F].in[0];
+  const int32_t* off = reinterpret_cast<const int32_t*>(a.n[OFF].ptr);
+  const int n_src = a.n[SRC].R * a.n[SRC].C;
 
   for (int base = blockIdx.x * WARPS; base < S; base += gridDim.x * WARPS) {
     __syncthreads();
