@@ -104,7 +104,7 @@ struct Launcher {
       const int blocks = (R + dev::kTile - 1) / dev::kTile;
       return (dev::tile_partials_off(blocks) + (int64_t)kRowFolds * blocks * R) * 4;
     }
-    if (kHasScan) return 16 + (int64_t)(((int64_t)R * C + kScanTile - 1) / kScanTile) * 8;
+    if (kHasScan) return 16 + (int64_t)R * ((C + kScanTile - 1) / kScanTile) * 8;
     if (kHasRowFold || kHasSegFold) return 0;
     int64_t words = dev::stream_acc64_off(kScalarFolds, sm_count() * 8);
     for (int i = 0; i < N; ++i)
@@ -221,12 +221,13 @@ struct Launcher {
       if (rc != 1) return rc;                            // 1 = shapes or shifts it does not cover: stream instead
     }
     if constexpr (kHasScan) {
-      if (R != 1) return set_error(ACC_ERR_NO_KERNEL, "scans of rank-2 arrays are not instantiated");
-      if (C == 0) return ACC_OK;
-      const int tiles = (C + kScanTile - 1) / kScanTile;
-      const int grid = std::min(tiles, sm_count() * 6);
-      if (vec) dev::k_scan<CL, true><<<grid, dev::kBlock, 0, L.stream>>>(a, tiles);
-      else dev::k_scan<CL, false><<<grid, dev::kBlock, 0, L.stream>>>(a, tiles);
+      if ((int64_t)R * C == 0) return ACC_OK;
+      const int per_row = (C + kScanTile - 1) / kScanTile;
+      const int64_t tiles = (int64_t)R * per_row;
+      if (tiles >= (int64_t(1) << 31)) return set_error(ACC_ERR_SHAPE, "too many rows to scan in one launch");
+      const int grid = (int)std::min<int64_t>(tiles, (int64_t)sm_count() * 6);
+      if (vec) dev::k_scan<CL, true><<<grid, dev::kBlock, 0, L.stream>>>(a, per_row, (int)tiles);
+      else dev::k_scan<CL, false><<<grid, dev::kBlock, 0, L.stream>>>(a, per_row, (int)tiles);
     } else if constexpr (kHasRowFold) {
       if (R == 0) return ACC_OK;
       const int grid = std::min(R, sm_count() * 16);

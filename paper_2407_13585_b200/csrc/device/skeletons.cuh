@@ -281,25 +281,39 @@ __device__ __forceinline__ void st_state(uint64_t* p, uint64_t flag, uint32_t v)
   *reinterpret_cast<volatile uint64_t*>(p) = (flag << 32) | v;
 }
 
+// stores at a descending chunk: the lanes go back into ascending memory order
+__device__ __forceinline__ void st(uint32_t* p, int C, const IxR4& i, const V4& v) {
+  *reinterpret_cast<uint4*>(p + (i.r * C + i.c - 3)) = make_uint4(v.v[3], v.v[2], v.v[1], v.v[0]);
+}
+
+// Rows of a rank-2 array are scanned independently: a row is cut into tiles of its own, the
+// look-back of a tile stops at the first tile of its row.  A right-to-left scan walks its row
+// from the far end: position p of the walk is element C-1-p of the row.
 template <class CL, bool VEC>
-__global__ void __launch_bounds__(kBlock) k_scan(const __grid_constant__ Args<CL::c.n> a, int n_tiles) {
+__global__ void __launch_bounds__(kBlock) k_scan(const __grid_constant__ Args<CL::c.n> a, int tiles_per_row, int n_tiles) {
   constexpr int N = CL::c.n;
   constexpr int W = VEC ? 4 : 1;
   constexpr int ROWS = VEC ? kScanRows : kScanRows * 4;   // 16 elements per thread either way
   constexpr int TILE = kBlock * 16;
-  using IX = std::conditional_t<VEC, Ix4, Ix>;
   constexpr int S = first_scan<CL>();
   static_assert(S >= 0, "k_scan needs a scan member");
   constexpr CNode sn = CL::c.nodes[S];
   constexpr int FN = sn.fn, DT = sn.dtype;
-  static_assert(sn.kind == ACC_SCANL, "right-to-left scans are not instantiated");
+  constexpr bool REV = sn.kind == ACC_SCANR;
+  using IX = std::conditional_t<VEC, std::conditional_t<REV, IxR4, Ix4>, Ix>;
 
   __shared__ uint32_t warp_total[kBlock / 32];
   __shared__ uint32_t tile_prefix;
   __shared__ int tile_id;
   uint64_t* states = reinterpret_cast<uint64_t*>(a.scratch + 4);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int n = a.C;                                       // rank-1 domain
+  const int n = a.C;                                       // length of a row
+  auto index_at = [&](int row, int p) {                    // walk position p (a multiple of W) of a row -> index
+    IX ix;
+    ix.r = row;
+    ix.c = REV ? n - 1 - p : p;
+    return ix;
+  };
 
   for (;;) {
     __syncthreads();
@@ -307,7 +321,8 @@ __global__ void __launch_bounds__(kBlock) k_scan(const __grid_constant__ Args<CL
     __syncthreads();
     const int tile = tile_id;
     if (tile >= n_tiles) return;
-    const int warp_base = tile * TILE + warp * (TILE / (kBlock / 32));
+    const int row = tile / tiles_per_row, in_row = tile - row * tiles_per_row;
+    const int warp_base = in_row * TILE + warp * (TILE / (kBlock / 32));
 
     uint32_t val[ROWS][W];
     uint32_t carry = identity_of<FN, DT>();                // running total of this warp's earlier rows
@@ -316,7 +331,7 @@ __global__ void __launch_bounds__(kBlock) k_scan(const __grid_constant__ Args<CL
       const int c = warp_base + (j * 32 + lane) * W;
       const bool live = c < n;
       if (live) {
-        const IX ix{0, c};
+        const IX ix = index_at(row, c);
         const auto v = eval<CL, sn.in[0]>(a, ix);
         if constexpr (VEC) {
 #pragma unroll
@@ -362,20 +377,21 @@ __global__ void __launch_bounds__(kBlock) k_scan(const __grid_constant__ Args<CL
 
     if (warp == 0) {
       uint32_t exclusive = identity_of<FN, DT>();
-      if (tile == 0) {
-        if (lane == 0) st_state(states, kFlagPrefix, tile_total);
+      if (in_row == 0) {
+        if (lane == 0) st_state(states + tile, kFlagPrefix, tile_total);
       } else {
         if (lane == 0) st_state(states + tile, kFlagAggregate, tile_total);
-        int look = tile - 1;
+        int look = in_row - 1;                             // tiles of this row before this one
         uint32_t spins = 0;
         bool gave_up = false;
         for (;;) {
           const int idx = look - lane;
-          uint64_t s = idx >= 0 ? ld_state(states + idx) : (kFlagPrefix << 32) | identity_of<FN, DT>();
+          const uint64_t* at = states + (tile - in_row) + idx;
+          uint64_t s = idx >= 0 ? ld_state(at) : (kFlagPrefix << 32) | identity_of<FN, DT>();
           while (__any_sync(0xFFFFFFFFu, (s >> 32) == 0)) {
             if (++spins > a.spin_limit) { gave_up = true; break; }
             __nanosleep(20);
-            if (idx >= 0) s = ld_state(states + idx);
+            if (idx >= 0) s = ld_state(at);
           }
           if (gave_up) break;
           const unsigned done = __ballot_sync(0xFFFFFFFFu, (s >> 32) == kFlagPrefix);
@@ -399,11 +415,12 @@ __global__ void __launch_bounds__(kBlock) k_scan(const __grid_constant__ Args<CL
     for (int j = 0; j < ROWS; ++j) {
       const int c = warp_base + (j * 32 + lane) * W;
       if (c < n) {
+        const IX ix = index_at(row, c);
         if constexpr (VEC) {
-          st(out, n, Ix4{0, c}, V4{{combine<FN, DT>(base, val[j][0]), combine<FN, DT>(base, val[j][1]),
-                                    combine<FN, DT>(base, val[j][2]), combine<FN, DT>(base, val[j][3])}});
+          st(out, n, ix, V4{{combine<FN, DT>(base, val[j][0]), combine<FN, DT>(base, val[j][1]),
+                             combine<FN, DT>(base, val[j][2]), combine<FN, DT>(base, val[j][3])}});
         } else {
-          out[c] = combine<FN, DT>(base, val[j][0]);
+          st(out, n, ix, combine<FN, DT>(base, val[j][0]));
         }
       }
     }

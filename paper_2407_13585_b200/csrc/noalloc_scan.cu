@@ -100,8 +100,8 @@ extern "C" int acc_scanl_add_i32_static(const int32_t* in, int32_t* out, int64_t
   a.grid = 0;
   const bool vec = n % 4 == 0 && ((reinterpret_cast<uintptr_t>(in) | reinterpret_cast<uintptr_t>(out)) & 15) == 0;
   const int grid = tiles < sm_count() * 6 ? tiles : sm_count() * 6;
-  if (vec) dev::k_scan<ScanCluster, true><<<grid, dev::kBlock, 0, stream>>>(a, tiles);
-  else dev::k_scan<ScanCluster, false><<<grid, dev::kBlock, 0, stream>>>(a, tiles);
+  if (vec) dev::k_scan<ScanCluster, true><<<grid, dev::kBlock, 0, stream>>>(a, tiles, tiles);
+  else dev::k_scan<ScanCluster, false><<<grid, dev::kBlock, 0, stream>>>(a, tiles, tiles);
   e = cudaGetLastError();
   if (e != cudaSuccess) return set_error(ACC_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
   uint32_t status = 0;

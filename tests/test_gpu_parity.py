@@ -211,3 +211,15 @@ def test_segmented_fold_reports_bad_offsets():
         with pytest.raises(B.AccError) as e:
             gpu_run(prog, inputs, [-1, -1, 0, 0, 0], B.FUSED)
         assert e.value.status == status
+
+
+@pytest.mark.parametrize("rows,cols", [(1, 5), (7, 100), (64, 300), (3, 5000), (2, 4096 * 3 + 8), (200, 4096)])
+def test_row_scans_both_directions(rows, cols):
+    # rank-2 arrays are scanned row by row (look-back stops at the row start); scanr walks from the far end;
+    # rows of several tiles and of a fraction of one, widths that allow 128-bit accesses and widths that do not
+    check_program(W.row_scans(rows, cols))
+
+
+@pytest.mark.parametrize("n", [1, 6, 4096, 100001, 1 << 18])
+def test_right_to_left_scan_int32(n):
+    check_program(W.suffix_sums(n))

@@ -259,4 +259,26 @@ def segmented_sums(n=1 << 20, segments=1 << 12):
     return Program("segmented_sums", nodes, [3, 4])
 
 
+def row_scans(rows=64, cols=300):
+    """Per-row scans of a rank-2 array: a left-to-right running sum, and a right-to-left running maximum of a fused map."""
+    sh = (rows, cols)
+    nodes = [
+        _inp("x", "f32", sh),
+        Node("scanl", "f32", sh, (0,), 1, fn="add", name="prefix"),
+        Node("map", "f32", sh, (0,), 1, fn="affine", fparam=(-2.0, 0.5), name="m"),
+        Node("scanr", "f32", sh, (2,), 1, fn="max", name="suffix_max"),
+    ]
+    return Program("row_scans", nodes, [1, 3])
+
+
+def suffix_sums(n=1 << 16):
+    """Right-to-left wrapping running sum of a masked int32 array."""
+    nodes = [
+        _inp("x", "i32", (n,)),
+        Node("map", "i32", (n,), (0,), 1, fn="and_mask", iparam=(0xFFFFF,), name="g"),
+        Node("scanr", "i32", (n,), (1,), 1, fn="add", name="suffix"),
+    ]
+    return Program("suffix_sums", nodes, [2])
+
+
 CONFIGS = {1: config1, 2: config2, 3: config3, 4: config4, 5: config5}
