@@ -329,11 +329,11 @@ def run_ours(args):
     wtop = [w for w in loads if w.cfg == top][0]
     peak, peak_kind = measured_peak()
     achieved = kernel_bytes[top](wtop) / (per[top]["ms_fused"] / kernel_launches[top]) / 1e6
-    names = {2: "k_tile_pair<transpose+zip+fold>", 3: "k_scan<hash+gather+mask+scan>", 4: "k_stream<jacobi iteration>",
+    names = {2: "k_tile_pair<transpose+zip+fold>", 3: "k_scan<hash+gather+mask+scan>", 4: "k_stencil<jacobi iteration>",
              5: "k_hist<hash+generate+permute+fold>", 1: "k_stream<chain>"}
     # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
     # summarised under profiles/, taken at these sizes; null for a kernel without a capture
-    ncu_traffic = {3: 6.267e9 + 0.258e9, 4: 268.4e6 + 226.8e6, 2: 269.4e6 + 6.2e6, 5: 542.6e6 + 3.9e6}
+    ncu_traffic = {3: 6.266e9 + 0.259e9, 4: 268.7e6 + 217.1e6, 2: 269.5e6 + 7.8e6, 5: 542.6e6 + 4.4e6}
     traffic = ncu_traffic.get(top) if args.shrink == 0 else None
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": traffic, "kernel": names[top], "of": peak_kind,
