@@ -171,8 +171,8 @@ k_stencil(const __grid_constant__ Args<CL::c.n> a, const __grid_constant__ Stenc
   for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
     // the other stage was last read before the barrier that ended the previous trip
     if (threadIdx.x == 0 && tile + gridDim.x < n_tiles) issue(tile + gridDim.x, stage ^ 1);
-    if (!wait_phase(&bar[stage], parity[stage])) atomicOr(a.status, kStatusTimeout);
-    parity[stage] ^= 1u;
+    const bool arrived = wait_phase(&bar[stage], parity[stage]);
+    if (!arrived) atomicOr(a.status, kStatusTimeout);
 
     const uint32_t ty = tile / tiles_x, tx = tile - ty * tiles_x;
     const uint32_t* box = boxes + stage * E * kStBoxStride;
@@ -189,7 +189,17 @@ k_stencil(const __grid_constant__ Args<CL::c.n> a, const __grid_constant__ Stenc
         });
       }
     }
-    __syncthreads();
+    // a stage that never arrived ends the walk: the block waits once more, again with a limit, for
+    // the copies it still has in flight (they must not land in the shared memory of a block that
+    // has gone) and returns; the host reports the status bit
+    if (__syncthreads_or(!arrived)) {
+      if (threadIdx.x == 0) {
+        if (!arrived) wait_phase(&bar[stage], parity[stage]);
+        if (tile + gridDim.x < n_tiles) wait_phase(&bar[stage ^ 1], parity[stage ^ 1]);
+      }
+      break;
+    }
+    parity[stage] ^= 1u;
     stage ^= 1;
   }
 }
