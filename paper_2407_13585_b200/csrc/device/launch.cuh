@@ -161,6 +161,49 @@ struct Launcher {
     }
   }
 
+  // Tile pairs staged by tensor copies (k_tile_pair_tma): clusters whose roots are row folds, rows
+  // 16-byte friendly.
+  // Returns ACC_OK after a launch, an error, or 1 when k_tile_pair should run instead.
+  static int launch_tiles_tma(const ClusterLaunch& L, dev::Args<N>& a, int n, bool vec) {
+    if constexpr (dev::tile_tma_eligible<CL>()) {
+      if (!vec || !cooperative_launch_ok()) return 1;
+      dev::TileMaps maps;
+      for (int i = 0; i < N; ++i)
+        if (dev::is_staged_external<CL>(i) &&
+            !make_tensor_map_2d(&maps.m[dev::tile_slot<CL>(i)], L.nodes[i].ptr, n, n, dev::kTile, dev::kTpBoxCols, true))
+          return 1;
+      auto kern = dev::k_tile_pair_tma<CL>;
+      constexpr int E = dev::staged_externals<CL>();
+      const size_t smem = (size_t)dev::tp_stages<E>() * E * dev::kTpSlotWords * 4 + 1024;   // + room to align to the swizzle
+      static int fit_on[64];                               // blocks of this kernel per SM, + 1, by device (asked once each)
+      int device = 0;
+      if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) { cudaGetLastError(); return 1; }
+      int per_sm = fit_on[device] - 1;
+      if (per_sm < 0) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+          return set_error(ACC_ERR_CUDA, "shared-memory opt-in failed: %s", cudaGetErrorString(cudaGetLastError()));
+        int fit = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&fit, kern, dev::kTpThreads, smem) != cudaSuccess) {
+          cudaGetLastError();
+          fit = 0;
+        }
+        per_sm = fit;
+        fit_on[device] = fit + 1;
+      }
+      if (per_sm < 1) return 1;
+      const int64_t blocks = (n + dev::kTile - 1) / dev::kTile;
+      const int64_t pairs = blocks * (blocks + 1) / 2;
+      const int grid = (int)std::min<int64_t>(pairs, (int64_t)sm_count() * per_sm);
+      void* params[] = {&a, &maps};                        // all blocks resident: they meet at a counter after their walk
+      cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kern), dim3(grid), dim3(dev::kTpThreads), params, smem, L.stream);
+      const cudaError_t e = cudaGetLastError();
+      if (e != cudaSuccess) return set_error(ACC_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+      return ACC_OK;
+    } else {
+      return 1;
+    }
+  }
+
   // Whether the scatter's bins go on chip: they must fit (see hist_plan) and there must be
   // enough elements per bin to repay clearing and flushing them.
   static bool use_hist(const ClusterLaunch& L, int R, int C, dev::HistPlan& plan) {
@@ -193,6 +236,8 @@ struct Launcher {
     fill(L, a, R, C);
     if (use_tiles(L, R, C)) {
       if constexpr (kTileShape) {
+        const int rc = launch_tiles_tma(L, a, R, vec);
+        if (rc != 1) return rc;                          // 1 = no tensor copies here: the threads stage the tiles
         auto kern = vec ? dev::k_tile_pair<CL, true> : dev::k_tile_pair<CL, false>;
         const size_t smem = (size_t)dev::staged_externals<CL>() * 2 * dev::kTileWords * 4;
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)

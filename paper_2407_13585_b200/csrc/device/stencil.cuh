@@ -11,7 +11,7 @@
 // the array first, and a clamped position always lies inside the tile or its halo.  All five
 // reads of a Jacobi iteration are then shared-memory reads.
 //
-// Every wait on an mbarrier is bounded: after kStSpinLimit polls the thread records
+// Every wait on an mbarrier is bounded: after kCopySpinLimit polls the thread records
 // ACC_ERR_DEVICE_TIMEOUT in the status word and goes on, so a lost copy cannot hang the GPU.
 #pragma once
 #include <cuda.h>
@@ -29,7 +29,6 @@ constexpr int kStBoxWords = kStBoxRows * kStBoxCols;  // 4624 words = 18496 byte
 constexpr int kStBoxStride = (kStBoxWords + 31) / 32 * 32;   // boxes start on 128-byte boundaries
 constexpr int kStStages = 2;
 constexpr int kStMaxExternals = 2;
-constexpr uint32_t kStSpinLimit = 1u << 20;
 
 struct StencilMaps { CUtensorMap m[kStMaxExternals]; };
 
@@ -113,23 +112,6 @@ template <class CL, int I, class A>
 __device__ __forceinline__ V4 ld_ext(const A&, const IxH4& ix) { return ld_box(tile_slot<CL>(I), ix); }
 template <class CL, int I, class A>
 __device__ __forceinline__ V4 ld_ext(const A& a, const IxHS4& ix) { return ld_box(tile_slot<CL>(I), ix, a.n[I].C); }
-
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-// Polls an mbarrier phase; false if it did not complete within the limit.
-__device__ __forceinline__ bool wait_phase(uint64_t* bar, uint32_t parity) {
-  const uint32_t addr = smem_addr(bar);
-  for (uint32_t spins = 0; spins < kStSpinLimit; ++spins) {
-    uint32_t done;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done) : "r"(addr), "r"(parity), "r"(2000u) : "memory");   // the thread may sleep up to 2 us per poll
-    if (done) return true;
-  }
-  return false;
-}
 
 template <class CL>
 __global__ void __launch_bounds__(kBlock)

@@ -18,6 +18,8 @@
 // each row goes to scratch, and the CTA that delivers the last partial of a block of rows adds
 // them up in a fixed order (so the result does not depend on arrival order) and writes them.
 #pragma once
+#include <cuda.h>
+
 #include "skeletons.cuh"
 
 namespace acc {
@@ -279,6 +281,318 @@ __global__ void __launch_bounds__(kBlock) k_tile_pair(const __grid_constant__ Ar
         });
       }
     }
+  }
+}
+
+// =========================================================================================
+// k_tile_pair_tma: the same pairing of tiles for clusters whose roots are row folds, with the
+// source tiles brought in by tensor copies (cp.async.bulk.tensor, no multicast) and the fold
+// bookkeeping taken off the critical path.
+//
+// A persistent CTA of eight consumer warps and a copy warp walks pairs p = blockIdx.x,
+// blockIdx.x + gridDim.x, ...  One lane of the copy warp issues the copies of a pair against
+// the stage's `full` mbarrier as soon as the consumers have released that stage (`empty`), so
+// up to kStages pairs are in flight.  A 64 x 64 tile arrives as two boxes of 64 rows x 32 words
+// (rows of 128 bytes) in the 128-byte swizzle: the 16-byte chunk q of row r of a box lies at
+// chunk q ^ (r & 7).  Parts of a box outside the array arrive as zeros and are never used.
+//
+// A consumer thread owns a 4 x 4 block of the output tile: four 128-bit reads give its block of
+// the tile that lies like the output, four more its block of the tile read transposed (whose
+// rows are the output's columns, so the transpose happens in registers).  The eight lanes that
+// share a 128-bit shared-memory access sit on a diagonal of blocks (block column l, block row
+// (l + d) mod 8), which makes both reads free of bank conflicts in the swizzled layout.  A
+// consumer warp releases the stage as soon as its blocks are in registers.  Row sums of the
+// blocks are combined through a small shared array (fixed order) and one partial per row and
+// tile goes to scratch.
+//
+// The kernel is launched cooperatively (all blocks resident).  After its walk a block
+// arrives at a grid-wide counter; once every block has arrived, each block adds up, in
+// column-tile order, the partials of its own slice of rows.  Publishing per pair instead
+// (fence + counter per block of rows, last arriver sums) was measured: the sum of 128 partials
+// for 64 rows by whichever block arrived last took 0.36 ms of tail at 8192 x 8192.
+//
+// Every wait is bounded (wait_phase; kCopySpinLimit polls of the counter); a wait that runs out
+// sets the time-out bit of the status word and the block's `abort` word, which ends the walk of
+// every warp; the copy warp then still waits, with the same bound, for copies in flight before
+// it leaves, and the block still arrives at the counter so that no other block waits for it.
+constexpr int kTpBoxCols = 32;
+constexpr int kTpBoxWords = kTile * kTpBoxCols;      // 2048 words = 8 KB per copy
+constexpr int kTpTileWords = 2 * kTpBoxWords;        // left and right half of a tile
+constexpr int kTpSlotWords = 2 * kTpTileWords;       // tiles [I,J] and [J,I] of one external
+constexpr int kTpMaxExternals = 3;
+constexpr int kTpConsumers = 256;                    // eight warps of 4 x 4 blocks = one 64 x 64 tile
+constexpr int kTpThreads = kTpConsumers + 32;                // + the copy warp
+constexpr int kTpRedStride = 20;                     // words per row of the row-sum exchange (16 used)
+constexpr uint32_t kCopySpinLimit = 1u << 20;
+template <int E> constexpr int tp_stages() { return E <= 2 ? 3 : 2; }
+
+struct TileMaps { CUtensorMap m[kTpMaxExternals]; };
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// Polls an mbarrier phase; false if it did not complete within the limit.
+__device__ __forceinline__ bool wait_phase(uint64_t* bar, uint32_t parity) {
+  const uint32_t addr = smem_addr(bar);
+  for (uint32_t spins = 0; spins < kCopySpinLimit; ++spins) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(addr), "r"(parity), "r"(2000u) : "memory");   // the thread may sleep up to 2 us per poll
+    if (done) return true;
+  }
+  return false;
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+// Barrier 1 over the consumer threads only, returning the OR of their predicates.
+__device__ __forceinline__ bool consumers_or(bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.or.pred p, 1, %2, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r) : "r"((uint32_t)pred), "n"(kTpConsumers) : "memory");
+  return r != 0;
+}
+
+// The thread's blocks of every staged external, in registers.
+struct BlkCtx {
+  uint4 D[kTpMaxExternals][4];   // row j of the block of the tile that lies like the output
+  uint4 T[kTpMaxExternals][4];   // row i of the block of the other tile = column i of the output block
+};
+// row r = r0 + 4*by + j of the output, columns c..c+3, as it lies / transposed
+struct IxB4  { int r, c, j; const BlkCtx* b; };
+struct IxBT4 { int r, c, j; const BlkCtx* b; };     // positions (c..c+3, r) of the source
+
+__device__ __forceinline__ Ix lane(const IxB4& i, int k) { return Ix{i.r, i.c + k}; }
+__device__ __forceinline__ Ix lane(const IxBT4& i, int k) { return Ix{i.c + k, i.r}; }
+
+template <int F> __device__ __forceinline__ auto map_index(const IxB4& i, const NodeArg&, const NodeArg&) {
+  static_assert(F == ACC_IDX_IDENTITY || F == ACC_IDX_TRANSPOSE, "only transposes are staged in tiles");
+  if constexpr (F == ACC_IDX_IDENTITY) return i;
+  else return IxBT4{i.r, i.c, i.j, i.b};
+}
+template <int F> __device__ __forceinline__ auto map_index(const IxBT4& i, const NodeArg&, const NodeArg&) {
+  static_assert(F == ACC_IDX_IDENTITY || F == ACC_IDX_TRANSPOSE, "only transposes are staged in tiles");
+  if constexpr (F == ACC_IDX_IDENTITY) return i;
+  else return IxB4{i.r, i.c, i.j, i.b};
+}
+
+__device__ __forceinline__ uint32_t word_of(const uint4& v, int j) { return j == 0 ? v.x : j == 1 ? v.y : j == 2 ? v.z : v.w; }
+
+template <class CL, int I, class A>
+__device__ __forceinline__ V4 ld_ext(const A&, const IxB4& ix) {
+  const uint4 v = ix.b->D[tile_slot<CL>(I)][ix.j];
+  return V4{{v.x, v.y, v.z, v.w}};
+}
+template <class CL, int I, class A>
+__device__ __forceinline__ V4 ld_ext(const A&, const IxBT4& ix) {
+  const uint4* t = ix.b->T[tile_slot<CL>(I)];
+  return V4{{word_of(t[0], ix.j), word_of(t[1], ix.j), word_of(t[2], ix.j), word_of(t[3], ix.j)}};
+}
+
+// Clusters this skeleton takes: tile-eligible, every root a row fold.
+template <class CL> constexpr bool tile_tma_eligible() {
+  if (!tile_eligible<CL>()) return false;
+  for (int i = 0; i < CL::c.n; ++i)
+    if (is_store_root(CL::c.nodes[i])) return false;
+  return count_if<CL>(is_row_fold) >= 1 && count_if<CL>(is_row_fold) <= 2;
+}
+
+template <class CL>
+__global__ void __launch_bounds__(kTpThreads) k_tile_pair_tma(const __grid_constant__ Args<CL::c.n> a,
+                                                              const __grid_constant__ TileMaps maps) {
+  constexpr int N = CL::c.n;
+  constexpr int NRF = count_if<CL>(is_row_fold);
+  constexpr int E = staged_externals<CL>();
+  constexpr int S = tp_stages<E>();
+  constexpr int kStageWords = E * kTpSlotWords;
+  extern __shared__ uint32_t tp_raw[];
+  __shared__ __align__(8) uint64_t full[S], empty[S];
+  __shared__ uint32_t abort_walk;        // set by whoever ran out of patience
+  __shared__ __align__(16) uint32_t red[2][NRF][kTile][kTpRedStride];
+  // the swizzle pattern is laid over 1024-byte blocks of shared memory
+  uint32_t* const tiles = tp_raw + ((1024u - (smem_addr(tp_raw) & 1023u)) & 1023u) / 4;
+  const int n = a.R;                                        // square domain: n x n
+  const int blocks = (n + kTile - 1) / kTile;
+  const uint32_t n_pairs = (uint32_t)blocks * (uint32_t)(blocks + 1) / 2;
+  uint32_t* const arrivals = a.scratch;                     // blocks that have finished their walk
+  uint32_t* partials = a.scratch + tile_partials_off(blocks);
+  const int lane_id = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&empty[s], kTpConsumers / 32);
+    }
+    abort_walk = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  volatile uint32_t* const v_abort = &abort_walk;
+
+  if (threadIdx.x >= kTpConsumers) {
+    // ---------------- copy warp: one lane keeps kStages - 1 pairs in flight ---------------------
+    if (lane_id != 0) return;
+    auto issue = [&](uint32_t pair, int stage) {
+      int I, J;
+      pair_of(pair, blocks, I, J);
+      const int n_tiles = I == J ? 1 : 2;
+      const uint32_t b = smem_addr(&full[stage]);
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"((uint32_t)(E * n_tiles * kTpTileWords * 4)) : "memory");
+#pragma unroll
+      for (int slot = 0; slot < E; ++slot) {
+        for (int t = 0; t < n_tiles; ++t) {
+          const int y = (t == 0 ? I : J) * kTile, x = (t == 0 ? J : I) * kTile;   // x: a multiple of 64 words
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const uint32_t dst = smem_addr(tiles + stage * kStageWords + slot * kTpSlotWords + t * kTpTileWords + h * kTpBoxWords);
+            asm volatile(
+                "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                ::"r"(dst), "l"(&maps.m[slot]), "r"(x + h * kTpBoxCols), "r"(y), "r"(b) : "memory");
+          }
+        }
+      }
+    };
+    uint32_t trip = 0;                                      // trips whose copies have been started
+    bool ok = true;
+    for (uint32_t pair = blockIdx.x; pair < n_pairs; pair += gridDim.x, ++trip) {
+      // its stage held trip - S: every consumer warp must have let go of that
+      if (trip >= (uint32_t)S) ok = wait_phase(&empty[trip % S], (trip / S - 1) & 1u) && !*v_abort;
+      if (!ok) break;
+      issue(pair, (int)(trip % S));
+    }
+    if (!ok) {
+      if (!*v_abort) { *v_abort = 1; atomicOr(a.status, kStatusTimeout); }
+      // copies still in flight must not land in the shared memory of a block that has gone
+      for (uint32_t q = 1; q <= (uint32_t)S && q <= trip; ++q) wait_phase(&full[(trip - q) % S], ((trip - q) / S) & 1u);
+    }
+    return;
+  }
+
+  // ---------------- consumer warps ------------------------------------------------------------
+  const int l = threadIdx.x & 7, dg = (threadIdx.x >> 3) & 7, quad = threadIdx.x >> 6;
+  const int bx = (quad & 1) * 8 + l, by = (quad >> 1) * 8 + ((l + dg) & 7);   // the thread's 4 x 4 block
+  int dofs[4], tofs[4];                                     // word offsets of the block's rows in a tile
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int dr = 4 * by + i, tr = 4 * bx + i;
+    dofs[i] = (bx >> 3) * kTpBoxWords + dr * kTpBoxCols + (((bx & 7) ^ (dr & 7)) << 2);
+    tofs[i] = (by >> 3) * kTpBoxWords + tr * kTpBoxCols + (((by & 7) ^ (tr & 7)) << 2);
+  }
+  const int red_row = threadIdx.x >> 2, red_q = threadIdx.x & 3;
+  int tp = 0;                                               // which half of `red` this tile uses
+  uint32_t it = 0;
+  for (uint32_t pair = blockIdx.x; pair < n_pairs; pair += gridDim.x, ++it) {
+    const int stage = (int)(it % S);
+    const bool arrived = wait_phase(&full[stage], (it / S) & 1u) && !*v_abort;
+    if (!arrived && !*v_abort) { *v_abort = 1; atomicOr(a.status, kStatusTimeout); }
+    int I, J;
+    pair_of(pair, blocks, I, J);
+    const int n_tiles = I == J ? 1 : 2;
+    bool stop = false;
+    // ---- output tile (I,J), then (J,I) with the roles of the two staged tiles swapped --------
+    for (int o = 0; o < n_tiles; ++o) {
+      const int r0 = (o == 0 ? I : J) * kTile, c0 = (o == 0 ? J : I) * kTile;
+      const int direct = (I == J) ? 0 : o, trans = (I == J) ? 0 : 1 - o;
+      const int col_tile = o == 0 ? J : I;
+      BlkCtx ctx;
+#pragma unroll
+      for (int slot = 0; slot < E; ++slot) {
+        const uint32_t* sb = tiles + stage * kStageWords + slot * kTpSlotWords;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          ctx.D[slot][i] = *reinterpret_cast<const uint4*>(sb + direct * kTpTileWords + dofs[i]);
+          ctx.T[slot][i] = *reinterpret_cast<const uint4*>(sb + trans * kTpTileWords + tofs[i]);
+        }
+      }
+      if (o == n_tiles - 1) {                               // the stage is in registers: let it be refilled
+        __syncwarp();
+        if (lane_id == 0) mbar_arrive(&empty[stage]);
+      }
+      const int r = r0 + 4 * by, c = c0 + 4 * bx;           // n is a multiple of 4: a block is inside or outside
+      const bool inside = r < n && c < n;
+      static_for<0, N>([&](auto ic) {
+        constexpr int i = decltype(ic)::value;
+        constexpr CNode nd = CL::c.nodes[i];
+        if constexpr (is_row_fold(nd)) {
+          constexpr int ord = count_if<CL>(is_row_fold, i);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            uint32_t s = identity_of<nd.fn, nd.dtype>();
+            if (inside) {
+              const V4 v = eval<CL, nd.in[0]>(a, IxB4{r + j, c, j, &ctx});
+              s = combine<nd.fn, nd.dtype>(combine<nd.fn, nd.dtype>(v.v[0], v.v[1]), combine<nd.fn, nd.dtype>(v.v[2], v.v[3]));
+            }
+            red[tp][ord][4 * by + j][bx] = s;
+          }
+        }
+      });
+      stop = consumers_or(!arrived);
+      static_for<0, N>([&](auto ic) {
+        constexpr int i = decltype(ic)::value;
+        constexpr CNode nd = CL::c.nodes[i];
+        if constexpr (is_row_fold(nd)) {
+          constexpr int ord = count_if<CL>(is_row_fold, i);
+          const uint4 v = *reinterpret_cast<const uint4*>(&red[tp][ord][red_row][4 * red_q]);
+          uint32_t s = combine<nd.fn, nd.dtype>(combine<nd.fn, nd.dtype>(v.x, v.y), combine<nd.fn, nd.dtype>(v.z, v.w));
+          s = combine<nd.fn, nd.dtype>(s, __shfl_xor_sync(0xFFFFFFFFu, s, 1));
+          s = combine<nd.fn, nd.dtype>(s, __shfl_xor_sync(0xFFFFFFFFu, s, 2));
+          if (red_q == 0 && r0 + red_row < n) partials[((size_t)ord * blocks + col_tile) * n + r0 + red_row] = s;
+        }
+      });
+      tp ^= 1;            // the next tile writes the other half: this one is still being read
+      if (stop) break;
+    }
+    if (stop) break;      // agreed on by all consumers at the barrier above
+  }
+
+  // ---- every block has walked: add up this block's slice of rows --------------------------------
+  // (barrier 1 makes the consumers' partials visible to thread 0, whose fence orders them before
+  // its arrival; the fence after the wait orders the other blocks' partials before the reads)
+  consumers_or(false);
+  if (threadIdx.x == 0) {
+    __threadfence();
+    atomicAdd(arrivals, 1u);
+    uint32_t spins = 0;
+    while (*reinterpret_cast<volatile uint32_t*>(arrivals) < gridDim.x) {
+      if (++spins > kCopySpinLimit) { atomicOr(a.status, kStatusTimeout); break; }
+      __nanosleep(200);
+    }
+    __threadfence();
+  }
+  consumers_or(false);
+  const int per_block = (n + (int)gridDim.x - 1) / (int)gridDim.x;
+  const int slice0 = (int)blockIdx.x * per_block, slice1 = min(n, slice0 + per_block);
+  for (int base = slice0; base < slice1; base += kTpConsumers / 4) {
+    const int row = base + red_row;
+    static_for<0, N>([&](auto ic) {
+      constexpr int i = decltype(ic)::value;
+      constexpr CNode nd = CL::c.nodes[i];
+      if constexpr (is_row_fold(nd)) {
+        constexpr int ord = count_if<CL>(is_row_fold, i);
+        const uint32_t* part = partials + (size_t)ord * blocks * n + min(row, n - 1);
+        uint32_t s = identity_of<nd.fn, nd.dtype>();
+        for (int t = red_q; t < blocks; t += 128) {          // this thread's column tiles: t, t + 4, ...
+          uint32_t v[32];                                     // all in flight together (128 tiles = 8192 columns per trip)
+#pragma unroll
+          for (int u = 0; u < 32; ++u) v[u] = __ldcg(part + (size_t)min(t + 4 * u, blocks - 1) * n);
+#pragma unroll
+          for (int u = 0; u < 32; ++u)
+            if (t + 4 * u < blocks) s = combine<nd.fn, nd.dtype>(s, v[u]);
+        }
+        s = combine<nd.fn, nd.dtype>(s, __shfl_xor_sync(0xFFFFFFFFu, s, 1));
+        s = combine<nd.fn, nd.dtype>(s, __shfl_xor_sync(0xFFFFFFFFu, s, 2));
+        if (red_q == 0 && row < slice1) reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr))[row] = s;
+      }
+    });
   }
 }
 

@@ -32,8 +32,9 @@ void register_kernel(const KernelEntry& e);
 const KernelEntry* find_kernel(const std::string& sig);
 int registry_size();
 int sm_count();
+bool cooperative_launch_ok();   // the current device can run a grid with all blocks resident
 // Fills the CUtensorMap at `out` for box copies from a row-major rows x cols array of 4-byte
 // elements; false if the driver call is unavailable or the array is not 16-byte friendly.
-bool make_tensor_map_2d(void* out, const void* base, int rows, int cols, int box_rows, int box_cols);
+bool make_tensor_map_2d(void* out, const void* base, int rows, int cols, int box_rows, int box_cols, bool swizzle_128b = false);
 
 }  // namespace acc

@@ -36,8 +36,10 @@ def test_config1_all_partitions(n):
 
 
 # below one 64 x 64 tile: generic kernels; from 64 rows on: shared-memory tile pairs, with ragged
-# edge tiles (100, 130), without 128-bit accesses (130, 67) and on whole tiles (64, 256)
-@pytest.mark.parametrize("rows", [1, 4, 33, 64, 67, 100, 130, 256])
+# edge tiles (100, 130), without 128-bit accesses (130, 67: the threads stage the tiles; otherwise
+# tensor copies do) and on whole tiles (64, 256); 1600 and 2052 give every persistent block
+# several tile pairs, 2052 with an edge tile that lies almost wholly outside the array
+@pytest.mark.parametrize("rows", [1, 4, 33, 64, 67, 100, 130, 256, 1600, 2052])
 def test_config2_all_partitions(rows):
     assert check_program(W.config2(rows)) == 4
 
