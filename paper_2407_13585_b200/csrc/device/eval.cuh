@@ -23,7 +23,22 @@ struct NodeArg {
   int32_t ip0, ip1;  // iparam[0..1] (uint32 constants keep their bit pattern)
   float fp0, fp1;    // fparam[0..1]
   int32_t R, C;      // shape as (rows, innermost extent); rank 1 -> R = 1; rank 0 -> 1 x 1
+  // division by a run-time constant d without a divider and without a branch, filled by the
+  // host (d = iparam[1] for ACC_FN_MUL_MOD, iparam[0] otherwise, 1 <= d < 2^32): for every 32-bit
+  // v, with t = umulhi(v, div_mul):  v / d == (t + ((v - t) >> div_sh1)) >> div_sh2
+  uint32_t div_mul, div_sh1, div_sh2;
+  uint32_t div_mask;   // d - 1 when d is a power of two (> 1), else 0: then v mod d is one AND
 };
+
+// v / d and v mod d with the host's multiplier for d (see NodeArg).
+__device__ __forceinline__ uint32_t div_by(uint32_t v, const NodeArg& p) {
+  const uint32_t t = __umulhi(v, p.div_mul);
+  return (t + ((v - t) >> p.div_sh1)) >> p.div_sh2;
+}
+__device__ __forceinline__ uint32_t mod_by(uint32_t v, uint32_t d, const NodeArg& p) {
+  if (p.div_mask != 0) return v & p.div_mask;             // the same for every thread of the launch
+  return v - div_by(v, p) * d;
+}
 
 template <int N>
 struct Args {
@@ -44,6 +59,15 @@ struct IxR4 { int r, c; };            // c, c-1, c-2, c-3  ((c-3) % 4 == 0)
 struct IxS4 { int r, c, dc; };        // clamp(c+dc+i, 0, C-1) for i = 0..3, row r (c % 4 == 0)
 struct IxG4 { Ix e[4]; };             // four unrelated positions
 
+// Two kinds that move no data: IxPF4 asks L2 to fetch the lines of a chunk that will be read a
+// few trips later, IxNone is what becomes of it behind an index map it cannot follow.  Evaluating
+// a member at either one touches no array (values come back as zeros and are dropped).
+struct IxPF4 { int r, c; };
+struct IxNone { int r, c; };
+template <class IX> struct is_prefetch { static constexpr bool value = false; };
+template <> struct is_prefetch<IxPF4> { static constexpr bool value = true; };
+template <> struct is_prefetch<IxNone> { static constexpr bool value = true; };
+
 template <class IX> struct width_of { static constexpr int value = 4; };
 template <> struct width_of<Ix> { static constexpr int value = 1; };
 template <class IX> using val_of = std::conditional_t<width_of<IX>::value == 1, uint32_t, V4>;
@@ -52,6 +76,8 @@ __device__ __forceinline__ Ix lane(const Ix& i, int) { return i; }
 __device__ __forceinline__ Ix lane(const Ix4& i, int j) { return Ix{i.r, i.c + j}; }
 __device__ __forceinline__ Ix lane(const IxR4& i, int j) { return Ix{i.r, i.c - j}; }
 __device__ __forceinline__ Ix lane(const IxG4& i, int j) { return i.e[j]; }
+__device__ __forceinline__ Ix lane(const IxPF4& i, int j) { return Ix{i.r, i.c + j}; }
+__device__ __forceinline__ Ix lane(const IxNone& i, int j) { return Ix{i.r, i.c + j}; }
 __device__ __forceinline__ Ix lane_clamped(const IxS4& i, int j, int C) {
   return Ix{i.r, min(max(i.c + i.dc + j, 0), C - 1)};
 }
@@ -71,6 +97,11 @@ __device__ __forceinline__ V4 ld(const uint32_t* p, int C, const IxR4& i) {
 __device__ __forceinline__ V4 ld(const uint32_t* p, int C, const IxG4& i) {
   return V4{{ld1(p, C, i.e[0]), ld1(p, C, i.e[1]), ld1(p, C, i.e[2]), ld1(p, C, i.e[3])}};
 }
+__device__ __forceinline__ V4 ld(const uint32_t* p, int C, const IxPF4& i) {
+  asm volatile("prefetch.global.L2 [%0];" ::"l"(p + (i.r * C + i.c)));
+  return V4{{0u, 0u, 0u, 0u}};
+}
+__device__ __forceinline__ V4 ld(const uint32_t*, int, const IxNone&) { return V4{{0u, 0u, 0u, 0u}}; }
 // A row chunk shifted by dc columns: the aligned chunk itself plus the one element that
 // slides in from the neighbouring chunk (|dc| = 1), clamped at the row ends.
 __device__ __forceinline__ V4 ld(const uint32_t* p, int C, const IxS4& i) {
@@ -128,6 +159,12 @@ template <int F> __device__ __forceinline__ auto map_index(const IxG4& i, const 
   if constexpr (F == ACC_IDX_IDENTITY) return i;
   else return map_lanes<F>(i, self, src);
 }
+template <int F> __device__ __forceinline__ auto map_index(const IxPF4& i, const NodeArg&, const NodeArg& src) {
+  if constexpr (F == ACC_IDX_IDENTITY) return i;
+  else if constexpr (F == ACC_IDX_REVERSE) return IxPF4{src.R - 1 - i.r, src.C - 4 - i.c};
+  else return IxNone{0, 0};
+}
+template <int F> __device__ __forceinline__ auto map_index(const IxNone& i, const NodeArg&, const NodeArg&) { return i; }
 // A shifted chunk names positions in the array it is applied to, which has the shape of
 // the node that receives it (`self`); a further map acts on its four clamped lanes.
 template <int F> __device__ __forceinline__ auto map_index(const IxS4& i, const NodeArg& self, const NodeArg& src) {
@@ -148,8 +185,8 @@ __device__ __forceinline__ uint32_t apply1(const NodeArg& p, uint32_t a, uint32_
   else if constexpr (FN == ACC_FN_HASH_MUL_XORSHIFT) return (a * (uint32_t)p.ip0) ^ (a >> (uint32_t)p.ip1);
   else if constexpr (FN == ACC_FN_AND_MASK) return a & (uint32_t)p.ip0;
   else if constexpr (FN == ACC_FN_MUL_MOD) {
-    const uint32_t m = (uint32_t)p.ip1, t = a * (uint32_t)p.ip0;
-    return (m & (m - 1)) == 0 ? (t & (m - 1)) : (t % m);
+    const uint32_t t = a * (uint32_t)p.ip0;
+    return mod_by(t, (uint32_t)p.ip1, p);
   }
   else if constexpr (FN == ACC_FN_MUL_CONST) return a * (uint32_t)p.ip0;
   else if constexpr (FN == ACC_FN_ADD_CONST) return a + (uint32_t)p.ip0;
@@ -175,7 +212,7 @@ template <int FN, int DT>
 __device__ __forceinline__ uint32_t generate1(const NodeArg& p, const Ix& i, uint32_t free0) {
   const uint32_t lin = (uint32_t)(i.r * p.C + i.c);
   if constexpr (FN == ACC_FN_IOTA) { if constexpr (DT == ACC_F32) return u_((float)lin); else return lin; }
-  else if constexpr (FN == ACC_FN_IMOD_TO_F32) return u_((float)(lin % (uint32_t)p.ip0));
+  else if constexpr (FN == ACC_FN_IMOD_TO_F32) return u_((float)mod_by(lin, (uint32_t)p.ip0, p));
   else if constexpr (FN == ACC_FN_ROW_INDEX) return (uint32_t)i.r;
   else if constexpr (FN == ACC_FN_IOTA_PLUS_FREE) return u_(__fadd_rn((float)lin, f_(free0)));
   else { static_assert(FN < 0, "not a generate function"); return 0; }
@@ -259,6 +296,11 @@ __device__ __forceinline__ val_of<IX> eval(const A& a, const IX& ix) {
     return ld_ext<CL, I>(a, ix);
   } else if constexpr (nd.kind == ACC_BACKPERMUTE) {
     return eval<CL, nd.in[0]>(a, map_index<nd.idxfn>(ix, a.n[I], a.n[nd.in[0]]));
+  } else if constexpr (is_prefetch<IX>::value && (nd.kind == ACC_GATHER || nd.kind == ACC_FOLD || nd.kind == ACC_FOLDSEG)) {
+    // where the data will be read from is not known before the data: only a gather's index
+    // operand, read in the cluster's own order, can be fetched ahead
+    if constexpr (nd.kind == ACC_GATHER) eval<CL, nd.in[0]>(a, ix);
+    return V4{{0u, 0u, 0u, 0u}};
   } else if constexpr (nd.kind == ACC_GATHER) {
     constexpr int src_rank = CL::c.nodes[nd.in[1]].rank;
     const auto k = eval<CL, nd.in[0]>(a, ix);
@@ -317,12 +359,16 @@ __device__ __forceinline__ val_of<IX> eval(const A& a, const IX& ix) {
     } else if constexpr (std::is_same<IX, Ix4>::value && nd.fn == ACC_FN_IMOD_TO_F32) {
       // one division for four consecutive indices: the remainders follow by stepping
       const uint32_t m = (uint32_t)a.n[I].ip0;
-      uint32_t r = (uint32_t)(ix.r * a.n[I].C + ix.c) % m;
-      const bool small = m <= (1u << 23);      // then float(r) = bits(2^23 + r) - 2^23, no conversion unit
+      uint32_t r[4];
+      r[0] = mod_by((uint32_t)(ix.r * a.n[I].C + ix.c), m, a.n[I]);
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        out.v[j] = small ? u_(__fadd_rn(__uint_as_float(0x4B000000u | r), -8388608.0f)) : u_((float)r);
-        r = r + 1 == m ? 0u : r + 1;
+      for (int j = 1; j < 4; ++j) r[j] = r[j - 1] + 1 == m ? 0u : r[j - 1] + 1;
+      if (m <= (1u << 23)) {                   // then float(r) = bits(2^23 + r) - 2^23, no conversion unit
+#pragma unroll
+        for (int j = 0; j < 4; ++j) out.v[j] = u_(__fadd_rn(__uint_as_float(0x4B000000u | r[j]), -8388608.0f));
+      } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) out.v[j] = u_((float)r[j]);
       }
     } else {
 #pragma unroll

@@ -34,6 +34,7 @@ constexpr int kHistBlock = 1024;
 constexpr int kHistMaxBinsPerCta = 56 * 1024;   // 224 KiB of 32-bit bins per CTA
 constexpr int kHistOverflowBins = 16 * 1024;    // further bins kept per CTA in global memory
 constexpr int kHistUnroll = 2;                  // independent chunks in flight per thread (4 measured no faster)
+constexpr int kHistAhead = 2;                   // trips between asking L2 for a chunk and reading it
 
 struct HistPlan {
   int group;        // CTAs that split the bins
@@ -57,6 +58,28 @@ inline bool hist_plan(int64_t bins, int sms, HistPlan& p) {
   if ((p.per_cta & (p.per_cta - 1)) == 0)
     for (p.shift = 0; (1 << p.shift) < p.per_cta; ++p.shift) {}
   return true;
+}
+
+// Fire-and-forget integer add on global memory (no value comes back, so nothing waits for it).
+__device__ __forceinline__ void red_add_global(int* p, int v) {
+  asm volatile("red.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+// Adds v to bin k: bins below `per_cta` are words of shared memory from `bins_addr`, the others
+// words of global memory from `rest` (which already points per_cta words before the first of
+// them).  One comparison and two predicated fire-and-forget adds, no branch.
+__device__ __forceinline__ void red_add_bin(uint32_t k, uint32_t per_cta, uint32_t bins_addr, const int* rest, int v) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .u32 sa;\n\t.reg .u64 ga;\n\t"
+      "setp.lt.u32 p, %0, %1;\n\t"
+      "mad.lo.u32 sa, %0, 4, %2;\n\t"
+      "mad.wide.u32 ga, %0, 4, %3;\n\t"
+      "@p red.shared.add.s32 [sa], %4;\n\t"
+      "@!p red.global.add.s32 [ga], %4;\n\t}"
+      ::"r"(k), "r"(per_cta), "r"(bins_addr), "l"(rest), "r"(v) : "memory");
+}
+__device__ __forceinline__ void red_add_global(double* p, double v) {
+  asm volatile("red.global.add.f64 [%0], %1;" ::"l"(p), "d"(v) : "memory");
 }
 
 template <class CL> constexpr int the_f32_add_permute() {
@@ -160,14 +183,29 @@ k_hist(const __grid_constant__ Args<CL::c.n> a, const HistPlan plan, int* overfl
       const int v = __float_as_int(shifted) - 0x4B400000;      // bits of 12582912.0f
       // two calls, so that each is an atomic on a known address space (shared / global)
       if (at < (uint32_t)per_cta) atomicAdd(bins_smem + at, v);
-      else atomicAdd(spill + (at - (uint32_t)per_cta), v);
+      else red_add_global(spill + (at - (uint32_t)per_cta), v);
     } else {
-      atomicAdd(acc64 + k, (double)x);
+      red_add_global(acc64 + k, (double)x);
     }
   };
 
+  const bool fast_ok = group == 1 && S >= 0;
+  const uint32_t bins_addr = (uint32_t)__cvta_generic_to_shared(bins_smem);
   uint32_t it = 0;
   for (uint32_t q0 = team * kHistBlock + threadIdx.x; q0 < total; q0 += stride * U, it += U) {
+    if constexpr (VEC) {
+      // ask L2 for what the trip after next will read: there are too few registers to keep
+      // enough loads in flight to cover DRAM latency, so the loads should find their lines in L2
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const uint32_t q = q0 + (kHistAhead * U + u) * stride;
+        if (q < total) {
+          const IX ix = index_of(q);
+          eval<CL, pn.in[1]>(a, IxPF4{ix.r, ix.c});
+          eval<CL, pn.in[2]>(a, IxPF4{ix.r, ix.c});
+        }
+      }
+    }
     // evaluate U independent chunks first so that their loads are in flight together
     VAL key[U], val[U];
     bool live[U];
@@ -192,7 +230,11 @@ k_hist(const __grid_constant__ Args<CL::c.n> a, const HistPlan plan, int* overfl
           if constexpr (is_store_root(nd)) {
             st(reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr)), a.n[i].C, ix, eval<CL, i>(a, ix));
           } else if constexpr (is_scalar_fold(nd)) {
-            const auto v = eval<CL, nd.in[0]>(a, ix);
+            // a fold over the scatter's own value or index operand shares its registers
+            VAL v;
+            if constexpr (nd.in[0] == CL::c.nodes[P].in[2]) v = val[u];
+            else if constexpr (nd.in[0] == CL::c.nodes[P].in[1]) v = key[u];
+            else v = eval<CL, nd.in[0]>(a, ix);
             if constexpr (VEC) {
 #pragma unroll
               for (int j = 0; j < 4; ++j) acc[i] = combine<nd.fn, nd.dtype>(acc[i], v.v[j]);
@@ -203,8 +245,29 @@ k_hist(const __grid_constant__ Args<CL::c.n> a, const HistPlan plan, int* overfl
         });
       }
       if constexpr (VEC) {
+        // The usual case in one piece, without a branch per element: all four indices in range and
+        // all four values exact integers below `cap` after scaling.  (With up >= 1 a non-zero x
+        // cannot underflow to a zero product; otherwise the careful path below is taken.)
+        const uint32_t kmax = max(max(key[u].v[0], key[u].v[1]), max(key[u].v[2], key[u].v[3]));
+        float t[4], shifted[4], off = 0.0f, big = 0.0f;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) scatter_one(key[u].v[j], val[u].v[j]);
+        for (int j = 0; j < 4; ++j) {
+          t[j] = __fmul_rn(f_(val[u].v[j]), up);
+          shifted[j] = __fadd_rn(t[j], 12582912.0f);
+          off = __fadd_rn(off, fabsf(__fadd_rn(__fadd_rn(shifted[j], -12582912.0f), -t[j])));   // 0 iff t is an integer (NaN otherwise)
+          big = fmaxf(big, fabsf(t[j]));
+        }
+        if (fast_ok & (kmax < n_bins) & (off == 0.0f) & (big < cap)) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint32_t k = key[u].v[j];
+            // (a zero is added like any other value: skipping it would cost more than it saves)
+            red_add_bin(k, (uint32_t)per_cta, bins_addr, spill - per_cta, __float_as_int(shifted[j]) - 0x4B400000);
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) scatter_one(key[u].v[j], val[u].v[j]);
+        }
       } else {
         scatter_one(key[u], val[u]);
       }
@@ -212,14 +275,19 @@ k_hist(const __grid_constant__ Args<CL::c.n> a, const HistPlan plan, int* overfl
   }
 
   __syncthreads();
-  for (int i = threadIdx.x; i < per_cta; i += kHistBlock) {
+  // every CTA starts its sweep somewhere else, so that the CTAs that finish together do not all
+  // queue up on the same accumulators
+  const int turn = (int)((blockIdx.x * 2654435761u) >> 8);
+  for (int i0 = threadIdx.x; i0 < per_cta; i0 += kHistBlock) {
+    const int i = (int)((uint32_t)(i0 + turn) % (uint32_t)per_cta);
     const int v = bins_smem[i];
     const uint32_t bin = rank * (uint32_t)per_cta + i;
-    if (v != 0 && bin < n_bins) atomicAdd(acc64 + bin, (double)v * down);
+    if (v != 0 && bin < n_bins) red_add_global(acc64 + bin, (double)v * down);
   }
-  for (int i = threadIdx.x; i < plan.overflow; i += kHistBlock) {
+  for (int i0 = threadIdx.x; i0 < plan.overflow; i0 += kHistBlock) {
+    const int i = (int)((uint32_t)(i0 + turn) % (uint32_t)plan.overflow);
     const int v = *reinterpret_cast<volatile int*>(spill + i);
-    if (v != 0) atomicAdd(acc64 + per_cta + i, (double)v * down);
+    if (v != 0) red_add_global(acc64 + per_cta + i, (double)v * down);
   }
 
   static_for<0, N>([&](auto ic) {

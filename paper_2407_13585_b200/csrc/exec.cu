@@ -53,6 +53,18 @@ static dev::NodeArg node_arg(const Node& n, const void* ptr) {
   a.ip1 = (int32_t)(uint32_t)(n.d.iparam[1] & 0xFFFFFFFFll);
   a.fp0 = (float)n.d.fparam[0];
   a.fp1 = (float)n.d.fparam[1];
+  // branch-free division by d (Granlund and Montgomery's round-up multiplier, 33 bits with the
+  // add-and-shift fix-up): l = ceil(log2 d), m = floor(2^32 (2^l - d) / d) + 1,
+  // v / d = (t + ((v - t) >> min(l, 1))) >> max(l - 1, 0) with t = umulhi(v, m); d = 1 gives v
+  const uint32_t d = (uint32_t)(n.d.fn_id == ACC_FN_MUL_MOD ? a.ip1 : a.ip0);
+  if (d >= 1) {
+    uint32_t l = 0;
+    while (l < 32 && (1ull << l) < d) ++l;
+    a.div_mul = (uint32_t)((((1ull << l) - d) << 32) / d + 1);
+    a.div_sh1 = l < 1 ? l : 1;
+    a.div_sh2 = l - a.div_sh1;
+    a.div_mask = (d > 1 && (d & (d - 1)) == 0) ? d - 1 : 0;
+  }
   a.R = n.d.rank == 2 ? (int32_t)n.d.shape[0] : 1;
   a.C = n.d.rank == 2 ? (int32_t)n.d.shape[1] : (n.d.rank == 1 ? (int32_t)n.d.shape[0] : 1);
   return a;
