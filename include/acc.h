@@ -201,6 +201,29 @@ int64_t acc_enumerate(acc_graph* g, int32_t* out_pi, int64_t max_partitions);
 /* Cost of a legal clustering under `cost` (lower is better). */
 int acc_partition_cost(acc_graph* g, const int32_t* cluster_of_node, int32_t n_nodes, int cost, double* out);
 
+/* ---- clusterings that recompute (the paper's future work, Section 6) ----------- */
+
+/* The paper's model gives every array one traversal order, so an array read in
+ * two orders by one cluster (once as it lies and once through a backpermute, or
+ * through several backpermutes) cannot be fused away there: Section 3.3's
+ * `simple5` reads it twice from memory instead, and Section 6 leaves fusion
+ * that duplicates work to future work.  The calls below accept such clusters:
+ * with max_depth > 0 a fused-away array may be evaluated once per order it is
+ * read in, as if each consumer had its own copy of the producer (and of the
+ * producer's producers inside the cluster).  What still fails: a scan asked for
+ * an order other than its own, the one stored copy of a manifest array asked
+ * for an order above 1, every rule that is not about orders, and more than
+ * max_depth gather-like nodes stacked on one fused path.  max_depth = 0 is the
+ * paper's model (the calls above).  The arrays computed are the same as under
+ * any legal clustering; only the work and the traffic differ.
+ * Arguments and results as for the calls of the same name above. */
+int acc_check_partition_recompute(acc_graph* g, const int32_t* cluster_of_node, int32_t n_nodes, int32_t max_depth);
+int acc_set_partition_recompute(acc_graph* g, const int32_t* cluster_of_node, int32_t n_nodes, int32_t max_depth);
+int acc_plan_recompute(acc_graph* g, int mode, int cost, int32_t max_depth, int32_t* cluster_of_node_out);
+int64_t acc_enumerate_recompute(acc_graph* g, int32_t max_depth, int32_t* out_pi, int64_t max_partitions);
+int acc_partition_cost_recompute(acc_graph* g, const int32_t* cluster_of_node, int32_t n_nodes, int32_t max_depth, int cost,
+                                 double* out);
+
 /* ---- running ------------------------------------------------------------------ */
 
 /* Binds a caller-owned DEVICE buffer to a node.  Required for INPUT nodes and

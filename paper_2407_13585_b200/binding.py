@@ -84,6 +84,11 @@ def load_library(path=LIB_PATH):
         "acc_plan": (C.c_int, [p, C.c_int, C.c_int, pi32]),
         "acc_enumerate": (i64, [p, pi32, i64]),
         "acc_partition_cost": (C.c_int, [p, pi32, i32, C.c_int, C.POINTER(C.c_double)]),
+        "acc_check_partition_recompute": (C.c_int, [p, pi32, i32, i32]),
+        "acc_set_partition_recompute": (C.c_int, [p, pi32, i32, i32]),
+        "acc_plan_recompute": (C.c_int, [p, C.c_int, C.c_int, i32, pi32]),
+        "acc_enumerate_recompute": (i64, [p, i32, pi32, i64]),
+        "acc_partition_cost_recompute": (C.c_int, [p, pi32, i32, i32, C.c_int, C.POINTER(C.c_double)]),
         "acc_bind": (C.c_int, [p, i32, p, sz]),
         "acc_bind_host": (C.c_int, [p, i32, p, sz]),
         "acc_workspace_bytes": (C.c_int, [p, C.c_int, C.POINTER(sz)]),
@@ -199,6 +204,30 @@ class Graph:
     def check_partition(self, pi):
         """Status name: 'ACC_OK' or the ACC_ERR_* that says which rule failed."""
         return STATUS_NAME[lib().acc_check_partition(self._h, _i32_array(pi), len(pi))]
+
+    # clusterings that recompute: max_depth > 0 lets a fused-away array be evaluated once per order
+    # it is read in, with at most max_depth gather-like nodes stacked on a fused path
+    def set_partition_recompute(self, pi, max_depth):
+        _check(lib().acc_set_partition_recompute(self._h, _i32_array(pi), len(pi), max_depth))
+
+    def check_partition_recompute(self, pi, max_depth):
+        return STATUS_NAME[lib().acc_check_partition_recompute(self._h, _i32_array(pi), len(pi), max_depth)]
+
+    def plan_recompute(self, mode, cost, max_depth):
+        out = (C.c_int32 * self.n)()
+        _check(lib().acc_plan_recompute(self._h, PLAN[mode], COST[cost], max_depth, out))
+        return list(out)
+
+    def enumerate_recompute(self, max_depth):
+        cnt = _check(lib().acc_enumerate_recompute(self._h, max_depth, None, 0))
+        buf = (C.c_int32 * (max(cnt, 1) * self.n))()
+        _check(lib().acc_enumerate_recompute(self._h, max_depth, buf, cnt))
+        return [list(buf[i * self.n:(i + 1) * self.n]) for i in range(cnt)]
+
+    def partition_cost_recompute(self, pi, max_depth, cost="bytes"):
+        out = C.c_double()
+        _check(lib().acc_partition_cost_recompute(self._h, _i32_array(pi), len(pi), max_depth, COST[cost], C.byref(out)))
+        return out.value
 
     def get_partition(self):
         out = (C.c_int32 * self.n)()

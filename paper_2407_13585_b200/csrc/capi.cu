@@ -90,26 +90,32 @@ int acc_edges(const acc_graph* g, int32_t* F, int32_t* nF, int32_t* I, int32_t* 
   return ACC_OK;
 }
 
-int acc_check_partition(acc_graph* g, const int32_t* pi, int32_t n_nodes) {
+int acc_check_partition_recompute(acc_graph* g, const int32_t* pi, int32_t n_nodes, int32_t max_depth) {
   clear_error();
   if (!g || !pi) return set_error(ACC_ERR_ARG, "null argument");
+  if (max_depth < 0) return set_error(ACC_ERR_ARG, "max_depth %d is negative", max_depth);
   if (n_nodes != (int32_t)g->nodes.size()) return set_error(ACC_ERR_ARG, "clustering has %d entries, graph has %zu nodes", n_nodes, g->nodes.size());
   for (int i = 0; i < n_nodes; ++i)
     if (!is_input(g->nodes[i]) && (pi[i] < 0 || pi[i] > n_nodes)) return set_error(ACC_ERR_ARG, "cluster number %d of node %d outside 0..n", pi[i], i);
-  return check_partition(*g, pi, nullptr);
+  return check_partition(*g, pi, nullptr, false, max_depth);
 }
 
-int acc_set_partition(acc_graph* g, const int32_t* pi, int32_t n_nodes) {
-  const int rc = acc_check_partition(g, pi, n_nodes);
+int acc_check_partition(acc_graph* g, const int32_t* pi, int32_t n_nodes) { return acc_check_partition_recompute(g, pi, n_nodes, 0); }
+
+int acc_set_partition_recompute(acc_graph* g, const int32_t* pi, int32_t n_nodes, int32_t max_depth) {
+  const int rc = acc_check_partition_recompute(g, pi, n_nodes, max_depth);
   if (rc != ACC_OK) return rc;
   g->pi.assign(pi, pi + n_nodes);
   for (int i = 0; i < n_nodes; ++i)
     if (is_input(g->nodes[i])) g->pi[i] = -1;
   manifest_of(*g, g->pi.data(), g->manifest);
   g->has_pi = true;
+  g->recompute_depth = max_depth;
   g->run_serial++;
   return ACC_OK;
 }
+
+int acc_set_partition(acc_graph* g, const int32_t* pi, int32_t n_nodes) { return acc_set_partition_recompute(g, pi, n_nodes, 0); }
 
 int acc_get_partition(const acc_graph* g, int32_t* out, int32_t n_nodes) {
   clear_error();
@@ -127,21 +133,27 @@ int acc_manifest(const acc_graph* g, int32_t* out, int32_t n_nodes) {
   return ACC_OK;
 }
 
-int acc_plan(acc_graph* g, int mode, int cost, int32_t* out) {
+int acc_plan_recompute(acc_graph* g, int mode, int cost, int32_t max_depth, int32_t* out) {
   clear_error();
   if (!g) return set_error(ACC_ERR_ARG, "graph is null");
+  if (max_depth < 0) return set_error(ACC_ERR_ARG, "max_depth %d is negative", max_depth);
   std::vector<int32_t> pi;
-  const int rc = plan(*g, mode, cost, pi);
+  const int rc = plan(*g, mode, cost, pi, max_depth);
   if (rc != ACC_OK) return rc;
   if (out) memcpy(out, pi.data(), sizeof(int32_t) * pi.size());
-  return acc_set_partition(g, pi.data(), (int32_t)pi.size());
+  return acc_set_partition_recompute(g, pi.data(), (int32_t)pi.size(), max_depth);
 }
 
-int64_t acc_enumerate(acc_graph* g, int32_t* out_pi, int64_t max_partitions) {
+int acc_plan(acc_graph* g, int mode, int cost, int32_t* out) { return acc_plan_recompute(g, mode, cost, 0, out); }
+
+int64_t acc_enumerate(acc_graph* g, int32_t* out_pi, int64_t max_partitions) { return acc_enumerate_recompute(g, 0, out_pi, max_partitions); }
+
+int64_t acc_enumerate_recompute(acc_graph* g, int32_t max_depth, int32_t* out_pi, int64_t max_partitions) {
   clear_error();
   if (!g) return set_error(ACC_ERR_ARG, "graph is null");
+  if (max_depth < 0) return set_error(ACC_ERR_ARG, "max_depth %d is negative", max_depth);
   std::vector<std::vector<int32_t>> all;
-  const int64_t cnt = enumerate_all(*g, all);
+  const int64_t cnt = enumerate_all(*g, all, max_depth);
   if (cnt < 0) return cnt;
   const size_t n = g->nodes.size();
   if (out_pi)
@@ -149,10 +161,14 @@ int64_t acc_enumerate(acc_graph* g, int32_t* out_pi, int64_t max_partitions) {
   return cnt;
 }
 
-int acc_partition_cost(acc_graph* g, const int32_t* pi, int32_t n_nodes, int cost, double* out) {
+int acc_partition_cost_recompute(acc_graph* g, const int32_t* pi, int32_t n_nodes, int32_t max_depth, int cost, double* out) {
   clear_error();
-  if (!g || !pi || !out || n_nodes != (int32_t)g->nodes.size()) return set_error(ACC_ERR_ARG, "bad argument");
-  return partition_cost(*g, pi, cost, out);
+  if (!g || !pi || !out || max_depth < 0 || n_nodes != (int32_t)g->nodes.size()) return set_error(ACC_ERR_ARG, "bad argument");
+  return partition_cost(*g, pi, cost, out, max_depth);
+}
+
+int acc_partition_cost(acc_graph* g, const int32_t* pi, int32_t n_nodes, int cost, double* out) {
+  return acc_partition_cost_recompute(g, pi, n_nodes, 0, cost, out);
 }
 
 int acc_bind(acc_graph* g, acc_node n, void* device_ptr, size_t bytes) {

@@ -19,7 +19,7 @@
 namespace acc {
 
 constexpr int kMaxSlots = ACC_MAX_INPUTS;
-constexpr int kMaxCluster = 24;   // local nodes per cluster
+constexpr int kMaxCluster = 40;   // local nodes per cluster
 constexpr int kMaxProgram = 40;   // nodes per build-time program
 
 struct PNode {                    // node of a build-time program

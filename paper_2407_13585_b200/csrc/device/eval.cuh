@@ -264,6 +264,12 @@ __device__ __forceinline__ val_of<IX> ld_ext(const A& a, const IX& ix) {
   return ld(reinterpret_cast<const uint32_t*>(a.n[I].ptr), a.n[I].C, ix);
 }
 
+// Skeletons that keep a MEMBER's values on chip (computed once over a tile, then read at
+// several indices) say so per index kind, and supply the read.
+template <class CL, int I, class IX> struct reads_staged { static constexpr bool value = false; };
+template <class CL, int I, class A, class IX>
+__device__ __forceinline__ val_of<IX> ld_staged(const A& a, const IX& ix);
+
 template <class CL, int I, class A>
 __device__ __forceinline__ uint32_t free_of(const A& a) {
   constexpr CNode nd = CL::c.nodes[I];
@@ -289,7 +295,18 @@ __device__ __forceinline__ uint32_t eval_member1(const A& a, const Ix& ix) {
 }
 
 template <class CL, int I, class A, class IX>
+__device__ __forceinline__ val_of<IX> eval_here(const A& a, const IX& ix);
+
+template <class CL, int I, class A, class IX>
 __device__ __forceinline__ val_of<IX> eval(const A& a, const IX& ix) {
+  if constexpr (reads_staged<CL, I, IX>::value) return ld_staged<CL, I>(a, ix);
+  else return eval_here<CL, I>(a, ix);
+}
+
+// The value of node I at an index, computed here (even where a skeleton keeps it on chip:
+// this is what fills that copy).
+template <class CL, int I, class A, class IX>
+__device__ __forceinline__ val_of<IX> eval_here(const A& a, const IX& ix) {
   constexpr CNode nd = CL::c.nodes[I];
   constexpr int W = width_of<IX>::value;
   if constexpr (!nd.member) {

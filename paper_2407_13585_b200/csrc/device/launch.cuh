@@ -135,6 +135,7 @@ struct Launcher {
   static int launch_stencil(const ClusterLaunch& L, dev::Args<N>& a, int R, int C, bool vec) {
     if constexpr (kStencilShape) {
       if (!vec || R < 1 || (int64_t)R * C < (int64_t)dev::kStRows * dev::kStCols * 64) return 1;
+      constexpr int depth = dev::max_shift_depth<CL>();
       dev::StencilMaps maps;
       for (int i = 0; i < N; ++i) {
         const CNode& n = CL::c.nodes[i];
@@ -143,15 +144,17 @@ struct Launcher {
           return 1;
         if (dev::is_staged_external<CL>(i)) {
           if (L.nodes[i].R != R || L.nodes[i].C != C) return 1;
-          if (!make_tensor_map_2d(&maps.m[dev::tile_slot<CL>(i)], L.nodes[i].ptr, R, C, dev::kStBoxRows, dev::kStBoxCols)) return 1;
+          if (!make_tensor_map_2d(&maps.m[dev::tile_slot<CL>(i)], L.nodes[i].ptr, R, C, dev::st_box_rows(depth), dev::kStBoxCols)) return 1;
         }
       }
       auto kern = dev::k_stencil<CL>;
-      const size_t smem = (size_t)dev::kStStages * dev::staged_externals<CL>() * dev::kStBoxStride * 4;
+      // two stages of every external's box, one box per member kept on chip
+      const size_t smem = (size_t)(dev::kStStages * dev::staged_externals<CL>() + dev::staged_members<CL>()) * dev::st_box_stride(depth) * 4;
       if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return set_error(ACC_ERR_CUDA, "shared-memory opt-in failed: %s", cudaGetErrorString(cudaGetLastError()));
       const int64_t tiles = (int64_t)((C + dev::kStCols - 1) / dev::kStCols) * ((R + dev::kStRows - 1) / dev::kStRows);
-      const int grid = (int)std::min<int64_t>(tiles, (int64_t)sm_count() * 3);
+      const int per_sm = std::max(1, std::min(3, (int)((size_t)220 * 1024 / (smem + 1024))));
+      const int grid = (int)std::min<int64_t>(tiles, (int64_t)sm_count() * per_sm);
       kern<<<grid, dev::kBlock, smem, L.stream>>>(a, maps);
       const cudaError_t e = cudaGetLastError();
       if (e != cudaSuccess) return set_error(ACC_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));

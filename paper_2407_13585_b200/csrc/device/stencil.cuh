@@ -1,15 +1,25 @@
 // k_stencil: the skeleton for rank-2 clusters whose only index maps are clamped shifts by at
 // most one row and one column (a stencil by horizontal fusion: several backpermutes of one
-// array feeding zipWiths).
+// array feeding zipWiths), stacked up to kStMaxDepth deep (several iterations of such a stencil
+// in one cluster, which needs the recomputing kind of clustering: the intermediate iterate is
+// read in five orders).
 //
-// A persistent CTA walks output tiles of kStRows x kStCols.  For each tile the tile plus its
-// halo (one row above and below, four columns left and right so that the copy starts on a
-// 16-byte boundary) of every external is brought into shared memory by ONE tensor copy
-// (cp.async.bulk.tensor, no multicast), issued by one thread and tracked by an mbarrier; the
-// copy of the next tile runs while the current one is computed (two stages).  Parts of the
-// box outside the array arrive as zeros and are never read: shifted positions are clamped to
-// the array first, and a clamped position always lies inside the tile or its halo.  All five
-// reads of a Jacobi iteration are then shared-memory reads.
+// A persistent CTA walks output tiles of kStRows x kStCols.  With D = the largest number of
+// shifts between an external and a root, the tile plus a halo of D rows above and below and
+// four columns left and right (so that the copy starts on a 16-byte boundary; D <= 4) of every
+// external is brought into shared memory by ONE tensor copy (cp.async.bulk.tensor, no
+// multicast), issued by one thread and tracked by an mbarrier; the copy of the next tile runs
+// while the current one is computed (two stages).  Parts of the box outside the array arrive
+// as zeros and are never read: shifted positions are clamped to the array first, and a clamped
+// position always lies inside the tile or its halo.
+//
+// A member that is itself the source of a shift (the previous iterate of a stacked stencil) is
+// computed ONCE per tile, over the tile plus the halo its readers still need, into a box of the
+// same geometry in shared memory, depth by depth; its readers then read that box.  So k
+// iterations cost one read and one write of the array and (1 + 2(D-k)/kStRows) of the
+// arithmetic per level instead of the 5^k-fold recomputation that pulling each read through
+// would do.  The values are those of the plain evaluation, bit for bit: every element is
+// computed by the same expression, at positions clamped in the same way.
 //
 // Every wait on an mbarrier is bounded: after kCopySpinLimit polls the thread records
 // ACC_ERR_DEVICE_TIMEOUT in the status word and goes on, so a lost copy cannot hang the GPU.
@@ -23,20 +33,26 @@ namespace acc {
 namespace dev {
 
 constexpr int kStRows = 64, kStCols = 128;            // output tile
-constexpr int kStBoxRows = kStRows + 2;               // + halo rows
 constexpr int kStBoxCols = kStCols + 8;               // + halo columns (4 each side: 16-byte alignment)
-constexpr int kStBoxWords = kStBoxRows * kStBoxCols;  // 4624 words = 18496 bytes per copy
-constexpr int kStBoxStride = (kStBoxWords + 31) / 32 * 32;   // boxes start on 128-byte boundaries
+constexpr int kStChunks = kStBoxCols / 4;             // 128-bit chunks per box row
 constexpr int kStStages = 2;
 constexpr int kStMaxExternals = 2;
+constexpr int kStMaxDepth = 4;                        // the column halo is four wide
+constexpr int kStMaxStagedMembers = 3;
+
+constexpr int st_box_rows(int depth) { return kStRows + 2 * depth; }
+constexpr int st_box_words(int depth) { return st_box_rows(depth) * kStBoxCols; }
+constexpr int st_box_stride(int depth) { return (st_box_words(depth) + 31) / 32 * 32; }   // boxes start on 128-byte boundaries
 
 struct StencilMaps { CUtensorMap m[kStMaxExternals]; };
 
-// four consecutive columns inside the staged tile / the same after one clamped shift.
-// `at` points to element (r, c) in the box of external slot 0 of the current stage; the boxes
-// of the other slots lie kStBoxStride words further each.
-struct IxH4  { int r, c; const uint32_t* at; };
-struct IxHS4 { int r, c, dc; const uint32_t* at; };    // row r (already clamped), columns clamp(c+dc+j)
+// Where the boxes of the current tile are: externals of this stage, members kept on chip.
+struct StCtx { const uint32_t* ext; const uint32_t* mem; };
+
+// four consecutive columns inside a box / the same after one clamped shift.  `off` is the word
+// offset of element (r, c) in a box; the box of slot k lies k box strides further.
+struct IxH4  { int r, c, off; StCtx t; };
+struct IxHS4 { int r, c, dc, off; StCtx t; };   // row r (already clamped), columns clamp(c+dc+j)
 
 __device__ __forceinline__ Ix lane(const IxH4& i, int j) { return Ix{i.r, i.c + j}; }
 
@@ -45,17 +61,16 @@ template <int F> __device__ __forceinline__ auto map_index(const IxH4& i, const 
   if constexpr (F == ACC_IDX_IDENTITY) return i;
   else {
     const int rr = min(max(i.r + self.ip0, 0), src.R - 1);
-    return IxHS4{rr, i.c, self.ip1, i.at + (rr - i.r) * kStBoxCols};
+    return IxHS4{rr, i.c, self.ip1, i.off + (rr - i.r) * kStBoxCols, i.t};
   }
 }
 template <int F> __device__ __forceinline__ auto map_index(const IxHS4& i, const NodeArg&, const NodeArg&) {
-  static_assert(F == ACC_IDX_IDENTITY, "a halo of one serves one shift, not a shift of a shift");
+  static_assert(F == ACC_IDX_IDENTITY, "the source of a shift is read from a box, never pulled through");
   return i;
 }
 
-// A cluster can use this skeleton if its members are element-wise, its only index maps are
-// shifts, no external is reached through more than one shift, every array it reads is a
-// rank-2 external, and its roots are rank-2 stores.
+// ---- compile-time layout of a stencil cluster -----------------------------------------------
+// shifts between the externals and node i (longest path)
 template <class CL> constexpr int shift_depth(int i) {
   const CNode& n = CL::c.nodes[i];
   if (!n.member) return 0;
@@ -66,6 +81,33 @@ template <class CL> constexpr int shift_depth(int i) {
   }
   return d + ((n.kind == ACC_BACKPERMUTE && n.idxfn == ACC_IDX_SHIFT_CLAMP) ? 1 : 0);
 }
+template <class CL> constexpr int max_shift_depth() {
+  int d = 0;
+  for (int i = 0; i < CL::c.n; ++i) {
+    const int k = shift_depth<CL>(i);
+    d = k > d ? k : d;
+  }
+  return d;
+}
+// a member that some shift reads: kept on chip
+template <class CL> constexpr bool is_staged_member(int i) {
+  if (!CL::c.nodes[i].member) return false;
+  for (int j = 0; j < CL::c.n; ++j) {
+    const CNode& n = CL::c.nodes[j];
+    if (n.member && n.kind == ACC_BACKPERMUTE && n.idxfn == ACC_IDX_SHIFT_CLAMP && n.in[0] == i) return true;
+  }
+  return false;
+}
+template <class CL> constexpr int member_slot(int i) {
+  int k = 0;
+  for (int j = 0; j < i; ++j) k += is_staged_member<CL>(j) ? 1 : 0;
+  return k;
+}
+template <class CL> constexpr int staged_members() { return member_slot<CL>(CL::c.n); }
+
+// A cluster can use this skeleton if its members are element-wise, its only index maps are
+// shifts stacked at most kStMaxDepth deep, every array it reads is a rank-2 external, and its
+// roots are rank-2 stores.
 template <class CL> constexpr bool stencil_eligible() {
   bool has_shift = false;
   int externals = 0;
@@ -89,19 +131,19 @@ template <class CL> constexpr bool stencil_eligible() {
     } else if (n.kind != ACC_MAP && n.kind != ACC_ZIPWITH) {
       return false;
     }
-    if (shift_depth<CL>(i) > 1) return false;
   }
-  return has_shift && externals >= 1 && externals <= kStMaxExternals;
+  return has_shift && externals >= 1 && externals <= kStMaxExternals && max_shift_depth<CL>() <= kStMaxDepth &&
+         staged_members<CL>() <= kStMaxStagedMembers;
 }
 
-// reads from the staged boxes (a tile's box starts at row r0-1, column c0-4, so the element
-// left of a chunk and the one right of it are always inside the box)
-__device__ __forceinline__ V4 ld_box(int slot, const IxH4& i) {
-  const uint4 v = *reinterpret_cast<const uint4*>(i.at + slot * kStBoxStride);
+// ---- reads from the boxes ----------------------------------------------------------------------
+// (a tile's box starts D rows above and four columns left of the tile, so the element left of a
+// chunk and the one right of it are always words of the box)
+__device__ __forceinline__ V4 ld_box(const uint32_t* p) {
+  const uint4 v = *reinterpret_cast<const uint4*>(p);
   return V4{{v.x, v.y, v.z, v.w}};
 }
-__device__ __forceinline__ V4 ld_box(int slot, const IxHS4& i, int C) {
-  const uint32_t* p = i.at + slot * kStBoxStride;
+__device__ __forceinline__ V4 ld_box(const uint32_t* p, const IxHS4& i, int C) {
   const uint4 v = *reinterpret_cast<const uint4*>(p);
   if (i.dc == 1) return V4{{v.y, v.z, v.w, p[min(4, C - 1 - i.c)]}};      // clamped at the last column
   if (i.dc == -1) return V4{{p[max(-1, -i.c)], v.x, v.y, v.z}};           // clamped at the first column
@@ -109,25 +151,38 @@ __device__ __forceinline__ V4 ld_box(int slot, const IxHS4& i, int C) {
 }
 
 template <class CL, int I, class A>
-__device__ __forceinline__ V4 ld_ext(const A&, const IxH4& ix) { return ld_box(tile_slot<CL>(I), ix); }
+__device__ __forceinline__ V4 ld_ext(const A&, const IxH4& ix) {
+  return ld_box(ix.t.ext + tile_slot<CL>(I) * st_box_stride(max_shift_depth<CL>()) + ix.off);
+}
 template <class CL, int I, class A>
-__device__ __forceinline__ V4 ld_ext(const A& a, const IxHS4& ix) { return ld_box(tile_slot<CL>(I), ix, a.n[I].C); }
+__device__ __forceinline__ V4 ld_ext(const A& a, const IxHS4& ix) {
+  return ld_box(ix.t.ext + tile_slot<CL>(I) * st_box_stride(max_shift_depth<CL>()) + ix.off, ix, a.n[I].C);
+}
+
+// members kept on chip are read from their box at a shifted index, computed anywhere else
+template <class CL, int I> struct reads_staged<CL, I, IxHS4> { static constexpr bool value = is_staged_member<CL>(I); };
+template <class CL, int I, class A>
+__device__ __forceinline__ V4 ld_staged(const A& a, const IxHS4& ix) {
+  return ld_box(ix.t.mem + member_slot<CL>(I) * st_box_stride(max_shift_depth<CL>()) + ix.off, ix, a.n[I].C);
+}
 
 template <class CL>
 __global__ void __launch_bounds__(kBlock)
 k_stencil(const __grid_constant__ Args<CL::c.n> a, const __grid_constant__ StencilMaps maps) {
   constexpr int N = CL::c.n;
   constexpr int E = staged_externals<CL>();
-  extern __shared__ __align__(128) uint32_t boxes[];          // [stage][external slot][kStBoxStride]
+  constexpr int D = max_shift_depth<CL>();
+  constexpr int BR = st_box_rows(D), BS = st_box_stride(D);
+  extern __shared__ __align__(128) uint32_t boxes[];          // [stage][external slot][BS], then [member slot][BS]
   __shared__ __align__(8) uint64_t bar[kStStages];
+  uint32_t* const members = boxes + kStStages * E * BS;
   const int R = a.R, C = a.C;
   const uint32_t tiles_x = (uint32_t)(C + kStCols - 1) / kStCols;
   const uint32_t n_tiles = tiles_x * ((uint32_t)(R + kStRows - 1) / kStRows);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStStages; ++s)
-      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bar[s])) : "memory");
+    for (int s = 0; s < kStStages; ++s) mbar_init(&bar[s], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -135,12 +190,12 @@ k_stencil(const __grid_constant__ Args<CL::c.n> a, const __grid_constant__ Stenc
   // one thread starts the copies of a tile into a stage; the stage's barrier counts their bytes
   auto issue = [&](uint32_t tile, int stage) {
     const uint32_t ty = tile / tiles_x, tx = tile - ty * tiles_x;
-    const int x = (int)(tx * kStCols) - 4, y = (int)(ty * kStRows) - 1;   // x stays a multiple of 4: 16-byte aligned
+    const int x = (int)(tx * kStCols) - 4, y = (int)(ty * kStRows) - D;   // x stays a multiple of 4: 16-byte aligned
     const uint32_t b = smem_addr(&bar[stage]);
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"((uint32_t)(E * kStBoxWords * 4)) : "memory");
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"((uint32_t)(E * st_box_words(D) * 4)) : "memory");
 #pragma unroll
     for (int slot = 0; slot < E; ++slot) {
-      const uint32_t dst = smem_addr(boxes + (stage * E + slot) * kStBoxStride);
+      const uint32_t dst = smem_addr(boxes + (stage * E + slot) * BS);
       asm volatile(
           "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
           ::"r"(dst), "l"(&maps.m[slot]), "r"(x), "r"(y), "r"(b) : "memory");
@@ -157,13 +212,39 @@ k_stencil(const __grid_constant__ Args<CL::c.n> a, const __grid_constant__ Stenc
     if (!arrived) atomicOr(a.status, kStatusTimeout);
 
     const uint32_t ty = tile / tiles_x, tx = tile - ty * tiles_x;
-    const uint32_t* box = boxes + stage * E * kStBoxStride;
     const int r0 = (int)(ty * kStRows), c0 = (int)(tx * kStCols);
+    StCtx ctx;
+    ctx.ext = boxes + stage * E * BS;
+    ctx.mem = members;
+
+    // members kept on chip, shallowest first: a member k shifts away from the externals is needed
+    // (and computable) on the box rows k .. BR-1-k; whole box rows are computed, of which the
+    // readers use the columns k away from the box edges at most
+    static_for<1, D>([&](auto kc) {
+      constexpr int k = decltype(kc)::value;
+      static_for<0, N>([&](auto ic) {
+        constexpr int i = decltype(ic)::value;
+        if constexpr (is_staged_member<CL>(i) && shift_depth<CL>(i) == k) {
+          uint32_t* out = members + member_slot<CL>(i) * BS;
+          for (int q = threadIdx.x; q < (BR - 2 * k) * kStChunks; q += kBlock) {
+            const int br = k + q / kStChunks, bc = 4 * (q % kStChunks);
+            const int r = r0 - D + br, c = c0 - 4 + bc;
+            if (r >= 0 && r < R && c >= 0 && c < C) {
+              const int off = br * kStBoxCols + bc;
+              const V4 v = eval_here<CL, i>(a, IxH4{r, c, off, ctx});
+              *reinterpret_cast<uint4*>(out + off) = make_uint4(v.v[0], v.v[1], v.v[2], v.v[3]);
+            }
+          }
+          __syncthreads();
+        }
+      });
+    });
+
 #pragma unroll
     for (int p = 0; p < kStRows / (kBlock / 32); ++p) {
       const int r = r0 + warp + (kBlock / 32) * p, c = c0 + 4 * lane;
       if (r < R && c < C) {
-        const IxH4 ix{r, c, box + (r - r0 + 1) * kStBoxCols + (c - c0 + 4)};
+        const IxH4 ix{r, c, (r - r0 + D) * kStBoxCols + (c - c0 + 4), ctx};
         static_for<0, N>([&](auto ic) {
           constexpr int i = decltype(ic)::value;
           if constexpr (is_store_root(CL::c.nodes[i]))

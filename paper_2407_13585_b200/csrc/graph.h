@@ -32,6 +32,7 @@ struct Graph {
   std::vector<Edge> edges;
   std::vector<int32_t> pi;         // stored clustering, -1 for inputs
   bool has_pi = false;
+  int recompute_depth = 0;         // the rules the stored clustering was checked under
   std::vector<uint8_t> manifest;   // under the stored clustering
   // bookkeeping of the last run
   int32_t launches = 0;
@@ -55,13 +56,15 @@ struct Solution {
   std::vector<uint8_t> manifest;   // per node
   std::vector<int32_t> order;      // d^o per node (for PERMUTE: order of its idx/vals slots), -1 for inputs
 };
-int  check_partition(const Graph& g, const int32_t* pi, Solution* sol, bool quiet = false);
+// recompute_depth 0: the paper's rules; k > 0: producers may be evaluated once per order they are
+// read in, with at most k gather-like members stacked on a fused path
+int  check_partition(const Graph& g, const int32_t* pi, Solution* sol, bool quiet = false, int recompute_depth = 0);
 void manifest_of(const Graph& g, const int32_t* pi, std::vector<uint8_t>& man);
 
 // planner.cpp
-int     plan(Graph& g, int mode, int cost, std::vector<int32_t>& out);
-int64_t enumerate_all(const Graph& g, std::vector<std::vector<int32_t>>& out);
-int     partition_cost(const Graph& g, const int32_t* pi, int cost, double* out);
+int     plan(Graph& g, int mode, int cost, std::vector<int32_t>& out, int recompute_depth = 0);
+int64_t enumerate_all(const Graph& g, std::vector<std::vector<int32_t>>& out, int recompute_depth = 0);
+int     partition_cost(const Graph& g, const int32_t* pi, int cost, double* out, int recompute_depth = 0);
 bool    canonical_numbering(const Graph& g, const std::vector<int>& block_of, int n_blocks, std::vector<int32_t>& pi);
 
 }  // namespace acc

@@ -8,6 +8,14 @@
 // order in {0,1}.  Order classes that stay free are 0 or 1; which one matters only for
 // whether two reads of a common outside parent are shared, i.e. for connectivity, and is
 // settled by a small exhaustive search.
+//
+// Recomputing clusterings (an extension; the paper leaves work duplication to future work in
+// its Section 6).  With `recompute_depth` > 0 an array that is fused away may be evaluated
+// once per order it is asked for, as if every consumer had a private copy of its producer (and
+// of that producer's producers inside the cluster).  The order equalities then only run from a
+// consumer to its own copies, so they can only fail at a scan (whose order is fixed) or at the
+// one stored copy of a manifest array (order 0 or 1).  At most `recompute_depth` gather-like
+// members may be stacked on a fused path.
 #include <algorithm>
 #include <map>
 
@@ -127,11 +135,101 @@ struct ClusterCheck {
     }
     return ACC_ERR_DISCONNECTED;
   }
+
+  // The recomputing variant.  Orders are symbols: a constant (0, 1, a label) or the variable of
+  // a stored copy / a scatter / a member nobody in the cluster reads (encoded -1 - local id),
+  // which is 0 or 1.  Members are visited consumers first; each passes the orders it is asked
+  // for on to its producers, slot by slot.
+  int run_recompute(std::vector<int32_t>* order_out, int max_depth) {
+    const int m = (int)members.size();
+    std::vector<std::vector<int>> asked(m);
+    std::vector<int> bound(m, kFree);                    // value of variable i once a scan fixed it
+    std::vector<uint8_t> read_inside(m, 0);
+    std::vector<int> depth(m, 0);
+    for (const Edge& e : g.edges)
+      if (local[e.a] >= 0 && local[e.b] >= 0) read_inside[local[e.a]] = 1;
+    auto resolve = [&](int o) { return o < 0 && bound[-1 - o] != kFree ? bound[-1 - o] : o; };
+    auto ask = [&](int i, int o) {
+      if (std::find(asked[i].begin(), asked[i].end(), o) == asked[i].end()) asked[i].push_back(o);
+    };
+    for (int i = m - 1; i >= 0; --i) {
+      const int a = members[i];
+      const int k = g.nodes[a].d.kind;
+      if (man[a] || k == ACC_PERMUTE || !read_inside[i]) ask(i, -1 - i);
+      if (k == ACC_SCANL || k == ACC_SCANR) {
+        const int fixed = k == ACC_SCANL ? 0 : 1;
+        for (int o : asked[i]) {
+          const int r = resolve(o);
+          if (r >= 0 && r != fixed) return ACC_ERR_ILLEGAL_TRAVERSAL;
+          if (r < 0) bound[-1 - r] = fixed;
+        }
+        asked[i].assign(1, fixed);
+      }
+      for (const Edge& e : g.edges) {
+        if (e.b != a || local[e.a] < 0) continue;
+        const int c = slot_const(a, e.slot);
+        for (int o : asked[i]) ask(local[e.a], c != kFree ? c : o);
+      }
+    }
+    // depth of stacking, producers first
+    int deepest = 0;
+    for (int i = 0; i < m; ++i) {
+      const int a = members[i];
+      int d = 0;
+      for (const Edge& e : g.edges)
+        if (e.b == a && local[e.a] >= 0) d = std::max(d, depth[local[e.a]]);
+      depth[i] = d + (gather_like(g.nodes[a]) ? 1 : 0);
+      deepest = std::max(deepest, depth[i]);
+    }
+    if (deepest > max_depth) return ACC_ERR_ILLEGAL_TRAVERSAL;
+    // connectivity: fused edges, or reads of one outside parent in one order
+    Dsu base(m);
+    for (const Edge& e : g.edges)
+      if (local[e.a] >= 0 && local[e.b] >= 0) base.unite(local[e.a], local[e.b]);
+    struct Read { int parent, order, node; };
+    std::vector<Read> reads;
+    for (const Edge& e : g.edges) {
+      if (local[e.b] < 0 || local[e.a] >= 0 || !e.ordered) continue;
+      if (slot_const(e.b, e.slot) != kFree) continue;
+      for (int o : asked[local[e.b]]) reads.push_back({e.a, resolve(o), local[e.b]});
+    }
+    std::vector<int> free_var;
+    for (const Read& r : reads)
+      if (r.order < 0 && std::find(free_var.begin(), free_var.end(), r.order) == free_var.end()) free_var.push_back(r.order);
+    const int k = (int)free_var.size();
+    const uint32_t combos = k > 16 ? 1u : (1u << k);
+    for (uint32_t bits = 0; bits < combos; ++bits) {
+      auto value_of = [&](int o) {
+        if (o >= 0) return o;
+        for (int j = 0; j < k; ++j)
+          if (free_var[j] == o) return k > 16 ? 0 : int((bits >> j) & 1u);
+        return 0;
+      };
+      Dsu conn = base;
+      std::map<std::pair<int, int>, int> first;
+      for (const Read& r : reads) {
+        auto key = std::make_pair(r.parent, value_of(r.order));
+        auto it = first.find(key);
+        if (it == first.end()) first[key] = r.node; else conn.unite(it->second, r.node);
+      }
+      bool one = true;
+      for (int i = 1; i < m && one; ++i) one = conn.find(i) == conn.find(0);
+      if (one) {
+        if (order_out)
+          for (int i = 0; i < m; ++i) {
+            const int o = asked[i].empty() ? 0 : value_of(resolve(asked[i].front()));
+            (*order_out)[members[i]] = o;
+          }
+        return ACC_OK;
+      }
+    }
+    return ACC_ERR_DISCONNECTED;
+  }
 };
 
 }  // namespace
 
-int check_partition(const Graph& g, const int32_t* pi, Solution* sol, bool quiet) {
+int check_partition(const Graph& g, const int32_t* pi, Solution* sol, bool quiet, int recompute_depth) {
   const int n = (int)g.nodes.size();
   auto fail = [&](int code, const char* what, int a, int b) {
     return quiet ? code : set_error(code, "illegal clustering: %s (nodes %d, %d)", what, a, b);
@@ -160,7 +258,7 @@ int check_partition(const Graph& g, const int32_t* pi, Solution* sol, bool quiet
   std::vector<int32_t> order(n, -1);
   for (auto& kv : clusters) {
     ClusterCheck cc(g, kv.second, man, label);
-    const int rc = cc.run(&order);
+    const int rc = recompute_depth > 0 ? cc.run_recompute(&order, recompute_depth) : cc.run(&order);
     if (rc != ACC_OK)
       return fail(rc, rc == ACC_ERR_DISCONNECTED ? "a cluster does not hang together through a fused array"
                                                  : "traversal orders cannot be matched",

@@ -50,9 +50,9 @@ bool canonical_numbering(const Graph& g, const std::vector<int>& block_of, int n
   return true;
 }
 
-int partition_cost(const Graph& g, const int32_t* pi, int cost, double* out) {
+int partition_cost(const Graph& g, const int32_t* pi, int cost, double* out, int recompute_depth) {
   Solution sol;
-  const int rc = check_partition(g, pi, &sol);
+  const int rc = check_partition(g, pi, &sol, false, recompute_depth);
   if (rc != ACC_OK) return rc;
   const int n = (int)g.nodes.size();
   auto bytes = [&](int a) { return double(std::max<int64_t>(g.nodes[a].count, 1)) * 4.0; };
@@ -96,7 +96,7 @@ int partition_cost(const Graph& g, const int32_t* pi, int cost, double* out) {
   return ACC_OK;
 }
 
-int64_t enumerate_all(const Graph& g, std::vector<std::vector<int32_t>>& out) {
+int64_t enumerate_all(const Graph& g, std::vector<std::vector<int32_t>>& out, int recompute_depth) {
   const int n = (int)g.nodes.size();
   std::vector<int> items;
   for (int i = 0; i < n; ++i)
@@ -110,7 +110,7 @@ int64_t enumerate_all(const Graph& g, std::vector<std::vector<int32_t>>& out) {
   std::vector<int32_t> pi;
   std::function<void(size_t, int)> grow = [&](size_t at, int n_blocks) {
     if (at == items.size()) {
-      if (canonical_numbering(g, block_of, n_blocks, pi) && check_partition(g, pi.data(), nullptr, true) == ACC_OK) out.push_back(pi);
+      if (canonical_numbering(g, block_of, n_blocks, pi) && check_partition(g, pi.data(), nullptr, true, recompute_depth) == ACC_OK) out.push_back(pi);
       return;
     }
     const int node = items[at];
@@ -133,7 +133,7 @@ namespace {
 
 // Greedy over fusible edges.  Fusing (a, b) merges their blocks and pulls in every node
 // lying on a path between the two blocks (otherwise no execution order exists).
-int greedy(const Graph& g, bool top_down, std::vector<int32_t>& out) {
+int greedy(const Graph& g, bool top_down, std::vector<int32_t>& out, int recompute_depth) {
   const int n = (int)g.nodes.size();
   std::vector<std::vector<uint8_t>> reach(n, std::vector<uint8_t>(n, 0));   // reach[a][b]: path a -> b
   for (int b = 0; b < n; ++b)
@@ -190,7 +190,7 @@ int greedy(const Graph& g, bool top_down, std::vector<int32_t>& out) {
       }
     }
     const int nb = densify(trial, dense);
-    if (canonical_numbering(g, dense, nb, pi) && check_partition(g, pi.data(), nullptr, true) == ACC_OK) block = trial;
+    if (canonical_numbering(g, dense, nb, pi) && check_partition(g, pi.data(), nullptr, true, recompute_depth) == ACC_OK) block = trial;
   }
   const int nb = densify(block, dense);
   if (!canonical_numbering(g, dense, nb, out)) return set_error(ACC_ERR_ARG, "greedy planner lost its execution order");
@@ -199,7 +199,7 @@ int greedy(const Graph& g, bool top_down, std::vector<int32_t>& out) {
 
 }  // namespace
 
-int plan(Graph& g, int mode, int cost, std::vector<int32_t>& out) {
+int plan(Graph& g, int mode, int cost, std::vector<int32_t>& out, int recompute_depth) {
   const int n = (int)g.nodes.size();
   switch (mode) {
     case ACC_PLAN_UNFUSED: {
@@ -211,22 +211,22 @@ int plan(Graph& g, int mode, int cost, std::vector<int32_t>& out) {
     }
     case ACC_PLAN_ENUMERATE: {
       std::vector<std::vector<int32_t>> all;
-      const int64_t cnt = enumerate_all(g, all);
+      const int64_t cnt = enumerate_all(g, all, recompute_depth);
       if (cnt < 0) return (int)cnt;
       if (cnt == 0) return set_error(ACC_ERR_ARG, "no legal clustering");
       double best = 0;
       int best_i = -1;
       for (int i = 0; i < (int)all.size(); ++i) {
         double c = 0;
-        const int rc = partition_cost(g, all[i].data(), cost, &c);
+        const int rc = partition_cost(g, all[i].data(), cost, &c, recompute_depth);
         if (rc != ACC_OK) return rc;
         if (best_i < 0 || c < best) { best = c; best_i = i; }
       }
       out = all[best_i];
       return ACC_OK;
     }
-    case ACC_PLAN_GREEDY_TOPDOWN: return greedy(g, true, out);
-    case ACC_PLAN_GREEDY_BOTTOMUP: return greedy(g, false, out);
+    case ACC_PLAN_GREEDY_TOPDOWN: return greedy(g, true, out, recompute_depth);
+    case ACC_PLAN_GREEDY_BOTTOMUP: return greedy(g, false, out, recompute_depth);
     default: return set_error(ACC_ERR_ARG, "unknown planner mode %d", mode);
   }
 }

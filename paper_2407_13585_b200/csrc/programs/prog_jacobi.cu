@@ -1,5 +1,6 @@
 // Kernels of one Jacobi iteration (five clamped shifts, four zipWiths): the nodes alone,
-// the whole iteration as one cluster, and the intermediate cuts the greedy planners reach.
+// the whole iteration as one cluster, the intermediate cuts the greedy planners reach, and
+// two to four whole iterations as one cluster.
 #include "../device/launch.cuh"
 #include "programs.h"
 
@@ -16,4 +17,10 @@ ACC_CLUSTER(kJacobi, 0x220, jac_w_Y)            // {w, Y}
 ACC_CLUSTER(kJacobi, 0x330, jac_ew_t3Y)         // {e, w, t3, Y}
 ACC_CLUSTER(kJacobi, 0x3C0, jac_sums)           // {t1, t2, t3, Y} over five manifest shifts
 ACC_CLUSTER(kJacobi, 0x380, jac_t2t3Y)          // {t2, t3, Y} over a manifest t1 and three manifest shifts
+// Several iterations in one cluster (a clustering that recomputes: the iterate in between is
+// read in five orders); the iterates in between stay in shared memory.
+using programs::kJacobiChain;
+ACC_CLUSTER(kJacobiChain, 0x7FFFEull, jac_two_iterations)
+ACC_CLUSTER(kJacobiChain, 0xFFFFFFEull, jac_three_iterations)
+ACC_CLUSTER(kJacobiChain, 0x1FFFFFFFFEull, jac_four_iterations)
 }  // namespace acc

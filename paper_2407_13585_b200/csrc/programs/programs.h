@@ -55,6 +55,23 @@ constexpr CProgram jacobi_iteration() {
   return p;
 }
 
+// A chain of Jacobi iterations (at most four): iteration t reads the result of iteration t - 1.
+constexpr CProgram jacobi_chain(int iters) {
+  CProgram p{1 + 9 * iters, 1ull << (9 * iters), {}};
+  p.nodes[0] = input(ACC_F32, 2);
+  int prev = 0;
+  for (int t = 0; t < iters; ++t) {
+    const int base = 1 + 9 * t;
+    for (int i = 0; i < 5; ++i) p.nodes[base + i] = pnode(ACC_BACKPERMUTE, ACC_F32, 2, 0, ACC_IDX_SHIFT_CLAMP, 1, prev);
+    p.nodes[base + 5] = pnode(ACC_ZIPWITH, ACC_F32, 2, ACC_FN_ADD, 0, 2, base + 0, base + 1);
+    p.nodes[base + 6] = pnode(ACC_ZIPWITH, ACC_F32, 2, ACC_FN_ADD, 0, 2, base + 5, base + 2);
+    p.nodes[base + 7] = pnode(ACC_ZIPWITH, ACC_F32, 2, ACC_FN_ADD, 0, 2, base + 6, base + 3);
+    p.nodes[base + 8] = pnode(ACC_ZIPWITH, ACC_F32, 2, ACC_FN_ADD_SCALE, 0, 2, base + 7, base + 4);
+    prev = base + 8;
+  }
+  return p;
+}
+
 // k = map(mul mod) keys; vals = generate(float(i mod m)); hist = permute(+) zeros k vals;
 // total = fold(+) vals; frac = map(/ total!0) hist
 constexpr CProgram histogram_diamond() {
@@ -73,6 +90,7 @@ inline constexpr CProgram kChain1d = chain1d();
 inline constexpr CProgram kTransposeReduce = transpose_reduce();
 inline constexpr CProgram kGatherScan = gather_scan();
 inline constexpr CProgram kJacobi = jacobi_iteration();
+inline constexpr CProgram kJacobiChain = jacobi_chain(4);
 inline constexpr CProgram kHistogram = histogram_diamond();
 
 }  // namespace programs

@@ -19,8 +19,9 @@ def count_of(nd):
     return int(np.prod(nd.shape, dtype=np.int64)) if len(nd.shape) else 1
 
 
-def gpu_run(prog, inputs_t, pi=None, executor=None, bind_all=True, runs=1):
+def gpu_run(prog, inputs_t, pi=None, executor=None, bind_all=True, runs=1, recompute=0):
     """Runs `prog` on the GPU.  pi=None with executor=UNFUSED runs one kernel per node.
+    recompute > 0: pi is checked under the recomputing rules with that depth.
     Returns ({node: numpy array} for every manifest non-input node, Graph)."""
     import torch
     from paper_2407_13585_b200 import binding as B
@@ -28,7 +29,10 @@ def gpu_run(prog, inputs_t, pi=None, executor=None, bind_all=True, runs=1):
     executor = B.FUSED if executor is None else executor
     g = B.Graph(prog.nodes, prog.outputs)
     if pi is not None:
-        g.set_partition(pi)
+        if recompute:
+            g.set_partition_recompute(pi, recompute)
+        else:
+            g.set_partition(pi)
     bufs = {}
     for i, nd in enumerate(prog.nodes):
         if nd.kind == "input":

@@ -72,6 +72,31 @@ def test_config4_iteration_cuts(rows, cols):
     check_program(prog, cuts)
 
 
+# Several Jacobi iterations per kernel (a clustering that recomputes: the iterate in between is
+# read in five orders).  Small domains are pulled through per read by the streaming kernel, from
+# 64 tiles on the iterates in between stay in shared memory; ragged edges in both directions,
+# tiles that lie on two array edges at once, depth 2 to 4.  Bit-exact like every element chain.
+@pytest.mark.parametrize("rows,cols,iters,depth", [
+    (8, 8, 2, 2), (40, 64, 4, 2), (33, 36, 3, 3),
+    (512, 1024, 4, 2), (520, 1028, 4, 2), (4100, 132, 2, 2), (64, 8192, 2, 2),
+    (515, 1028, 3, 3), (512, 1024, 4, 3), (520, 1036, 4, 4),
+])
+def test_config4_recomputing_clusters(rows, cols, iters, depth):
+    from paper_2407_13585_b200 import binding as B
+    prog = W.config4(rows, cols, iters=iters)
+    g = B.Graph(prog.nodes, prog.outputs)
+    assert g.plan("greedy_topdown", "bytes") == [-1] + [t for t in range(iters) for _ in range(9)]
+    pi = g.plan_recompute("greedy_topdown", "bytes", depth)
+    n_clusters = len({c for c in pi if c >= 0})
+    assert n_clusters == -(-iters // depth)
+    assert g.check_partition(pi) == "ACC_ERR_ILLEGAL_TRAVERSAL"        # not a clustering of the paper's model
+    inputs_t = W.make_inputs(prog)
+    ref = oracle_run(prog, np_inputs(inputs_t))
+    got, g2 = gpu_run(prog, inputs_t, pi, B.FUSED, recompute=depth, runs=2)
+    assert g2.launch_count() == n_clusters
+    compare(prog, ref, got, f"config4 {rows}x{cols} depth {depth}")
+
+
 def test_config4_four_iterations_planned():
     from paper_2407_13585_b200 import binding as B
     prog = W.config4(96, 128, iters=4)
