@@ -213,8 +213,9 @@ int acc_partition_cost(acc_graph* g, const int32_t* cluster_of_node, int32_t n_n
  * producer's producers inside the cluster).  What still fails: a scan asked for
  * an order other than its own, the one stored copy of a manifest array asked
  * for an order above 1, every rule that is not about orders, and more than
- * max_depth gather-like nodes stacked on one fused path.  max_depth = 0 is the
- * paper's model (the calls above).  The arrays computed are the same as under
+ * max_depth gather-like nodes stacked on one fused path of a cluster that needs
+ * such copies (a cluster that is legal in the paper's model stays legal).
+ * max_depth = 0 is the paper's model (the calls above).  The arrays computed are the same as under
  * any legal clustering; only the work and the traffic differ.
  * Arguments and results as for the calls of the same name above. */
 int acc_check_partition_recompute(acc_graph* g, const int32_t* cluster_of_node, int32_t n_nodes, int32_t max_depth);

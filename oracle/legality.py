@@ -27,6 +27,20 @@ numbers instead of being solved:
 
 The search over the free 0/1 orders of the manifest nodes of a cluster is
 done by plain enumeration.
+
+Clusterings that recompute (`recompute=k > 0`; not in the paper, whose
+Section 6 leaves fusion that duplicates work to future work).  The model is
+the paper's own, applied to an unfolded cluster: every member that is stored
+(manifest), is a scatter, or has no reader inside the cluster is a root, and
+below each root the cluster is unfolded into a tree in which every reader has
+a private copy of each producer it reads inside the cluster.  A copy has one
+reader, so its order is simply the order of the slot that reads it; roots are
+0 or 1; a copy of a scan must come out in the scan's own order; copies of
+gather-like nodes carry labels of their own.  No path of the tree may hold
+more than k gather-like nodes (a cluster that is legal without copies is
+legal whatever its depth).  Whether the cluster hangs together is judged
+on the original members: through fused edges, or through a common outside
+parent that copies of two members read in the same order.
 """
 from itertools import product
 
@@ -96,15 +110,15 @@ def manifest_set(nodes, outputs, pi, edges):
     return man
 
 
-def check(nodes, outputs, pi):
+def check(nodes, outputs, pi, recompute=0):
     """(True, "") if pi is legal, else (False, reason).  pi[i] is ignored for inputs."""
-    ok, why, _ = solve(nodes, outputs, pi)
+    ok, why, _ = solve(nodes, outputs, pi, recompute)
     return ok, why
 
 
-def solve(nodes, outputs, pi):
+def solve(nodes, outputs, pi, recompute=0):
     """check() plus, when legal, one satisfying order d^o per node (for a scatter: the
-    order of its index/value slots)."""
+    order of its index/value slots; under recompute: the order of a node's first copy)."""
     edges = edges_of(nodes)
     is_in = [nd.kind == "input" for nd in nodes]
     for e in edges:
@@ -130,6 +144,8 @@ def solve(nodes, outputs, pi):
     orders = {}
     for c in sorted(clusters):
         ok, why, d = _cluster_ok(nodes, edges, clusters[c], man, lab, pi)
+        if not ok and recompute:                    # a cluster of the paper's model needs no copies
+            ok, why, d = _cluster_ok_recompute(nodes, edges, clusters[c], man, recompute)
         if not ok:
             return False, f"cluster {c}: {why}", None
         orders.update(d)
@@ -174,6 +190,86 @@ def _cluster_ok(nodes, edges, members, man, lab, pi):
             continue
         if _connected(nodes, members, inner, outer, lab, d):
             return True, "", d
+        why = "disconnected: no fused array links all of its nodes"
+    return False, why, None
+
+
+def _cluster_ok_recompute(nodes, edges, members, man, max_depth):
+    """The unfolded-tree model described in the module text."""
+    mset = set(members)
+    inner = [e for e in edges if e.a in mset and e.b in mset]
+    outer = [e for e in edges if e.b in mset and e.a not in mset and e.ordered]
+    producers = {b: [e for e in inner if e.b == b] for b in members}
+    read_inside = {e.a for e in inner}
+    roots = [a for a in members if a in man or nodes[a].kind == "permute" or a not in read_inside]
+
+    # depth of stacking first: it also bounds the size of the tree
+    depth = {}
+    for a in members:                                  # producers come earlier in program order
+        below = max((depth[e.a] for e in producers[a]), default=0)
+        depth[a] = below + (1 if nodes[a].kind in ("gather", "backpermute") else 0)
+    if max(depth.values()) > max_depth:
+        return False, f"more than {max_depth} gather-like nodes stacked on a fused path", None
+
+    # the tree: copies[i] = (node, reader copy or None, slot of the reader)
+    copies = []
+
+    def unfold(a, reader, slot):
+        me = len(copies)
+        copies.append((a, reader, slot))
+        for e in producers[a]:
+            unfold(e.a, me, e.slot)
+
+    for r in roots:
+        unfold(r, None, None)
+
+    def label_slot(b, slot):
+        k = nodes[b].kind
+        return k == "backpermute" or (k == "gather" and slot == 1)
+
+    why = "traversal orders cannot be matched"
+    for choice in product((0, 1), repeat=len(roots)):
+        root_order = dict(zip(roots, choice))
+        d = []
+        ok = True
+        for i, (a, reader, slot) in enumerate(copies):
+            if reader is None:
+                o = root_order[a]
+            elif label_slot(copies[reader][0], slot):
+                o = ("label", reader)                  # the reader copy's own label: shared with nobody
+            else:
+                o = d[reader]
+            k = nodes[a].kind
+            if k == "scanl" and o != 0 or k == "scanr" and o != 1:
+                ok = False
+                break
+            d.append(o)
+        if not ok:
+            continue
+        # hanging together, on the original members
+        parent = {a: a for a in members}
+
+        def find(x):
+            while parent[x] != x:
+                parent[x] = parent[parent[x]]
+                x = parent[x]
+            return x
+
+        for e in inner:
+            parent[find(e.a)] = find(e.b)
+        groups = {}
+        for i, (a, _, _) in enumerate(copies):
+            for e in outer:
+                if e.b == a and not label_slot(a, e.slot):
+                    groups.setdefault((e.a, d[i]), []).append(a)
+        for g in groups.values():
+            for b in g[1:]:
+                parent[find(g[0])] = find(b)
+        if len({find(a) for a in members}) == 1:
+            first = {}
+            for i, (a, _, _) in enumerate(copies):
+                first.setdefault(a, d[i] if not isinstance(d[i], tuple) else 2 + d[i][1])
+            return True, "", first
         why = "disconnected: no fused array links all of its nodes"
     return False, why, None
 
@@ -246,7 +342,7 @@ def canonical_pi(nodes, blocks):
     return pi
 
 
-def enumerate_partitions(nodes, outputs):
+def enumerate_partitions(nodes, outputs, recompute=0):
     """Every legal clustering, each as a canonical pi list (inputs get -1), sorted."""
     items = [i for i, nd in enumerate(nodes) if nd.kind != "input"]
     found = []
@@ -254,7 +350,7 @@ def enumerate_partitions(nodes, outputs):
         pi = canonical_pi(nodes, blocks)
         if pi is None:
             continue
-        if check(nodes, outputs, pi)[0]:
+        if check(nodes, outputs, pi, recompute)[0]:
             found.append(pi)
     return sorted(found)
 

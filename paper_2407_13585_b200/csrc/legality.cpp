@@ -15,7 +15,8 @@
 // of that producer's producers inside the cluster).  The order equalities then only run from a
 // consumer to its own copies, so they can only fail at a scan (whose order is fixed) or at the
 // one stored copy of a manifest array (order 0 or 1).  At most `recompute_depth` gather-like
-// members may be stacked on a fused path.
+// members may be stacked on a fused path of a cluster that needs such copies; a cluster that is
+// legal in the paper's model stays legal whatever its depth.
 #include <algorithm>
 #include <map>
 
@@ -258,7 +259,8 @@ int check_partition(const Graph& g, const int32_t* pi, Solution* sol, bool quiet
   std::vector<int32_t> order(n, -1);
   for (auto& kv : clusters) {
     ClusterCheck cc(g, kv.second, man, label);
-    const int rc = recompute_depth > 0 ? cc.run_recompute(&order, recompute_depth) : cc.run(&order);
+    int rc = cc.run(&order);                             // a cluster of the paper's model needs no copies
+    if (rc != ACC_OK && recompute_depth > 0) rc = cc.run_recompute(&order, recompute_depth);
     if (rc != ACC_OK)
       return fail(rc, rc == ACC_ERR_DISCONNECTED ? "a cluster does not hang together through a fused array"
                                                  : "traversal orders cannot be matched",

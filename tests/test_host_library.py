@@ -87,6 +87,68 @@ def test_checker_equals_oracle_on_random_graphs():
     assert total > 500
 
 
+def _stencil_1d(iters):
+    # a three-point stencil per iteration: small enough to enumerate two iterations (10 nodes)
+    nodes = [Node("input", "f32", (1, 8), name="x")]
+    prev = 0
+    for _ in range(iters):
+        b = len(nodes)
+        for d in (0, -1, 1):
+            nodes.append(Node("backpermute", "f32", (1, 8), (prev,), 1, idx_fn="shift_clamp", iparam=(0, d)))
+        nodes.append(Node("zipwith", "f32", (1, 8), (b, b + 1), 2, fn="add"))
+        nodes.append(Node("zipwith", "f32", (1, 8), (b + 3, b + 2), 2, fn="add_scale", fparam=(0.25,)))
+        prev = b + 4
+    return nodes, [prev]
+
+
+@pytest.mark.parametrize("depth", [1, 2, 3])
+def test_recompute_enumeration_equals_oracle(depth):
+    progs = [(p.nodes, p.outputs) for p in (W.config1(64), W.config2(8), W.config3(64), W.config5(256, 16), W.simple2(),
+                                             W.simple3(), W.simple5(), W.scatter_example(16), W.greedy_bottom_up_bad(4, 5))]
+    progs.append(_stencil_1d(2))
+    grew = 0
+    for nodes, outputs in progs:
+        g = B.Graph(nodes, outputs)
+        mine, ref = g.enumerate_recompute(depth), L.enumerate_partitions(nodes, outputs, recompute=depth)
+        assert mine == ref, (nodes, outputs)
+        strict = g.enumerate()
+        assert set(map(tuple, strict)) <= set(map(tuple, mine))          # recomputing only adds clusterings
+        grew += len(mine) > len(strict)
+    assert grew >= 2
+
+
+def test_recompute_checker_equals_oracle_on_random_graphs():
+    rng = random.Random(4321)
+    more = 0
+    for _ in range(120):
+        nodes, outputs = _random_program(rng)
+        g = B.Graph(nodes, outputs)
+        for depth in (1, 2):
+            mine, ref = g.enumerate_recompute(depth), L.enumerate_partitions(nodes, outputs, recompute=depth)
+            assert mine == ref, (nodes, outputs, depth)
+        more += len(ref) > len(g.enumerate())
+        for _ in range(6):
+            pi = [-1, -1] + [rng.randrange(len(nodes) - 2) for _ in range(len(nodes) - 2)]
+            assert (g.check_partition_recompute(pi, 2) == "ACC_OK") == L.check(nodes, outputs, pi, recompute=2)[0], (nodes, outputs, pi)
+    assert more >= 5                       # graphs that gained clusterings by recomputing
+
+
+def test_recompute_planner_and_costs():
+    p = W.config4(8, 8, iters=4)
+    g = B.Graph(p.nodes, p.outputs)
+    strict = g.plan("greedy_topdown", "bytes")
+    assert len({c for c in strict if c >= 0}) == 4
+    paired = g.plan_recompute("greedy_topdown", "bytes", 2)
+    assert paired == [-1] + [0] * 18 + [1] * 18
+    assert g.check_partition(paired) == "ACC_ERR_ILLEGAL_TRAVERSAL" and g.check_partition_recompute(paired, 2) == "ACC_OK"
+    assert g.manifest() == [True] + [False] * 17 + [True] + [False] * 17 + [True]
+    # traffic halves: two kernels read and write one array each instead of four
+    assert g.partition_cost_recompute(paired, 2, "bytes") * 2 == g.partition_cost(strict, "bytes")
+    assert g.plan_recompute("greedy_topdown", "bytes", 4) == [-1] + [0] * 36
+    with pytest.raises(B.AccError):
+        g.plan_recompute("greedy_topdown", "bytes", -1)
+
+
 def test_check_partition_names_the_broken_rule():
     p = W.scatter_example_paper_graph()
     g = B.Graph(p.nodes, p.outputs)

@@ -209,3 +209,82 @@ def test_traffic_counts_shared_and_separate_reads():
     assert L.traffic(p.nodes, p.outputs, [-1, 0, 0, 0, 0]) == (2, 1)   # x in two orders; only s written
     q = W.simple5()
     assert L.traffic(q.nodes, q.outputs, [-1, -1, 0, 0, 0]) == (3, 1)  # is, xs in order 0, xs in the label
+
+
+# ---- clusterings that recompute (an extension: Section 6 leaves duplicated work to future work) ----
+
+def _two_orders():
+    # ys is read as it lies (by zs) and reversed (by bp): the pattern of Section 3.3's `simple5`
+    return [_inp("xs"),
+            Node("map", "f32", (8,), (0,), 1, fn="affine", fparam=(2.0, 1.0), name="ys"),
+            Node("backpermute", "f32", (8,), (1,), 1, idx_fn="reverse", name="bp"),
+            Node("zipwith", "f32", (8,), (2, 1), 2, fn="add", name="zs")]
+
+
+def test_recompute_lets_one_array_be_read_in_two_orders():
+    nodes = _two_orders()
+    # the paper's model: ys must be stored before bp reads it, so only {bp, zs} can fuse
+    assert L.enumerate_partitions(nodes, [3]) == [[-1, 0, 1, 1], [-1, 0, 1, 2]]
+    # with one copy of ys per order, ys fuses into bp (its stored copy still serves zs), and all
+    # three share a cluster; {ys, zs} without bp stays impossible (bp lies between them)
+    assert L.enumerate_partitions(nodes, [3], recompute=1) == [[-1, 0, 0, 0], [-1, 0, 0, 1], [-1, 0, 1, 1], [-1, 0, 1, 2]]
+    assert not L.check(nodes, [3], [-1, 0, 1, 0], recompute=1)[0]
+
+
+def test_recompute_does_not_change_what_is_not_about_orders():
+    # a scan can still not be produced in a gather's order
+    nodes = [_inp("is", "i32"), _inp("xs"),
+             Node("scanl", "f32", (8,), (1,), 1, fn="add", name="sc"),
+             Node("gather", "f32", (8,), (0, 2), 2, name="g")]
+    assert not L.check(nodes, [3], [-1, -1, 0, 0], recompute=2)[0]
+    # nor a stored array in both scan orders at once
+    nodes = [_inp("x"), Node("scanl", "f32", (8,), (0,), 1, fn="add"), Node("scanr", "f32", (8,), (0,), 1, fn="add"),
+             Node("zipwith", "f32", (8,), (1, 2), 2, fn="add")]
+    assert not L.check(nodes, [3], [-1, 0, 0, 0], recompute=2)[0]
+    # infusible edges, the execution order and the scatter rule are as before
+    p = W.scatter_example(16)
+    strict = L.enumerate_partitions(p.nodes, p.outputs)
+    assert L.enumerate_partitions(p.nodes, p.outputs, recompute=2) == strict
+    for prog in (W.config1(64), W.config3(64), W.config5(256, 16)):
+        assert L.enumerate_partitions(prog.nodes, prog.outputs, recompute=2) == L.enumerate_partitions(prog.nodes, prog.outputs)
+
+
+def test_recompute_copies_a_shared_producer_for_each_scan_direction():
+    # m feeds a scanl and a scanr: one order for m is impossible, one copy per scan is fine
+    nodes = [_inp("x"), Node("map", "f32", (8,), (0,), 1, fn="identity", name="m"),
+             Node("scanl", "f32", (8,), (1,), 1, fn="add"), Node("scanr", "f32", (8,), (1,), 1, fn="add")]
+    assert not L.check(nodes, [2, 3], [-1, 0, 0, 0])[0]
+    assert L.check(nodes, [2, 3], [-1, 0, 0, 0], recompute=1)[0]
+
+
+def test_recompute_depth_bounds_stacked_stencil_iterations():
+    p = W.config4(4, 4, iters=3)
+    one = [-1] + [0] * 27
+    two_one = [-1] + [0] * 18 + [1] * 9
+    assert not L.check(p.nodes, p.outputs, two_one)[0]                      # the paper's model: one iteration each
+    assert not L.check(p.nodes, p.outputs, two_one, recompute=1)[0]        # two shifts stacked
+    assert L.check(p.nodes, p.outputs, two_one, recompute=2)[0]
+    assert not L.check(p.nodes, p.outputs, one, recompute=2)[0]
+    assert L.check(p.nodes, p.outputs, one, recompute=3)[0]
+    # a cut inside an iteration ({c, n, s, t1, t2} | {e, w, t3, Y}) is as legal as before
+    cut = [-1, 0, 0, 0, 1, 1, 0, 0, 1, 1] + [2] * 18
+    assert not L.check(p.nodes, p.outputs, cut)[0] and L.check(p.nodes, p.outputs, cut, recompute=2)[0]
+    cut = [-1, 0, 0, 0, 1, 1, 0, 0, 1, 1] + [2] * 9 + [3] * 9
+    assert L.check(p.nodes, p.outputs, cut)[0] and L.check(p.nodes, p.outputs, cut, recompute=1)[0]
+
+
+def test_recomputing_clusters_compute_the_same_arrays():
+    import numpy as np
+    from oracle import cluster_loop, interp
+    nodes = _two_orders()
+    x = np.linspace(-1, 1, 8).astype(np.float32)
+    want = interp.run(nodes, {0: x}).values[3]
+    np.testing.assert_array_equal(want, (2 * x + 1)[::-1] + (2 * x + 1))     # worked by hand
+    for pi in L.enumerate_partitions(nodes, [3], recompute=1):
+        got = cluster_loop.run(nodes, [3], pi, {0: x})
+        assert np.array_equal(got[3].view(np.uint32), want.view(np.uint32)), pi
+    p = W.config4(5, 6, iters=2)
+    x = W.make_inputs(p)[0].numpy()
+    want = interp.run(p.nodes, {0: x}).values[p.outputs[0]]
+    got = cluster_loop.run(p.nodes, p.outputs, [-1] + [0] * 18, {0: x})
+    assert np.array_equal(got[p.outputs[0]].view(np.uint32), want.view(np.uint32))
