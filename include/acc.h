@@ -101,7 +101,9 @@ enum acc_plan_mode {
   ACC_PLAN_UNFUSED = 0,      /* every node its own cluster                             */
   ACC_PLAN_ENUMERATE,        /* best of all legal clusterings (small graphs only)      */
   ACC_PLAN_GREEDY_TOPDOWN,   /* Section 5 "Greedy": edges from the top of the graph    */
-  ACC_PLAN_GREEDY_BOTTOMUP   /* Section 5 "Greedy": edges from the bottom              */
+  ACC_PLAN_GREEDY_BOTTOMUP,  /* Section 5 "Greedy": edges from the bottom              */
+  ACC_PLAN_BRANCH_BOUND      /* exact search with a traffic lower bound (costs BYTES,
+                                READS_WRITES), started from the better greedy result    */
 };
 
 /* Cost functions of Section 4.1 (a)-(e), the sum of them ("everything" in
@@ -189,9 +191,16 @@ int acc_get_partition(const acc_graph* g, int32_t* cluster_of_node_out, int32_t 
 /* For the stored clustering: manifest_out[i] = 1 if node i is written to
  * memory (m_i = 0 in Figure 3), 0 if it is fused away. */
 int acc_manifest(const acc_graph* g, int32_t* manifest_out, int32_t n_nodes);
-/* Plans a clustering (Section 5, "Greedy"; exhaustive search in place of the
- * ILP solver) under `cost`, writes it to cluster_of_node_out (may be null) and
- * stores it.  ENUMERATE fails with ACC_ERR_TOO_LARGE beyond 12 non-input nodes. */
+/* Plans a clustering (Section 5, "Greedy"; exhaustive search or branch and
+ * bound in place of the ILP solver of Section 4) under `cost`, writes it to
+ * cluster_of_node_out (may be null) and stores it.  ENUMERATE fails with
+ * ACC_ERR_TOO_LARGE beyond 12 non-input nodes.  BRANCH_BOUND minimises
+ * Section 4.1's reads-and-writes objective (e), in arrays or in bytes: it assigns
+ * nodes to clusters in program order, drops a partial clustering as soon as it
+ * breaks a rule that more nodes cannot mend or as soon as the traffic it is
+ * already sure of (arrays that must be manifest in every clustering included)
+ * reaches the best clustering known, and gives up the proof, not the result,
+ * after 2^22 partial clusterings. */
 int acc_plan(acc_graph* g, int mode, int cost, int32_t* cluster_of_node_out);
 /* Every legal clustering, each as n_nodes int32 with canonical numbering
  * (clusters numbered in an execution order, ties by smallest node id), in
@@ -200,6 +209,12 @@ int acc_plan(acc_graph* g, int mode, int cost, int32_t* cluster_of_node_out);
 int64_t acc_enumerate(acc_graph* g, int32_t* out_pi, int64_t max_partitions);
 /* Cost of a legal clustering under `cost` (lower is better). */
 int acc_partition_cost(acc_graph* g, const int32_t* cluster_of_node, int32_t n_nodes, int cost, double* out);
+
+/* About the last acc_plan / acc_plan_recompute call on g: how many partial
+ * clusterings the search visited, and whether the result is proven to have the
+ * least cost (always for ENUMERATE; for BRANCH_BOUND unless the search stopped
+ * at its limit of visited clusterings; never for the greedy planners). */
+int acc_plan_info(const acc_graph* g, int64_t* visited_out, int32_t* proven_optimal_out);
 
 /* ---- clusterings that recompute (the paper's future work, Section 6) ----------- */
 

@@ -46,7 +46,8 @@ IDX_FN = {k[8:].lower(): v for k, v in ENUM.items() if k.startswith("ACC_IDX_")}
 STATUS_NAME = {v: k for k, v in ENUM.items() if k.startswith("ACC_ERR_") or k == "ACC_OK"}
 FUSED, UNFUSED = ENUM["ACC_EXEC_FUSED"], ENUM["ACC_EXEC_UNFUSED"]
 PLAN = {"unfused": ENUM["ACC_PLAN_UNFUSED"], "enumerate": ENUM["ACC_PLAN_ENUMERATE"],
-        "greedy_topdown": ENUM["ACC_PLAN_GREEDY_TOPDOWN"], "greedy_bottomup": ENUM["ACC_PLAN_GREEDY_BOTTOMUP"]}
+        "greedy_topdown": ENUM["ACC_PLAN_GREEDY_TOPDOWN"], "greedy_bottomup": ENUM["ACC_PLAN_GREEDY_BOTTOMUP"],
+        "branch_bound": ENUM["ACC_PLAN_BRANCH_BOUND"]}
 COST = {k[9:].lower(): v for k, v in ENUM.items() if k.startswith("ACC_COST_")}
 
 
@@ -89,6 +90,7 @@ def load_library(path=LIB_PATH):
         "acc_plan_recompute": (C.c_int, [p, C.c_int, C.c_int, i32, pi32]),
         "acc_enumerate_recompute": (i64, [p, i32, pi32, i64]),
         "acc_partition_cost_recompute": (C.c_int, [p, pi32, i32, i32, C.c_int, C.POINTER(C.c_double)]),
+        "acc_plan_info": (C.c_int, [p, C.POINTER(i64), C.POINTER(i32)]),
         "acc_bind": (C.c_int, [p, i32, p, sz]),
         "acc_bind_host": (C.c_int, [p, i32, p, sz]),
         "acc_workspace_bytes": (C.c_int, [p, C.c_int, C.POINTER(sz)]),
@@ -243,6 +245,12 @@ class Graph:
         out = (C.c_int32 * self.n)()
         _check(lib().acc_plan(self._h, PLAN[mode], COST[cost], out))
         return list(out)
+
+    def plan_info(self):
+        """(partial clusterings visited, result proven optimal) of the last plan call."""
+        visited, proven = C.c_int64(), C.c_int32()
+        _check(lib().acc_plan_info(self._h, C.byref(visited), C.byref(proven)))
+        return visited.value, bool(proven.value)
 
     def enumerate(self):
         cnt = _check(lib().acc_enumerate(self._h, None, 0))

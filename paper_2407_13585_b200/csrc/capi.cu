@@ -146,6 +146,14 @@ int acc_plan_recompute(acc_graph* g, int mode, int cost, int32_t max_depth, int3
 
 int acc_plan(acc_graph* g, int mode, int cost, int32_t* out) { return acc_plan_recompute(g, mode, cost, 0, out); }
 
+int acc_plan_info(const acc_graph* g, int64_t* visited, int32_t* proven) {
+  clear_error();
+  if (!g) return set_error(ACC_ERR_ARG, "graph is null");
+  if (visited) *visited = g->plan_visited;
+  if (proven) *proven = g->plan_proven ? 1 : 0;
+  return ACC_OK;
+}
+
 int64_t acc_enumerate(acc_graph* g, int32_t* out_pi, int64_t max_partitions) { return acc_enumerate_recompute(g, 0, out_pi, max_partitions); }
 
 int64_t acc_enumerate_recompute(acc_graph* g, int32_t max_depth, int32_t* out_pi, int64_t max_partitions) {

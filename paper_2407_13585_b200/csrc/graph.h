@@ -35,6 +35,8 @@ struct Graph {
   int recompute_depth = 0;         // the rules the stored clustering was checked under
   std::vector<uint8_t> manifest;   // under the stored clustering
   // bookkeeping of the last run
+  int64_t plan_visited = 0;        // partial clusterings the last planner call looked at
+  bool plan_proven = false;        // ... and whether its result is proven optimal
   int32_t launches = 0;
   std::string schedule;
   uint32_t host_status = 0;
@@ -55,11 +57,15 @@ int  add_node(Graph& g, const acc_node_desc& d);
 struct Solution {
   std::vector<uint8_t> manifest;   // per node
   std::vector<int32_t> order;      // d^o per node (for PERMUTE: order of its idx/vals slots), -1 for inputs
+  std::vector<std::vector<int32_t>> copies;   // clusters that recompute: every order a node is evaluated in (else empty)
 };
 // recompute_depth 0: the paper's rules; k > 0: producers may be evaluated once per order they are
 // read in, with at most k gather-like members stacked on a fused path
 int  check_partition(const Graph& g, const int32_t* pi, Solution* sol, bool quiet = false, int recompute_depth = 0);
 void manifest_of(const Graph& g, const int32_t* pi, std::vector<uint8_t>& man);
+bool partial_clustering_possible(const Graph& g, const std::vector<int>& block_of, int n_blocks, const std::vector<uint8_t>& man,
+                                 bool check_orders);
+void forced_manifest(const Graph& g, std::vector<uint8_t>& forced, std::vector<uint8_t>& must_read);
 
 // planner.cpp
 int     plan(Graph& g, int mode, int cost, std::vector<int32_t>& out, int recompute_depth = 0);

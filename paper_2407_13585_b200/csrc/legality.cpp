@@ -66,7 +66,9 @@ struct ClusterCheck {
     return kFree;
   }
 
-  int run(std::vector<int32_t>* order_out) {
+  // With need_connected = false only the order equalities are checked: what a cluster that is
+  // still growing can already get wrong for good.
+  int run(std::vector<int32_t>* order_out, bool need_connected = true) {
     const int m = (int)members.size();
     Dsu cls(m);
     for (const Edge& e : g.edges) {
@@ -97,6 +99,7 @@ struct ClusterCheck {
       const int r = cls.find(i);
       if (zero_one[r] && value[r] > 1) return ACC_ERR_ILLEGAL_TRAVERSAL;
     }
+    if (!need_connected) return ACC_OK;
     // connectivity: fused edges, or reads of one outside parent in one order
     Dsu base(m);
     for (const Edge& e : g.edges)
@@ -141,7 +144,7 @@ struct ClusterCheck {
   // a stored copy / a scatter / a member nobody in the cluster reads (encoded -1 - local id),
   // which is 0 or 1.  Members are visited consumers first; each passes the orders it is asked
   // for on to its producers, slot by slot.
-  int run_recompute(std::vector<int32_t>* order_out, int max_depth) {
+  int run_recompute(std::vector<int32_t>* order_out, int max_depth, std::vector<std::vector<int32_t>>* copies_out = nullptr) {
     const int m = (int)members.size();
     std::vector<std::vector<int>> asked(m);
     std::vector<int> bound(m, kFree);                    // value of variable i once a scan fixed it
@@ -220,6 +223,14 @@ struct ClusterCheck {
           for (int i = 0; i < m; ++i) {
             const int o = asked[i].empty() ? 0 : value_of(resolve(asked[i].front()));
             (*order_out)[members[i]] = o;
+            if (copies_out) {
+              std::vector<int32_t>& all = (*copies_out)[members[i]];
+              all.clear();
+              for (int q : asked[i]) {
+                const int v = value_of(resolve(q));
+                if (std::find(all.begin(), all.end(), v) == all.end()) all.push_back(v);
+              }
+            }
           }
         return ACC_OK;
       }
@@ -229,6 +240,90 @@ struct ClusterCheck {
 };
 
 }  // namespace
+
+// For a clustering of only some nodes (block_of[i] < 0: not placed yet): false if the placed
+// nodes already break a rule of the paper's model that placing more nodes cannot mend: an
+// infusible edge or a scatter and another reader of its destination inside one block, blocks
+// that need each other's results, or order equalities without a solution.  `man` marks arrays
+// that are manifest whatever happens to the nodes not placed yet.
+bool partial_clustering_possible(const Graph& g, const std::vector<int>& block_of, int n_blocks, const std::vector<uint8_t>& man,
+                                 bool check_orders) {
+  const int n = (int)g.nodes.size();
+  std::vector<std::vector<int>> after(n_blocks);
+  std::vector<int> waiting(n_blocks, 0);
+  auto link = [&](int from, int to) {
+    if (std::find(after[from].begin(), after[from].end(), to) == after[from].end()) { after[from].push_back(to); ++waiting[to]; }
+  };
+  for (const Edge& e : g.edges) {
+    if (block_of[e.a] < 0 || block_of[e.b] < 0) continue;
+    if (block_of[e.a] == block_of[e.b]) { if (!e.fusible) return false; }
+    else link(block_of[e.a], block_of[e.b]);
+  }
+  for (int j = 0; j < n; ++j) {
+    if (g.nodes[j].d.kind != ACC_PERMUTE || block_of[j] < 0) continue;
+    const int dest = g.nodes[j].d.inputs[0];
+    for (const Edge& e : g.edges)
+      if (e.a == dest && e.b != j && block_of[e.b] >= 0) {
+        if (block_of[e.b] == block_of[j]) return false;
+        link(block_of[e.b], block_of[j]);
+      }
+  }
+  std::vector<int> ready;
+  for (int b = 0; b < n_blocks; ++b)
+    if (waiting[b] == 0) ready.push_back(b);
+  int done = 0;
+  while (!ready.empty()) {
+    const int b = ready.back();
+    ready.pop_back();
+    ++done;
+    for (int t : after[b])
+      if (--waiting[t] == 0) ready.push_back(t);
+  }
+  if (done != n_blocks) return false;
+  if (!check_orders) return true;
+  std::vector<int> label(n, 0);
+  int next = 2;
+  for (int i = 0; i < n; ++i)
+    if (gather_like(g.nodes[i])) label[i] = next++;
+  std::vector<std::vector<int>> members(n_blocks);
+  for (int i = 0; i < n; ++i)
+    if (block_of[i] >= 0) members[block_of[i]].push_back(i);
+  for (int b = 0; b < n_blocks; ++b) {
+    if (members[b].size() < 2) continue;
+    ClusterCheck cc(g, members[b], man, label);
+    if (cc.run(nullptr, false) != ACC_OK) return false;
+  }
+  return true;
+}
+
+// Arrays that are manifest in every clustering of the paper's model: program outputs, arrays
+// nobody reads, arrays with an infusible out-edge, arrays read through a gather-like source slot
+// and by anyone else (fused with the gather-like reader its order is that reader's label, which
+// no second reader and no stored copy can have), arrays read by a scanl and a scanr.  must_read
+// marks those of them (and the inputs) that some cluster is sure to read from memory.
+void forced_manifest(const Graph& g, std::vector<uint8_t>& forced, std::vector<uint8_t>& must_read) {
+  const int n = (int)g.nodes.size();
+  forced.assign(n, 0);
+  must_read.assign(n, 0);
+  std::vector<int> readers(n, 0), label_readers(n, 0), array_readers(n, 0);
+  std::vector<uint8_t> infusible(n, 0), scanl(n, 0), scanr(n, 0);
+  for (const Edge& e : g.edges) {
+    ++readers[e.a];
+    const Node& b = g.nodes[e.b];
+    const bool array_slot = e.slot < b.d.n_array_inputs;
+    if (array_slot) ++array_readers[e.a];
+    if (!e.fusible && array_slot) infusible[e.a] = 1;
+    if (!e.fusible) forced[e.a] = 1;
+    if (b.d.kind == ACC_BACKPERMUTE || (b.d.kind == ACC_GATHER && e.slot == 1)) ++label_readers[e.a];
+    if (b.d.kind == ACC_SCANL) scanl[e.a] = 1;
+    if (b.d.kind == ACC_SCANR) scanr[e.a] = 1;
+  }
+  for (int i = 0; i < n; ++i) {
+    const bool clash = (label_readers[i] > 0 && readers[i] > 1) || (scanl[i] && scanr[i]);
+    if (is_input(g.nodes[i]) || g.nodes[i].output || readers[i] == 0 || clash) forced[i] = 1;
+    must_read[i] = (is_input(g.nodes[i]) && array_readers[i] > 0) || infusible[i] || clash;
+  }
+}
 
 int check_partition(const Graph& g, const int32_t* pi, Solution* sol, bool quiet, int recompute_depth) {
   const int n = (int)g.nodes.size();
@@ -257,10 +352,11 @@ int check_partition(const Graph& g, const int32_t* pi, Solution* sol, bool quiet
   for (int i = 0; i < n; ++i)
     if (!is_input(g.nodes[i])) clusters[pi[i]].push_back(i);
   std::vector<int32_t> order(n, -1);
+  std::vector<std::vector<int32_t>> copies(n);
   for (auto& kv : clusters) {
     ClusterCheck cc(g, kv.second, man, label);
     int rc = cc.run(&order);                             // a cluster of the paper's model needs no copies
-    if (rc != ACC_OK && recompute_depth > 0) rc = cc.run_recompute(&order, recompute_depth);
+    if (rc != ACC_OK && recompute_depth > 0) rc = cc.run_recompute(&order, recompute_depth, &copies);
     if (rc != ACC_OK)
       return fail(rc, rc == ACC_ERR_DISCONNECTED ? "a cluster does not hang together through a fused array"
                                                  : "traversal orders cannot be matched",
@@ -269,6 +365,7 @@ int check_partition(const Graph& g, const int32_t* pi, Solution* sol, bool quiet
   if (sol) {
     sol->manifest = man;
     sol->order = order;
+    sol->copies = copies;
   }
   return ACC_OK;
 }

@@ -80,6 +80,9 @@ int partition_cost(const Graph& g, const int32_t* pi, int cost, double* out, int
     else if (k == ACC_BACKPERMUTE || (k == ACC_GATHER && e.slot == 1)) order = lab[e.b];
     else order = sol.order[e.b];
     reads.insert(std::make_tuple(e.a, pi[e.b], order, uniq));
+    // a reader that is evaluated in several orders (a cluster that recomputes) reads once per order
+    if (e.ordered && order == sol.order[e.b] && e.b < (int)sol.copies.size())
+      for (int32_t o : sol.copies[e.b]) reads.insert(std::make_tuple(e.a, pi[e.b], (int)o, uniq));
   }
   double n_reads = 0, read_bytes = 0;
   for (auto& r : reads) { n_reads += 1; read_bytes += bytes(std::get<0>(r)); }
@@ -197,9 +200,124 @@ int greedy(const Graph& g, bool top_down, std::vector<int32_t>& out, int recompu
   return ACC_OK;
 }
 
+// Exact search for the cheapest clustering under the reads-and-writes objective of Section 4.1
+// (e), in arrays or in bytes.  Nodes are placed in program order, each into one of the blocks
+// that exist or into a new one (its producers' blocks first, so that the first leaves look like
+// the greedy results).  A partial clustering is dropped when it can no longer become legal
+// (partial_clustering_possible) or when the traffic it is already sure of is no less than the
+// best complete clustering known: every array that is manifest for certain is written once, and
+// read once by every placed block that reads it from outside and once more by each gather-like
+// reader, whose order no other read shares (at least once by somebody if that is certain too).
+struct BranchBound {
+  static constexpr int64_t kLimit = int64_t(1) << 22;
+  Graph& g;
+  const int cost, depth;
+  std::vector<int> items, block_of;
+  std::vector<uint8_t> forced, must_read, apart;
+  int n = 0, n_blocks = 0;
+  double best = 0;
+  std::vector<int32_t> best_pi;
+  int64_t visited = 0;
+  bool complete = true;
+
+  BranchBound(Graph& g_, int cost_, int depth_) : g(g_), cost(cost_), depth(depth_) {
+    n = (int)g.nodes.size();
+    block_of.assign(n, -1);
+    for (int i = 0; i < n; ++i)
+      if (!is_input(g.nodes[i])) items.push_back(i);
+    forced_manifest(g, forced, must_read);
+    if (depth > 0) {                       // with copies an array read in two orders can be fused away after all
+      for (int i = 0; i < n; ++i) {
+        bool infusible_out = false;
+        int readers = 0;
+        for (const Edge& e : g.edges)
+          if (e.a == i) { ++readers; infusible_out = infusible_out || !e.fusible; }
+        forced[i] = is_input(g.nodes[i]) || g.nodes[i].output || readers == 0 || infusible_out;
+        if (!is_input(g.nodes[i]) && !infusible_out) must_read[i] = 0;
+      }
+    }
+    apart.assign((size_t)n * n, 0);
+    for (const Edge& e : g.edges)
+      if (!e.fusible) apart[(size_t)e.a * n + e.b] = apart[(size_t)e.b * n + e.a] = 1;
+  }
+
+  double weight(int a) const { return cost == ACC_COST_BYTES ? double(std::max<int64_t>(g.nodes[a].count, 1)) * 4.0 : 1.0; }
+
+  // arrays that are manifest whatever happens to the nodes not placed yet
+  void certain_manifest(std::vector<uint8_t>& man) const {
+    man = forced;
+    for (const Edge& e : g.edges)
+      if (block_of[e.b] >= 0 && block_of[e.a] >= 0 && block_of[e.a] != block_of[e.b]) man[e.a] = 1;
+  }
+
+  double bound(const std::vector<uint8_t>& man) const {
+    double sum = 0;
+    std::vector<int> seen;
+    for (int a = 0; a < n; ++a) {
+      if (!man[a]) continue;
+      if (!is_input(g.nodes[a])) sum += weight(a);
+      seen.clear();
+      size_t by_label = 0;                                // a gather-like reader has an order of its own: a read of its own
+      for (const Edge& e : g.edges) {
+        if (e.a != a || e.slot >= g.nodes[e.b].d.n_array_inputs) continue;
+        const int k = g.nodes[e.b].d.kind;
+        const bool label_slot = k == ACC_BACKPERMUTE || (k == ACC_GATHER && e.slot == 1);
+        // in the paper's model a stored array cannot be fused into such a reader, placed or not
+        if (label_slot && depth == 0) { ++by_label; continue; }
+        if (block_of[e.b] < 0) continue;
+        if (!is_input(g.nodes[a]) && block_of[e.b] == block_of[a]) continue;
+        if (label_slot) { ++by_label; continue; }
+        if (std::find(seen.begin(), seen.end(), block_of[e.b]) == seen.end()) seen.push_back(block_of[e.b]);
+      }
+      sum += weight(a) * (double)std::max<size_t>(seen.size() + by_label, must_read[a] ? 1 : 0);
+    }
+    return sum;
+  }
+
+  void leaf() {
+    std::vector<int32_t> pi;
+    if (!canonical_numbering(g, block_of, n_blocks, pi)) return;
+    double c = 0;
+    if (check_partition(g, pi.data(), nullptr, true, depth) != ACC_OK) return;
+    if (partition_cost(g, pi.data(), cost, &c, depth) != ACC_OK) return;
+    if (c < best) { best = c; best_pi = pi; }
+  }
+
+  void search(size_t at) {
+    if (at == items.size()) { leaf(); return; }
+    const int node = items[at];
+    std::vector<int> order;                               // blocks to try: producers' first, then the rest, then a new one
+    for (int s = g.nodes[node].d.n_inputs - 1; s >= 0; --s) {
+      const int b = block_of[g.nodes[node].d.inputs[s]];
+      if (b >= 0 && std::find(order.begin(), order.end(), b) == order.end()) order.push_back(b);
+    }
+    for (int b = n_blocks - 1; b >= 0; --b)
+      if (std::find(order.begin(), order.end(), b) == order.end()) order.push_back(b);
+    order.push_back(n_blocks);
+    std::vector<uint8_t> man;
+    for (int b : order) {
+      bool ok = true;
+      for (size_t j = 0; j < at && ok; ++j)
+        if (block_of[items[j]] == b && apart[(size_t)items[j] * n + node]) ok = false;
+      if (!ok) continue;
+      if (++visited > kLimit) { complete = false; return; }
+      block_of[node] = b;
+      const int grown = b == n_blocks ? 1 : 0;
+      n_blocks += grown;
+      certain_manifest(man);
+      if (partial_clustering_possible(g, block_of, n_blocks, man, depth == 0) && bound(man) < best) search(at + 1);
+      n_blocks -= grown;
+      block_of[node] = -1;
+      if (!complete) return;
+    }
+  }
+};
+
 }  // namespace
 
 int plan(Graph& g, int mode, int cost, std::vector<int32_t>& out, int recompute_depth) {
+  g.plan_visited = 0;
+  g.plan_proven = false;
   const int n = (int)g.nodes.size();
   switch (mode) {
     case ACC_PLAN_UNFUSED: {
@@ -223,6 +341,28 @@ int plan(Graph& g, int mode, int cost, std::vector<int32_t>& out, int recompute_
         if (best_i < 0 || c < best) { best = c; best_i = i; }
       }
       out = all[best_i];
+      g.plan_visited = cnt;
+      g.plan_proven = true;
+      return ACC_OK;
+    }
+    case ACC_PLAN_BRANCH_BOUND: {
+      if (cost != ACC_COST_BYTES && cost != ACC_COST_READS_WRITES)
+        return set_error(ACC_ERR_ARG, "branch and bound minimises reads and writes (cost READS_WRITES or BYTES)");
+      BranchBound bb(g, cost, recompute_depth);
+      for (int top_down = 0; top_down < 2; ++top_down) {           // the better greedy result is the first incumbent
+        std::vector<int32_t> pi;
+        double c = 0;
+        if (greedy(g, top_down != 0, pi, recompute_depth) != ACC_OK) continue;
+        if (partition_cost(g, pi.data(), cost, &c, recompute_depth) != ACC_OK) continue;
+        if (bb.best_pi.empty() || c < bb.best) { bb.best = c; bb.best_pi = pi; }
+      }
+      if (bb.best_pi.empty()) bb.best = 1e300;                     // no greedy result: any legal clustering is better
+      clear_error();
+      bb.search(0);
+      if (bb.best_pi.empty()) return set_error(ACC_ERR_ARG, "no legal clustering");
+      out = bb.best_pi;
+      g.plan_visited = bb.visited;
+      g.plan_proven = bb.complete;
       return ACC_OK;
     }
     case ACC_PLAN_GREEDY_TOPDOWN: return greedy(g, true, out, recompute_depth);

@@ -7,6 +7,7 @@ import os
 import random
 import re
 
+import numpy as np
 import pytest
 
 import workloads as W
@@ -147,6 +148,60 @@ def test_recompute_planner_and_costs():
     assert g.plan_recompute("greedy_topdown", "bytes", 4) == [-1] + [0] * 36
     with pytest.raises(B.AccError):
         g.plan_recompute("greedy_topdown", "bytes", -1)
+
+
+def _oracle_minimum(nodes, outputs, weighted):
+    weight = (lambda nd: 4 * max(1, int(np.prod(nd.shape, dtype=np.int64)))) if weighted else (lambda nd: 1)
+    return min(sum(L.traffic(nodes, outputs, pi, weight)) for pi in L.enumerate_partitions(nodes, outputs))
+
+
+@pytest.mark.parametrize("prog", PROGRAMS, ids=lambda p: p.name)
+def test_branch_and_bound_finds_the_oracle_minimum(prog):
+    # the least reads + writes over the oracle's own enumeration, in arrays and in bytes
+    g = B.Graph(prog.nodes, prog.outputs)
+    for cost, weighted in (("reads_writes", False), ("bytes", True)):
+        pi = g.plan("branch_bound", cost)
+        visited, proven = g.plan_info()
+        assert proven and L.check(prog.nodes, prog.outputs, pi)[0]
+        assert g.partition_cost(pi, cost) == _oracle_minimum(prog.nodes, prog.outputs, weighted)
+    with pytest.raises(B.AccError):
+        g.plan("branch_bound", "clusters")
+
+
+def test_branch_and_bound_on_random_graphs_and_greedy_traps():
+    rng = random.Random(99)
+    for _ in range(60):
+        nodes, outputs = _random_program(rng)
+        g = B.Graph(nodes, outputs)
+        if not L.enumerate_partitions(nodes, outputs):            # e.g. a scatter whose destination depends on its result
+            with pytest.raises(B.AccError):
+                g.plan("branch_bound", "reads_writes")
+            continue
+        pi = g.plan("branch_bound", "reads_writes")
+        assert g.plan_info()[1]
+        assert g.partition_cost(pi, "reads_writes") == _oracle_minimum(nodes, outputs, False), (nodes, outputs)
+    # the two programs of Section 5 on which one of the greedy orders goes wrong
+    for prog, bad in ((W.greedy_bottom_up_bad(4, 5), "greedy_bottomup"), (W.greedy_top_down_bad(16), "greedy_topdown")):
+        g = B.Graph(prog.nodes, prog.outputs)
+        exact = g.partition_cost(g.plan("branch_bound", "bytes"), "bytes")
+        assert exact < g.partition_cost(g.plan(bad, "bytes"), "bytes")
+        assert exact == g.partition_cost(g.plan("enumerate", "bytes"), "bytes")
+
+
+def test_branch_and_bound_proves_the_jacobi_chain():
+    # 36 nodes: far beyond enumeration.  Every iterate is read by five backpermutes, so it is manifest
+    # in every clustering and read five times (five orders): 4 x (5 reads + 1 write) arrays is a lower
+    # bound, and the greedy clustering, one cluster per iteration, attains it.
+    p = W.config4(8, 8, iters=4)
+    g = B.Graph(p.nodes, p.outputs)
+    pi = g.plan("branch_bound", "reads_writes")
+    visited, proven = g.plan_info()
+    assert proven and visited < 1000
+    assert pi == [-1] + [t for t in range(4) for _ in range(9)] and g.partition_cost(pi, "reads_writes") == 24
+    # with recomputation allowed two iterations share a cluster: 2 x (5 reads + 1 write)
+    pi = g.plan_recompute("branch_bound", "reads_writes", 2)
+    assert g.plan_info()[1] and g.partition_cost_recompute(pi, 2, "reads_writes") == 12
+    assert pi == [-1] + [0] * 18 + [1] * 18
 
 
 def test_check_partition_names_the_broken_rule():
