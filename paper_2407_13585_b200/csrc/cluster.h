@@ -22,9 +22,14 @@ constexpr int kMaxSlots = ACC_MAX_INPUTS;
 constexpr int kMaxCluster = 40;   // local nodes per cluster
 constexpr int kMaxProgram = 40;   // nodes per build-time program
 
+// Constants of a node that select code instead of being run-time arguments: so far the
+// row and column offsets of a clamped shift when both lie in -1..1 (kRunTime: not fixed).
+constexpr int kRunTime = 9;
+
 struct PNode {                    // node of a build-time program
-  int kind, dtype, rank, fn, idxfn, nin, narr;
-  int in[kMaxSlots];
+  int kind = 0, dtype = 0, rank = 0, fn = 0, idxfn = 0, nin = 0, narr = 0;
+  int in[kMaxSlots] = {};
+  int p0 = kRunTime, p1 = kRunTime;
 };
 
 struct CProgram {
@@ -34,9 +39,10 @@ struct CProgram {
 };
 
 struct CNode {
-  int kind, dtype, rank, fn, idxfn, nin, narr;
-  int in[kMaxSlots];              // local ids
-  bool member, manifest;
+  int kind = 0, dtype = 0, rank = 0, fn = 0, idxfn = 0, nin = 0, narr = 0;
+  int in[kMaxSlots] = {};         // local ids
+  bool member = false, manifest = false;
+  int p0 = kRunTime, p1 = kRunTime;
 };
 
 struct CCluster {
@@ -50,6 +56,13 @@ constexpr PNode pnode(int kind, int dtype, int rank, int fn, int idxfn, int narr
   PNode p{kind, dtype, rank, fn, idxfn, 0, narr, {i0, i1, i2, i3, i4, i5}};
   for (int s = 0; s < kMaxSlots; ++s)
     if (p.in[s] >= 0) p.nin = s + 1;
+  return p;
+}
+
+// The same node with its two constants fixed at build time.
+constexpr PNode fixed(PNode p, int p0, int p1) {
+  p.p0 = p0;
+  p.p1 = p1;
   return p;
 }
 
@@ -73,6 +86,8 @@ constexpr CCluster extract(const CProgram& p, uint64_t mask) {
     }
     CNode m{nd.kind, nd.dtype, nd.rank, nd.fn, nd.idxfn, nd.nin, nd.narr, {-1, -1, -1, -1, -1, -1}, true, false};
     for (int s = 0; s < nd.nin; ++s) m.in[s] = local[nd.in[s]];
+    m.p0 = nd.p0;
+    m.p1 = nd.p1;
     bool consumed = false, outside = false;
     for (int j = i + 1; j < p.n; ++j)
       for (int s = 0; s < p.nodes[j].nin; ++s)
@@ -100,7 +115,8 @@ inline std::string signature(const CCluster& c) {
       s += buf;
       continue;
     }
-    snprintf(buf, sizeof buf, "M%d.%d.%d.%d.%d.%d.%d(", nd.kind, nd.dtype, nd.rank, nd.fn, nd.idxfn, nd.narr, (int)nd.manifest);
+    snprintf(buf, sizeof buf, "M%d.%d.%d.%d.%d.%d.%d.%d.%d(", nd.kind, nd.dtype, nd.rank, nd.fn, nd.idxfn, nd.narr, (int)nd.manifest,
+             nd.p0, nd.p1);
     s += buf;
     for (int k = 0; k < nd.nin; ++k) {
       snprintf(buf, sizeof buf, "%d,", nd.in[k]);

@@ -141,33 +141,33 @@ __device__ __forceinline__ IxG4 expand(const IxS4& i, int C) {
   return IxG4{{lane_clamped(i, 0, C), lane_clamped(i, 1, C), lane_clamped(i, 2, C), lane_clamped(i, 3, C)}};
 }
 
-template <int F> __device__ __forceinline__ auto map_index(const Ix& i, const NodeArg& self, const NodeArg& src) {
+template <int F, int P0 = kRunTime, int P1 = kRunTime> __device__ __forceinline__ auto map_index(const Ix& i, const NodeArg& self, const NodeArg& src) {
   return map1<F>(i, self, src);
 }
-template <int F> __device__ __forceinline__ auto map_index(const Ix4& i, const NodeArg& self, const NodeArg& src) {
+template <int F, int P0 = kRunTime, int P1 = kRunTime> __device__ __forceinline__ auto map_index(const Ix4& i, const NodeArg& self, const NodeArg& src) {
   if constexpr (F == ACC_IDX_IDENTITY) return i;
   else if constexpr (F == ACC_IDX_REVERSE) return IxR4{src.R - 1 - i.r, src.C - 1 - i.c};
   else if constexpr (F == ACC_IDX_SHIFT_CLAMP) return IxS4{min(max(i.r + self.ip0, 0), src.R - 1), i.c, self.ip1};
   else return map_lanes<F>(i, self, src);
 }
-template <int F> __device__ __forceinline__ auto map_index(const IxR4& i, const NodeArg& self, const NodeArg& src) {
+template <int F, int P0 = kRunTime, int P1 = kRunTime> __device__ __forceinline__ auto map_index(const IxR4& i, const NodeArg& self, const NodeArg& src) {
   if constexpr (F == ACC_IDX_IDENTITY) return i;
   else if constexpr (F == ACC_IDX_REVERSE) return Ix4{src.R - 1 - i.r, src.C - 1 - i.c};
   else return map_lanes<F>(i, self, src);
 }
-template <int F> __device__ __forceinline__ auto map_index(const IxG4& i, const NodeArg& self, const NodeArg& src) {
+template <int F, int P0 = kRunTime, int P1 = kRunTime> __device__ __forceinline__ auto map_index(const IxG4& i, const NodeArg& self, const NodeArg& src) {
   if constexpr (F == ACC_IDX_IDENTITY) return i;
   else return map_lanes<F>(i, self, src);
 }
-template <int F> __device__ __forceinline__ auto map_index(const IxPF4& i, const NodeArg&, const NodeArg& src) {
+template <int F, int P0 = kRunTime, int P1 = kRunTime> __device__ __forceinline__ auto map_index(const IxPF4& i, const NodeArg&, const NodeArg& src) {
   if constexpr (F == ACC_IDX_IDENTITY) return i;
   else if constexpr (F == ACC_IDX_REVERSE) return IxPF4{src.R - 1 - i.r, src.C - 4 - i.c};
   else return IxNone{0, 0};
 }
-template <int F> __device__ __forceinline__ auto map_index(const IxNone& i, const NodeArg&, const NodeArg&) { return i; }
+template <int F, int P0 = kRunTime, int P1 = kRunTime> __device__ __forceinline__ auto map_index(const IxNone& i, const NodeArg&, const NodeArg&) { return i; }
 // A shifted chunk names positions in the array it is applied to, which has the shape of
 // the node that receives it (`self`); a further map acts on its four clamped lanes.
-template <int F> __device__ __forceinline__ auto map_index(const IxS4& i, const NodeArg& self, const NodeArg& src) {
+template <int F, int P0 = kRunTime, int P1 = kRunTime> __device__ __forceinline__ auto map_index(const IxS4& i, const NodeArg& self, const NodeArg& src) {
   if constexpr (F == ACC_IDX_IDENTITY) return i;
   else return map_lanes<F>(expand(i, self.C), self, src);
 }
@@ -312,7 +312,7 @@ __device__ __forceinline__ val_of<IX> eval_here(const A& a, const IX& ix) {
   if constexpr (!nd.member) {
     return ld_ext<CL, I>(a, ix);
   } else if constexpr (nd.kind == ACC_BACKPERMUTE) {
-    return eval<CL, nd.in[0]>(a, map_index<nd.idxfn>(ix, a.n[I], a.n[nd.in[0]]));
+    return eval<CL, nd.in[0]>(a, map_index<nd.idxfn, nd.p0, nd.p1>(ix, a.n[I], a.n[nd.in[0]]));
   } else if constexpr (is_prefetch<IX>::value && (nd.kind == ACC_GATHER || nd.kind == ACC_FOLD || nd.kind == ACC_FOLDSEG)) {
     // where the data will be read from is not known before the data: only a gather's index
     // operand, read in the cluster's own order, can be fetched ahead

@@ -52,19 +52,24 @@ struct StCtx { const uint32_t* ext; const uint32_t* mem; };
 // four consecutive columns inside a box / the same after one clamped shift.  `off` is the word
 // offset of element (r, c) in a box; the box of slot k lies k box strides further.
 struct IxH4  { int r, c, off; StCtx t; };
-struct IxHS4 { int r, c, dc, off; StCtx t; };   // row r (already clamped), columns clamp(c+dc+j)
+// row r (already clamped), columns clamp(c+dc+j); DC is the column offset when the cluster was
+// built for it, else kRunTime and `dc` holds it
+template <int DC> struct IxHS4 { int r, c, dc, off; StCtx t; };
 
 __device__ __forceinline__ Ix lane(const IxH4& i, int j) { return Ix{i.r, i.c + j}; }
 
-template <int F> __device__ __forceinline__ auto map_index(const IxH4& i, const NodeArg& self, const NodeArg& src) {
+template <int F, int P0 = kRunTime, int P1 = kRunTime>
+__device__ __forceinline__ auto map_index(const IxH4& i, const NodeArg& self, const NodeArg& src) {
   static_assert(F == ACC_IDX_IDENTITY || F == ACC_IDX_SHIFT_CLAMP, "only clamped shifts are staged with a halo");
   if constexpr (F == ACC_IDX_IDENTITY) return i;
+  else if constexpr (P0 == 0) return IxHS4<P1>{i.r, i.c, self.ip1, i.off, i.t};
   else {
-    const int rr = min(max(i.r + self.ip0, 0), src.R - 1);
-    return IxHS4{rr, i.c, self.ip1, i.off + (rr - i.r) * kStBoxCols, i.t};
+    const int rr = min(max(i.r + (P0 != kRunTime ? P0 : self.ip0), 0), src.R - 1);
+    return IxHS4<P1>{rr, i.c, self.ip1, i.off + (rr - i.r) * kStBoxCols, i.t};
   }
 }
-template <int F> __device__ __forceinline__ auto map_index(const IxHS4& i, const NodeArg&, const NodeArg&) {
+template <int F, int P0 = kRunTime, int P1 = kRunTime, int DC>
+__device__ __forceinline__ auto map_index(const IxHS4<DC>& i, const NodeArg&, const NodeArg&) {
   static_assert(F == ACC_IDX_IDENTITY, "the source of a shift is read from a box, never pulled through");
   return i;
 }
@@ -143,10 +148,12 @@ __device__ __forceinline__ V4 ld_box(const uint32_t* p) {
   const uint4 v = *reinterpret_cast<const uint4*>(p);
   return V4{{v.x, v.y, v.z, v.w}};
 }
-__device__ __forceinline__ V4 ld_box(const uint32_t* p, const IxHS4& i, int C) {
+template <int DC>
+__device__ __forceinline__ V4 ld_box(const uint32_t* p, const IxHS4<DC>& i, int C) {
   const uint4 v = *reinterpret_cast<const uint4*>(p);
-  if (i.dc == 1) return V4{{v.y, v.z, v.w, p[min(4, C - 1 - i.c)]}};      // clamped at the last column
-  if (i.dc == -1) return V4{{p[max(-1, -i.c)], v.x, v.y, v.z}};           // clamped at the first column
+  const int dc = DC != kRunTime ? DC : i.dc;
+  if (dc == 1) return V4{{v.y, v.z, v.w, p[min(4, C - 1 - i.c)]}};        // clamped at the last column
+  if (dc == -1) return V4{{p[max(-1, -i.c)], v.x, v.y, v.z}};             // clamped at the first column
   return V4{{v.x, v.y, v.z, v.w}};                                         // dc == 0 (larger shifts never get here)
 }
 
@@ -154,15 +161,15 @@ template <class CL, int I, class A>
 __device__ __forceinline__ V4 ld_ext(const A&, const IxH4& ix) {
   return ld_box(ix.t.ext + tile_slot<CL>(I) * st_box_stride(max_shift_depth<CL>()) + ix.off);
 }
-template <class CL, int I, class A>
-__device__ __forceinline__ V4 ld_ext(const A& a, const IxHS4& ix) {
+template <class CL, int I, class A, int DC>
+__device__ __forceinline__ V4 ld_ext(const A& a, const IxHS4<DC>& ix) {
   return ld_box(ix.t.ext + tile_slot<CL>(I) * st_box_stride(max_shift_depth<CL>()) + ix.off, ix, a.n[I].C);
 }
 
 // members kept on chip are read from their box at a shifted index, computed anywhere else
-template <class CL, int I> struct reads_staged<CL, I, IxHS4> { static constexpr bool value = is_staged_member<CL>(I); };
-template <class CL, int I, class A>
-__device__ __forceinline__ V4 ld_staged(const A& a, const IxHS4& ix) {
+template <class CL, int I, int DC> struct reads_staged<CL, I, IxHS4<DC>> { static constexpr bool value = is_staged_member<CL>(I); };
+template <class CL, int I, class A, int DC>
+__device__ __forceinline__ V4 ld_staged(const A& a, const IxHS4<DC>& ix) {
   return ld_box(ix.t.mem + member_slot<CL>(I) * st_box_stride(max_shift_depth<CL>()) + ix.off, ix, a.n[I].C);
 }
 

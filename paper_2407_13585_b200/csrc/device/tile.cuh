@@ -43,12 +43,12 @@ struct IxQ4 { int r, c; const TileCtx* t; };     // positions (c, r+j) of the so
 __device__ __forceinline__ Ix lane(const IxP4& i, int j) { return Ix{i.r + j, i.c}; }
 __device__ __forceinline__ Ix lane(const IxQ4& i, int j) { return Ix{i.c, i.r + j}; }
 
-template <int F> __device__ __forceinline__ auto map_index(const IxP4& i, const NodeArg&, const NodeArg&) {
+template <int F, int P0 = kRunTime, int P1 = kRunTime> __device__ __forceinline__ auto map_index(const IxP4& i, const NodeArg&, const NodeArg&) {
   static_assert(F == ACC_IDX_IDENTITY || F == ACC_IDX_TRANSPOSE, "only transposes are staged in tiles");
   if constexpr (F == ACC_IDX_IDENTITY) return i;
   else return IxQ4{i.r, i.c, i.t};
 }
-template <int F> __device__ __forceinline__ auto map_index(const IxQ4& i, const NodeArg&, const NodeArg&) {
+template <int F, int P0 = kRunTime, int P1 = kRunTime> __device__ __forceinline__ auto map_index(const IxQ4& i, const NodeArg&, const NodeArg&) {
   static_assert(F == ACC_IDX_IDENTITY || F == ACC_IDX_TRANSPOSE, "only transposes are staged in tiles");
   if constexpr (F == ACC_IDX_IDENTITY) return i;
   else return IxP4{i.r, i.c, i.t};
@@ -374,12 +374,12 @@ struct IxBT4 { int r, c, j; const BlkCtx* b; };     // positions (c..c+3, r) of 
 __device__ __forceinline__ Ix lane(const IxB4& i, int k) { return Ix{i.r, i.c + k}; }
 __device__ __forceinline__ Ix lane(const IxBT4& i, int k) { return Ix{i.c + k, i.r}; }
 
-template <int F> __device__ __forceinline__ auto map_index(const IxB4& i, const NodeArg&, const NodeArg&) {
+template <int F, int P0 = kRunTime, int P1 = kRunTime> __device__ __forceinline__ auto map_index(const IxB4& i, const NodeArg&, const NodeArg&) {
   static_assert(F == ACC_IDX_IDENTITY || F == ACC_IDX_TRANSPOSE, "only transposes are staged in tiles");
   if constexpr (F == ACC_IDX_IDENTITY) return i;
   else return IxBT4{i.r, i.c, i.j, i.b};
 }
-template <int F> __device__ __forceinline__ auto map_index(const IxBT4& i, const NodeArg&, const NodeArg&) {
+template <int F, int P0 = kRunTime, int P1 = kRunTime> __device__ __forceinline__ auto map_index(const IxBT4& i, const NodeArg&, const NodeArg&) {
   static_assert(F == ACC_IDX_IDENTITY || F == ACC_IDX_TRANSPOSE, "only transposes are staged in tiles");
   if constexpr (F == ACC_IDX_IDENTITY) return i;
   else return IxB4{i.r, i.c, i.j, i.b};

@@ -38,6 +38,11 @@ static bool extract_runtime(const Graph& g, const std::vector<int>& members, con
     CNode n{d.kind, d.dtype, d.rank, d.fn_id, d.idx_fn_id, d.n_inputs, d.n_array_inputs, {-1, -1, -1, -1, -1, -1}, true, man[m] != 0};
     if (d.kind != ACC_BACKPERMUTE) n.idxfn = 0;
     if (d.kind == ACC_BACKPERMUTE || d.kind == ACC_GATHER) n.fn = 0;
+    if (d.kind == ACC_BACKPERMUTE && d.idx_fn_id == ACC_IDX_SHIFT_CLAMP && d.iparam[0] >= -1 && d.iparam[0] <= 1 &&
+        d.iparam[1] >= -1 && d.iparam[1] <= 1) {
+      n.p0 = (int)d.iparam[0];                         // kernels built for these very offsets are looked up first
+      n.p1 = (int)d.iparam[1];
+    }
     for (int s = 0; s < d.n_inputs; ++s) n.in[s] = local[d.inputs[s]];
     local[m] = c.n;
     c.source[c.n] = m;
@@ -114,8 +119,13 @@ int build_schedule(Graph& g, int executor, Schedule& sch) {
     st.n_members = (int)kv.second.size();
     if (!extract_runtime(g, kv.second, man, st.cc))
       return set_error(ACC_ERR_NO_KERNEL, "cluster at node %d has more than %d local nodes", st.first_node, kMaxCluster);
-    const std::string sig = signature(st.cc);
+    std::string sig = signature(st.cc);
     st.kernel = find_kernel(sig);
+    if (!st.kernel) {                                   // none for these constants: the one that takes them at run time
+      for (int li = 0; li < st.cc.n; ++li) st.cc.nodes[li].p0 = st.cc.nodes[li].p1 = kRunTime;
+      sig = signature(st.cc);
+      st.kernel = find_kernel(sig);
+    }
     if (!st.kernel)
       return set_error(ACC_ERR_NO_KERNEL, "no kernel instantiated for the cluster of %d nodes starting at node %d [%s]",
                        st.n_members, st.first_node, sig.c_str());

@@ -56,13 +56,17 @@ constexpr CProgram jacobi_iteration() {
 }
 
 // A chain of Jacobi iterations (at most four): iteration t reads the result of iteration t - 1.
+// The shifts are the five-point pattern, fixed at build time: centre, row above, row below, column
+// to the right, column to the left.
 constexpr CProgram jacobi_chain(int iters) {
   CProgram p{1 + 9 * iters, 1ull << (9 * iters), {}};
   p.nodes[0] = input(ACC_F32, 2);
   int prev = 0;
+  constexpr int dr[5] = {0, -1, 1, 0, 0}, dc[5] = {0, 0, 0, 1, -1};
   for (int t = 0; t < iters; ++t) {
     const int base = 1 + 9 * t;
-    for (int i = 0; i < 5; ++i) p.nodes[base + i] = pnode(ACC_BACKPERMUTE, ACC_F32, 2, 0, ACC_IDX_SHIFT_CLAMP, 1, prev);
+    for (int i = 0; i < 5; ++i)
+      p.nodes[base + i] = fixed(pnode(ACC_BACKPERMUTE, ACC_F32, 2, 0, ACC_IDX_SHIFT_CLAMP, 1, prev), dr[i], dc[i]);
     p.nodes[base + 5] = pnode(ACC_ZIPWITH, ACC_F32, 2, ACC_FN_ADD, 0, 2, base + 0, base + 1);
     p.nodes[base + 6] = pnode(ACC_ZIPWITH, ACC_F32, 2, ACC_FN_ADD, 0, 2, base + 5, base + 2);
     p.nodes[base + 7] = pnode(ACC_ZIPWITH, ACC_F32, 2, ACC_FN_ADD, 0, 2, base + 6, base + 3);
