@@ -114,7 +114,7 @@ class ClockSampler:
 class Workload:
     """One program at one size: graph, device buffers, pinned host mirrors."""
 
-    def __init__(self, cfg, sizes, device, host=True):
+    def __init__(self, cfg, sizes, device, host=True, recompute=0):
         import torch
         import workloads as W
         from paper_2407_13585_b200 import binding as B
@@ -124,8 +124,12 @@ class Workload:
         self.elements = elements_of(self.prog)
         self.g = B.Graph(self.prog.nodes, self.prog.outputs)
         n_ops = sum(nd.kind != "input" for nd in self.prog.nodes)
-        self.plan_mode = "enumerate" if n_ops <= 12 else "greedy_topdown"
-        self.pi = self.g.plan(self.plan_mode, "bytes")
+        # small graphs: best of all legal clusterings; larger ones: branch and bound from the greedy result
+        self.plan_mode = "enumerate" if n_ops <= 12 else "branch_bound"
+        t0 = time.perf_counter()
+        self.pi = self.g.plan_recompute(self.plan_mode, "bytes", recompute) if recompute else self.g.plan(self.plan_mode, "bytes")
+        self.plan_ms = (time.perf_counter() - t0) * 1e3
+        self.plan_visited, self.plan_proven = self.g.plan_info()
         self.inputs = W.make_inputs(self.prog, device=device)
         self.outputs = {}
         self.host = {}
@@ -239,7 +243,8 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     order = [c for c in ORDER if c in args.configs]
-    loads = [Workload(cfg, scaled(FULL[cfg], args.shrink), device, host=not args.fused_only) for cfg in order]
+    loads = [Workload(cfg, scaled(FULL[cfg], args.shrink), device, host=not args.fused_only,
+                      recompute=args.recompute_depth if args.fused_only else 0) for cfg in order]
     step_bytes = sum(w.bytes for w in loads)
 
     def step():
@@ -289,11 +294,35 @@ def run_ours(args):
         w.g.workspace = w.ws[B.FUSED]
         torch.cuda.empty_cache()
         per[w.cfg] = {
-            "clustering": w.pi, "planner": w.plan_mode, "ms_fused": ms_f, "ms_unfused": ms_u, "speedup": ms_u / ms_f,
+            "clustering": w.pi, "planner": w.plan_mode, "planner_ms": w.plan_ms, "planner_visited": w.plan_visited,
+            "planner_proven_optimal": w.plan_proven, "ms_fused": ms_f, "ms_unfused": ms_u, "speedup": ms_u / ms_f,
             "launches_fused": n_f, "launches_unfused": n_u, "compulsory_bytes": w.bytes,
             "effective_gbs": w.bytes / ms_f / 1e6, "pct_of_8TBs": 100.0 * w.bytes / ms_f / 1e6 / NOMINAL_HBM_GBS,
             "gelem_s": w.elements / ms_f / 1e6,
         }
+
+    # Beside the paper's model: the Jacobi chain under a clustering that recomputes (two stacked
+    # iterations per kernel, the iterate in between kept in shared memory).  Not part of the timed step.
+    for w in loads:
+        if w.cfg != 4:
+            continue
+        strict_pi = list(w.pi)
+        pi2 = w.g.plan_recompute("branch_bound", "bytes", 2)
+        w.g.workspace = None
+        ws2 = w.g.ensure_workspace(B.FUSED)
+        for _ in range(3):
+            w.g.run(B.FUSED, finish=False)
+        ms_r = time_region(lambda: w.g.run(B.FUSED, finish=False), reps)
+        n_r = w.g.launch_count()
+        w.g.finish()
+        per[4]["recompute_depth_2"] = {
+            "clustering": pi2, "ms_fused": ms_r, "launches_fused": n_r, "effective_gbs": w.bytes / ms_r / 1e6,
+            "pct_of_8TBs": 100.0 * w.bytes / ms_r / 1e6 / NOMINAL_HBM_GBS, "speedup_vs_unfused": per[4]["ms_unfused"] / ms_r,
+            "note": "outside the paper's legality model (its Section 6 leaves duplicated work to future work)"}
+        w.g.set_partition(strict_pi)
+        del ws2
+        w.g.workspace = w.ws[B.FUSED]
+        torch.cuda.empty_cache()
 
     # end to end: pinned host inputs in, outputs out, every step
     def e2e_step():
@@ -329,11 +358,11 @@ def run_ours(args):
     wtop = [w for w in loads if w.cfg == top][0]
     peak, peak_kind = measured_peak()
     achieved = kernel_bytes[top](wtop) / (per[top]["ms_fused"] / kernel_launches[top]) / 1e6
-    names = {2: "k_tile_pair<transpose+zip+fold>", 3: "k_scan<hash+gather+mask+scan>", 4: "k_stencil<jacobi iteration>",
+    names = {2: "k_tile_pair_tma<transpose+zip+fold>", 3: "k_scan<hash+gather+mask+scan>", 4: "k_stencil<jacobi iteration>",
              5: "k_hist<hash+generate+permute+fold>", 1: "k_stream<chain>"}
     # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
     # summarised under profiles/, taken at these sizes; null for a kernel without a capture
-    ncu_traffic = {3: 6.266e9 + 0.259e9, 4: 268.7e6 + 217.1e6, 2: 269.5e6 + 7.8e6, 5: 542.6e6 + 4.4e6}
+    ncu_traffic = {3: 6.266e9 + 0.2575e9, 4: 268.5e6 + 217.4e6, 2: 270.8e6 + 7.6e6, 5: 542.6e6 + 3.7e6}
     traffic = ncu_traffic.get(top) if args.shrink == 0 else None
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": traffic, "kernel": names[top], "of": peak_kind,
@@ -376,6 +405,8 @@ def main():
     ap.add_argument("--configs", default="1,2,3,4,5", help="programs to include (profiling aid)")
     ap.add_argument("--shrink", type=int, default=0, help="divide every element count by 2^SHRINK (profiling aid)")
     ap.add_argument("--fused-only", action="store_true", help="time the fused steps only (profiling aid)")
+    ap.add_argument("--recompute-depth", type=int, default=0,
+                    help="with --fused-only: plan with clusterings that recompute, this many stacked gather-like nodes (profiling aid)")
     args = ap.parse_args()
     args.configs = [int(c) for c in args.configs.split(",")]
     if args.impl == "reference":
