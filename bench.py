@@ -325,12 +325,25 @@ def run_ours(args):
         torch.cuda.empty_cache()
 
     # end to end: pinned host inputs in, outputs out, every step
+    # (the programs go to two streams in turn, so that one program's copy back overlaps the next
+    # one's copy in; the step ends when every program has been waited for)
+    main = torch.cuda.current_stream()
+    lanes = [torch.cuda.Stream(), torch.cuda.Stream()]
+
     def e2e_step():
         up = down = 0
-        for w in loads:
+        for lane in lanes:
+            lane.wait_stream(main)
+        for k, w in enumerate(loads):
             w.g.workspace = w.ws[B.FUSED]
-            u, d = w.g.run_e2e(B.FUSED)
+            with torch.cuda.stream(lanes[k % 2]):
+                u, d = w.g.run_e2e(B.FUSED, finish=False)
             up, down = up + u, down + d
+        for k, w in enumerate(loads):
+            with torch.cuda.stream(lanes[k % 2]):
+                w.finish()
+        for lane in lanes:
+            main.wait_stream(lane)
         return up, down
 
     e2e_step()

@@ -267,6 +267,12 @@ int acc_finish(acc_graph* g, void* workspace, void* cuda_stream);
  * returns as acc_finish.  h2d/d2h receive the bytes copied (may be null). */
 int acc_run_e2e(acc_graph* g, void* workspace, size_t workspace_bytes, void* cuda_stream, int executor,
                 size_t* h2d_bytes, size_t* d2h_bytes);
+/* The same without the wait: the copies and the launches are enqueued and the
+ * call returns; acc_finish on the same stream waits and reports.  Programs
+ * enqueued this way on different streams overlap their copies in both
+ * directions with each other and with the kernels. */
+int acc_run_e2e_async(acc_graph* g, void* workspace, size_t workspace_bytes, void* cuda_stream, int executor,
+                      size_t* h2d_bytes, size_t* d2h_bytes);
 /* Kernels launched by the last acc_run / acc_run_e2e on this graph. */
 int32_t acc_launch_count(const acc_graph* g);
 /* Clusters of the last run, as "first_node:count" items separated by blanks,

@@ -97,6 +97,7 @@ def load_library(path=LIB_PATH):
         "acc_run": (C.c_int, [p, p, sz, p, C.c_int]),
         "acc_finish": (C.c_int, [p, p, p]),
         "acc_run_e2e": (C.c_int, [p, p, sz, p, C.c_int, C.POINTER(sz), C.POINTER(sz)]),
+        "acc_run_e2e_async": (C.c_int, [p, p, sz, p, C.c_int, C.POINTER(sz), C.POINTER(sz)]),
         "acc_launch_count": (i32, [p]),
         "acc_last_schedule": (C.c_int, [p, C.c_char_p, sz]),
         "acc_scanl_add_i32_static": (C.c_int, [p, p, i64, p]),
@@ -302,11 +303,13 @@ class Graph:
         ws = self.workspace
         _check(lib().acc_finish(self._h, C.c_void_p(ws.data_ptr()) if ws is not None else None, self._stream()))
 
-    def run_e2e(self, executor=FUSED):
+    def run_e2e(self, executor=FUSED, finish=True):
+        """Host inputs in, program, host outputs out on the current stream; finish=False returns
+        after enqueueing (call finish() under the same stream later)."""
         ws = self.ensure_workspace(executor)
         up, down = C.c_size_t(), C.c_size_t()
-        _check(lib().acc_run_e2e(self._h, C.c_void_p(ws.data_ptr()), ws.numel(), self._stream(), executor,
-                                 C.byref(up), C.byref(down)))
+        fn = lib().acc_run_e2e if finish else lib().acc_run_e2e_async
+        _check(fn(self._h, C.c_void_p(ws.data_ptr()), ws.numel(), self._stream(), executor, C.byref(up), C.byref(down)))
         return up.value, down.value
 
     def launch_count(self):

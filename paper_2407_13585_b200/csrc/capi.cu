@@ -230,6 +230,13 @@ int acc_finish(acc_graph* g, void* workspace, void* cuda_stream) {
 
 int acc_run_e2e(acc_graph* g, void* workspace, size_t workspace_bytes, void* cuda_stream, int executor,
                 size_t* h2d_bytes, size_t* d2h_bytes) {
+  const int rc = acc_run_e2e_async(g, workspace, workspace_bytes, cuda_stream, executor, h2d_bytes, d2h_bytes);
+  if (rc != ACC_OK) return rc;
+  return finish(*g, workspace, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int acc_run_e2e_async(acc_graph* g, void* workspace, size_t workspace_bytes, void* cuda_stream, int executor,
+                      size_t* h2d_bytes, size_t* d2h_bytes) {
   clear_error();
   if (!g) return set_error(ACC_ERR_ARG, "graph is null");
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -253,7 +260,7 @@ int acc_run_e2e(acc_graph* g, void* workspace, size_t workspace_bytes, void* cud
     }
   if (h2d_bytes) *h2d_bytes = up;
   if (d2h_bytes) *d2h_bytes = down;
-  return finish(*g, workspace, stream);
+  return ACC_OK;
 }
 
 int32_t acc_launch_count(const acc_graph* g) { return g ? g->launches : ACC_ERR_ARG; }

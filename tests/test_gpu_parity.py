@@ -122,6 +122,57 @@ def test_runs_are_repeatable():
     check_program(W.config5(1 << 16, 256), runs=3)
 
 
+def test_end_to_end_with_host_buffers():
+    # acc_run_e2e: pinned host inputs in, program, host outputs out; then two programs enqueued on two
+    # streams with acc_run_e2e_async and waited for afterwards (their copies may overlap)
+    import torch
+    from paper_2407_13585_b200 import binding as B
+
+    def prepare(prog):
+        g = B.Graph(prog.nodes, prog.outputs)
+        g.plan("enumerate", "bytes")
+        inputs = W.make_inputs(prog)
+        host = {}
+        for i, t in inputs.items():
+            g.bind(i, torch.empty_like(t, device="cuda"))          # device copy filled by the call
+            host[i] = t.contiguous().pin_memory()
+            g.bind_host(i, host[i])
+        for o in prog.outputs:
+            nd = prog.nodes[o]
+            n = max(int(np.prod(nd.shape, dtype=np.int64)) if nd.shape else 1, 4)
+            g.bind(o, torch.empty(n, dtype=torch.int32, device="cuda"))
+            host[o] = torch.full((n,), -7, dtype=torch.int32).pin_memory()
+            g.bind_host(o, host[o])
+        return g, inputs, host
+
+    def check(prog, inputs, host, what):
+        ref = oracle_run(prog, np_inputs(inputs))
+        got = {}
+        for o in prog.outputs:
+            nd = prog.nodes[o]
+            n = int(np.prod(nd.shape, dtype=np.int64)) if nd.shape else 1
+            a = host[o][:n].numpy()
+            got[o] = (a.view(np.float32) if nd.dtype == "f32" else a.view(np.uint32)).reshape(tuple(nd.shape))
+        compare(prog, ref, got, what)
+
+    p3, p5 = W.config3(1 << 18), W.config5(1 << 18, 1 << 10)
+    g3, in3, h3 = prepare(p3)
+    up, down = g3.run_e2e(B.FUSED)
+    assert up == 2 * 4 * (1 << 18) and down == 4 * (1 << 18)
+    check(p3, in3, h3, "config3 end to end")
+    g5, in5, h5 = prepare(p5)
+    h3[p3.outputs[0]].fill_(-7)
+    lanes = [torch.cuda.Stream(), torch.cuda.Stream()]
+    for lane, g in zip(lanes, (g3, g5)):
+        with torch.cuda.stream(lane):
+            g.run_e2e(B.FUSED, finish=False)
+    for lane, g in zip(lanes, (g3, g5)):
+        with torch.cuda.stream(lane):
+            g.finish()
+    check(p3, in3, h3, "config3 end to end, enqueued")
+    check(p5, in5, h5, "config5 end to end, enqueued")
+
+
 PAPER_EXAMPLES = [W.scatter_example(64), W.single_loop(100), W.simple1(), W.simple2(), W.simple4(), W.simple5(),
                   W.greedy_bottom_up_bad(16, 100), W.greedy_top_down_bad(1000)]
 
