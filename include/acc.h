@@ -141,6 +141,11 @@ enum acc_status {
 
 #define ACC_MAX_INPUTS 6
 #define ACC_FLAG_FORCE_SLOT(s) (1u << (s)) /* the read of slot s goes through force() */
+/* SCANL / SCANR only.  The paper's scans (Section 2) have no seed and keep the length, which is
+ * read as inclusive.  With this flag the scan is seeded and exclusive: element k is the seed
+ * (fparam[0] for F32, iparam[0] otherwise) combined with the elements before k in scan order, so
+ * the first element is the seed itself and the last element of the source is left out. */
+#define ACC_FLAG_SCAN_EXCLUSIVE (1u << 16)
 
 typedef struct acc_node_desc {
   int32_t  kind;                 /* acc_kind                                             */
@@ -154,7 +159,7 @@ typedef struct acc_node_desc {
   int32_t  idx_fn_id;            /* acc_idx_fn (BACKPERMUTE only)                        */
   int64_t  iparam[4];
   double   fparam[4];
-  uint32_t flags;                /* ACC_FLAG_FORCE_SLOT(s)                               */
+  uint32_t flags;                /* ACC_FLAG_FORCE_SLOT(s), ACC_FLAG_SCAN_EXCLUSIVE      */
 } acc_node_desc;
 
 /* ---- building the graph (Section 4.1, "Data dependence graph") ------------- */

@@ -126,14 +126,19 @@ class _Cluster:
             order = range(inner) if nd.kind == "scanl" else range(inner - 1, -1, -1)
             vals = {}
             acc = None
+            excl = getattr(nd, "exclusive", False)
+            if excl:                                   # seeded: position t gets what was combined before it
+                acc = float(F32(nd.fparam[0])) if nd.dtype == "f32" else U32(int(nd.iparam[0]) & 0xFFFFFFFF)
             for t in order:
                 x = self.pull(src, row * inner + t)
+                if excl:
+                    vals[t] = F32(acc) if nd.dtype == "f32" else U32(acc)
                 if nd.dtype == "f32":
                     acc = float(x) if acc is None else float(fns.combine(nd.fn, F64(acc), F64(x)))
-                    vals[t] = F32(acc)
                 else:
                     acc = x if acc is None else self._icombine(nd, acc, x)
-                    vals[t] = U32(acc)
+                if not excl:
+                    vals[t] = F32(acc) if nd.dtype == "f32" else U32(acc)
             self.scan_cache[key] = vals
         return self.scan_cache[key][col]
 

@@ -10,6 +10,7 @@ combinator:
   backpermute  ys[j] = xs[f(j)]                    (== gather(generate(sz, f), xs))
   fold         reduce the innermost extent, no seed, rank one lower
   scanl/scanr  inclusive running combine along each innermost row, left/right
+               (exclusive=True: seeded with fparam[0] / iparam[0], element k leaves itself out)
   scatter      copy dest, then dest[i] = op(dest[i], x) for every (i, x) of src
                (Section 2's text has `f (src!i, x)`; the destructive-update
                sentence that follows fixes the reading dest[i] = f(dest[i], x))
@@ -186,6 +187,13 @@ def _foldseg(res, i, nd, src, offsets):
 def _scan(res, i, nd, src, right):
     op = nd.fn
     a = src[..., ::-1] if right else src
+    if getattr(nd, "exclusive", False):
+        # seeded and exclusive: element k combines the seed and the k elements before it, which is
+        # the inclusive scan of the row with the seed put in front and the last element dropped
+        seed = np.asarray(nd.fparam[0] if nd.dtype == "f32" else nd.iparam[0]).astype(F32 if nd.dtype == "f32" else np.int64)
+        seed = seed.astype(F32) if nd.dtype == "f32" else np.asarray(int(seed) & 0xFFFFFFFF, dtype=U32)
+        front = np.broadcast_to(seed, a.shape[:-1] + (1,)).astype(a.dtype)
+        a = np.concatenate([front, a[..., :-1]], axis=-1)
     if nd.dtype == "f32":
         a64 = a.astype(F64)
         ufunc = {"add": np.add, "mul": np.multiply, "min": np.minimum, "max": np.maximum}[op]

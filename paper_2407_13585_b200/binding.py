@@ -147,6 +147,8 @@ def make_desc(nd):
     flags = 0
     for s in getattr(nd, "force", ()):
         flags |= 1 << s
+    if getattr(nd, "exclusive", False):
+        flags |= 1 << 16                      # ACC_FLAG_SCAN_EXCLUSIVE
     d.flags = flags
     return d
 

@@ -22,8 +22,9 @@ constexpr int kMaxSlots = ACC_MAX_INPUTS;
 constexpr int kMaxCluster = 40;   // local nodes per cluster
 constexpr int kMaxProgram = 40;   // nodes per build-time program
 
-// Constants of a node that select code instead of being run-time arguments: so far the
-// row and column offsets of a clamped shift when both lie in -1..1 (kRunTime: not fixed).
+// Constants of a node that select code instead of being run-time arguments: the row and
+// column offsets of a clamped shift when both lie in -1..1 (kRunTime: not fixed), and
+// p0 = 1 for a seeded exclusive scan.
 constexpr int kRunTime = 9;
 
 struct PNode {                    // node of a build-time program

@@ -300,6 +300,7 @@ __global__ void __launch_bounds__(kBlock) k_scan(const __grid_constant__ Args<CL
   constexpr CNode sn = CL::c.nodes[S];
   constexpr int FN = sn.fn, DT = sn.dtype;
   constexpr bool REV = sn.kind == ACC_SCANR;
+  constexpr bool EXCL = sn.p0 == 1;                        // seeded and exclusive: element k leaves itself out
   using IX = std::conditional_t<VEC, std::conditional_t<REV, IxR4, Ix4>, Ix>;
 
   __shared__ uint32_t warp_total[kBlock / 32];
@@ -360,8 +361,15 @@ __global__ void __launch_bounds__(kBlock) k_scan(const __grid_constant__ Args<CL
       uint32_t excl = __shfl_up_sync(0xFFFFFFFFu, incl, 1);
       if (lane == 0) excl = identity_of<FN, DT>();
       excl = combine<FN, DT>(carry, excl);
+      if constexpr (EXCL) {
+        // what came before each element: the thread's own earlier elements on top of `excl`
 #pragma unroll
-      for (int e = 0; e < W; ++e) val[j][e] = combine<FN, DT>(excl, val[j][e]);
+        for (int e = W - 1; e >= 1; --e) val[j][e] = combine<FN, DT>(excl, val[j][e - 1]);
+        val[j][0] = excl;
+      } else {
+#pragma unroll
+        for (int e = 0; e < W; ++e) val[j][e] = combine<FN, DT>(excl, val[j][e]);
+      }
       carry = combine<FN, DT>(carry, __shfl_sync(0xFFFFFFFFu, incl, 31));
     }
     if (lane == 0) warp_total[warp] = carry;
@@ -409,7 +417,8 @@ __global__ void __launch_bounds__(kBlock) k_scan(const __grid_constant__ Args<CL
       if (lane == 0) tile_prefix = exclusive;
     }
     __syncthreads();
-    const uint32_t base = combine<FN, DT>(tile_prefix, offset);
+    uint32_t base = combine<FN, DT>(tile_prefix, offset);
+    if constexpr (EXCL) base = combine<FN, DT>(DT == ACC_F32 ? u_(a.n[S].fp0) : (uint32_t)a.n[S].ip0, base);   // the seed comes first
     uint32_t* out = reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[S].ptr));
 #pragma unroll
     for (int j = 0; j < ROWS; ++j) {

@@ -43,6 +43,7 @@ static bool extract_runtime(const Graph& g, const std::vector<int>& members, con
       n.p0 = (int)d.iparam[0];                         // kernels built for these very offsets are looked up first
       n.p1 = (int)d.iparam[1];
     }
+    if ((d.kind == ACC_SCANL || d.kind == ACC_SCANR) && (d.flags & ACC_FLAG_SCAN_EXCLUSIVE)) n.p0 = 1;   // other code, not another argument
     for (int s = 0; s < d.n_inputs; ++s) n.in[s] = local[d.inputs[s]];
     local[m] = c.n;
     c.source[c.n] = m;
@@ -122,7 +123,8 @@ int build_schedule(Graph& g, int executor, Schedule& sch) {
     std::string sig = signature(st.cc);
     st.kernel = find_kernel(sig);
     if (!st.kernel) {                                   // none for these constants: the one that takes them at run time
-      for (int li = 0; li < st.cc.n; ++li) st.cc.nodes[li].p0 = st.cc.nodes[li].p1 = kRunTime;
+      for (int li = 0; li < st.cc.n; ++li)
+        if (st.cc.nodes[li].kind == ACC_BACKPERMUTE) st.cc.nodes[li].p0 = st.cc.nodes[li].p1 = kRunTime;
       sig = signature(st.cc);
       st.kernel = find_kernel(sig);
     }

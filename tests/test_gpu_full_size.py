@@ -86,3 +86,16 @@ def test_config4_full_on_row_bands():
         ref = oracle_run(sub, {0: X[a:b].cpu().numpy()})
         want = ref.values[sub.outputs[0]][lo - a: hi - a]
         assert np.array_equal(Y[lo:hi].view(np.uint32), want.view(np.uint32)), (lo, hi)
+
+
+def test_greedy_bottom_up_bad_at_paper_scale():
+    # Section 5's program on which the bottom-up greedy goes wrong, at the size the paper names
+    # (m = 10^6 columns): under the best clustering the gathered n x m array and both folds share a
+    # kernel and the large array never exists; the bottom-up greedy clustering stores it (64 MB).
+    from paper_2407_13585_b200 import binding as B
+    prog = W.greedy_bottom_up_bad(16, 1000000)
+    got, inputs, pi, g = run_full(prog, "branch_bound")
+    assert pi == [-1, 0, 0, 0, 0, 1] and g.launch_count() == 2 and g.plan_info()[1]
+    assert g.partition_cost(pi, "bytes") < g.partition_cost(g.plan("greedy_bottomup", "bytes"), "bytes") / 1000
+    ref = oracle_run(prog, {k: v.cpu().numpy() for k, v in inputs.items()})
+    compare(prog, ref, got, "greedy_bottom_up_bad, m = 10^6")

@@ -301,3 +301,15 @@ def test_row_scans_both_directions(rows, cols):
 @pytest.mark.parametrize("n", [1, 6, 4096, 100001, 1 << 18])
 def test_right_to_left_scan_int32(n):
     check_program(W.suffix_sums(n))
+
+
+# seeded exclusive scans: an int32 running sum fed by a fused map (bit-exact), an fp32 sum from the right
+# and a per-row running maximum; one element, a fraction of a tile, tile boundaries, ragged tails
+@pytest.mark.parametrize("n", [1, 3, 4096, 4097, 70001, 1 << 18])
+def test_exclusive_seeded_scans(n):
+    assert check_program(W.exclusive_scans(n)) == 2
+
+
+@pytest.mark.parametrize("rows,cols", [(3, 10), (5, 4096), (2, 9000), (64, 301)])
+def test_exclusive_row_scans(rows, cols):
+    check_program(W.exclusive_row_scans(rows, cols))

@@ -93,6 +93,40 @@ def test_scans_worked():
     assert v[1].tolist() == [[1, 3, 6], [4, 9, 15]] and v[2].tolist() == [[6, 5, 3], [15, 11, 6]]
 
 
+def test_exclusive_seeded_scans_worked():
+    # exclusive, seeded: scanl(+, seed 0) [1,2,3,4] = [0,1,3,6]; seed 10 -> [10,11,13,16]; from the right
+    # [9,7,4,0]; element k is the seed combined with the inclusive scan's element before it, and the
+    # inclusive scan's last element is the exclusive one's last element combined with the last input
+    x = np.array([1, 2, 3, 4], I32)
+    nodes = [_inp("x", "i32", (4,)),
+             Node("scanl", "i32", (4,), (0,), 1, fn="add", iparam=(0,), exclusive=True),
+             Node("scanl", "i32", (4,), (0,), 1, fn="add", iparam=(10,), exclusive=True),
+             Node("scanr", "i32", (4,), (0,), 1, fn="add", iparam=(0,), exclusive=True),
+             Node("scanl", "i32", (4,), (0,), 1, fn="add")]
+    v = run(nodes, {0: x})
+    assert v[1].tolist() == [0, 1, 3, 6] and v[2].tolist() == [10, 11, 13, 16] and v[3].tolist() == [9, 7, 4, 0]
+    assert (v[1][1:] == v[4][:-1]).all() and int(v[1][-1]) + int(x[-1]) == int(v[4][-1])
+    # per row, another operator: the running maximum of what lies to the left, seeded with -1
+    nodes = [_inp("x", "f32", (2, 3)), Node("scanl", "f32", (2, 3), (0,), 1, fn="max", fparam=(-1.0,), exclusive=True)]
+    v = run(nodes, {0: np.array([[1, 5, 3], [-4, -5, 6]], F32)})
+    assert v[1].tolist() == [[-1, 1, 5], [-1, -1, -1]]
+    # a wrapping int32 sum, seeded at the top of the range
+    nodes = [_inp("x", "i32", (3,)), Node("scanl", "i32", (3,), (0,), 1, fn="add", iparam=(2**31 - 1,), exclusive=True)]
+    out = interp.to_external(run(nodes, {0: np.array([1, 1, 7], I32)})[1], "i32")
+    assert out.tolist() == [2**31 - 1, -2**31, -2**31 + 1]
+    # the loop a cluster denotes gives the same arrays, alone and with the map fused in
+    from oracle import cluster_loop, legality
+    p = W.exclusive_scans(50)
+    inputs = {k: t.numpy() for k, t in W.make_inputs(p).items()}
+    want = interp.run(p.nodes, inputs)
+    parts = legality.enumerate_partitions(p.nodes, p.outputs)
+    assert len(parts) == 2
+    for pi in parts:
+        got = cluster_loop.run(p.nodes, p.outputs, pi, inputs)
+        assert np.array_equal(got[3], want.values[3])
+        assert np.allclose(got[4], want.values[4], rtol=0, atol=1e-5 * np.abs(inputs[1]).sum())
+
+
 def test_scan_wraps_int32():
     nodes = [_inp("x", "i32", (2,)), Node("scanl", "i32", (2,), (0,), 1, fn="add")]
     out = interp.to_external(run(nodes, {0: np.array([2**31 - 1, 1], I32)})[1], "i32")

@@ -11,7 +11,7 @@ inputs, so every list is a DAG in topological order.  Slot layout by kind:
   gather       [idx, src]                      idx holds row-major linear indices
   permute      [defaults, idx, vals]           combine op named by fn
   fold         [src]                           reduces the innermost extent
-  scanl/scanr  [src]                           inclusive, per innermost row
+  scanl/scanr  [src]                           inclusive, per innermost row (exclusive=True: seeded, exclusive)
   foldseg      [src, offsets]                  n_array = 1; ys[s] = fold of src[offsets[s] .. offsets[s+1])
 
 Slots at positions >= n_array are "free variable" reads (element-level
@@ -34,6 +34,7 @@ class Node:
     iparam: Tuple[int, ...] = ()
     fparam: Tuple[float, ...] = ()
     force: Tuple[int, ...] = ()     # slots whose read is wrapped in force()
+    exclusive: bool = False         # scans: ys[i] combines the seed (fparam[0] / iparam[0]) and the elements before i
     name: str = ""
 
 
@@ -279,6 +280,29 @@ def suffix_sums(n=1 << 16):
         Node("scanr", "i32", (n,), (1,), 1, fn="add", name="suffix"),
     ]
     return Program("suffix_sums", nodes, [2])
+
+
+def exclusive_scans(n=1 << 16):
+    """Seeded exclusive scans: offsets from counts (wrapping int32 sum from the left of a masked array) and a
+    right-to-left exclusive fp32 sum."""
+    nodes = [
+        _inp("x", "i32", (n,)),
+        _inp("w", "f32", (n,)),
+        Node("map", "i32", (n,), (0,), 1, fn="and_mask", iparam=(0xFF,), name="counts"),
+        Node("scanl", "i32", (n,), (2,), 1, fn="add", iparam=(1000,), exclusive=True, name="offsets"),
+        Node("scanr", "f32", (n,), (1,), 1, fn="add", fparam=(0.5,), exclusive=True, name="after"),
+    ]
+    return Program("exclusive_scans", nodes, [3, 4])
+
+
+def exclusive_row_scans(rows=64, cols=300):
+    """Per row of a rank-2 array: the running maximum of everything to the left, seeded with -1."""
+    sh = (rows, cols)
+    nodes = [
+        _inp("x", "f32", sh),
+        Node("scanl", "f32", sh, (0,), 1, fn="max", fparam=(-1.0,), exclusive=True, name="best_before"),
+    ]
+    return Program("exclusive_row_scans", nodes, [1])
 
 
 CONFIGS = {1: config1, 2: config2, 3: config3, 4: config4, 5: config5}
