@@ -67,7 +67,8 @@ def measured_peak():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed steps, and the same steps repeated
+    right after them, run."""
     QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
@@ -251,14 +252,21 @@ def run_ours(args):
         for w in loads:
             w.run(B.FUSED)
 
+    sampler = ClockSampler(local) if rank == 0 else None     # nvidia-smi needs a few tenths of a second to start
     for _ in range(max(args.warmup, 3)):
         step()
     for w in loads:
         w.finish()
 
     barrier()
-    sampler = ClockSampler(local) if rank == 0 else None
     ms_step = time_region(step, args.steps)
+    if sampler:
+        # the timed region may be shorter than the sampler's start-up: keep the same load running
+        # (untimed) for half a second so that the clocks are read under it
+        t_end = time.perf_counter() + 0.5
+        while time.perf_counter() < t_end:
+            step()
+            torch.cuda.synchronize()
     clocks = sampler.stop() if sampler else {}
     barrier()
     launches = sum(w.g.launch_count() for w in loads)
