@@ -267,6 +267,20 @@ int acc_run(acc_graph* g, void* workspace, size_t workspace_bytes, void* cuda_st
 /* Waits for the stream and returns the device status of the last acc_run
  * (ACC_OK, ACC_ERR_DEVICE_TIMEOUT, ACC_ERR_INDEX_RANGE, ACC_ERR_CUDA). */
 int acc_finish(acc_graph* g, void* workspace, void* cuda_stream);
+/* acc_run followed by acc_finish, with a CUDA event before the first launch and
+ * after every cluster: ms_per_cluster_out[k] receives the device time of the
+ * k-th launch in execution order (up to `cap` entries), *n_out their number.
+ * For looking at where a program's time goes; the events cost a little, so time
+ * whole programs with acc_run. */
+int acc_run_timed(acc_graph* g, void* workspace, size_t workspace_bytes, void* cuda_stream, int executor,
+                  float* ms_per_cluster_out, int32_t cap, int32_t* n_out);
+/* Gather is defined for valid indices only (Section 2), and the kernels do not
+ * check them: an index outside the source reads memory that is not the
+ * caller's.  This call checks, on the device and without running the program,
+ * every GATHER whose index array is a program INPUT with a bound device buffer
+ * against the size of its source; it waits for the stream and returns ACC_OK or
+ * ACC_ERR_INDEX_RANGE.  `workspace` needs 256 bytes (the status word). */
+int acc_check_gather_indices(acc_graph* g, void* workspace, size_t workspace_bytes, void* cuda_stream);
 /* End to end with HOST buffers: copies every host-bound INPUT to its device
  * buffer, runs as acc_run, copies every host-bound output back, waits, and
  * returns as acc_finish.  h2d/d2h receive the bytes copied (may be null). */

@@ -98,6 +98,8 @@ def load_library(path=LIB_PATH):
         "acc_finish": (C.c_int, [p, p, p]),
         "acc_run_e2e": (C.c_int, [p, p, sz, p, C.c_int, C.POINTER(sz), C.POINTER(sz)]),
         "acc_run_e2e_async": (C.c_int, [p, p, sz, p, C.c_int, C.POINTER(sz), C.POINTER(sz)]),
+        "acc_run_timed": (C.c_int, [p, p, sz, p, C.c_int, C.POINTER(C.c_float), i32, pi32]),
+        "acc_check_gather_indices": (C.c_int, [p, p, sz, p]),
         "acc_launch_count": (i32, [p]),
         "acc_last_schedule": (C.c_int, [p, C.c_char_p, sz]),
         "acc_scanl_add_i32_static": (C.c_int, [p, p, i64, p]),
@@ -313,6 +315,19 @@ class Graph:
         fn = lib().acc_run_e2e if finish else lib().acc_run_e2e_async
         _check(fn(self._h, C.c_void_p(ws.data_ptr()), ws.numel(), self._stream(), executor, C.byref(up), C.byref(down)))
         return up.value, down.value
+
+    def run_timed(self, executor=FUSED):
+        """Runs and waits; returns the device time of every cluster launch in ms, in execution order."""
+        ws = self.ensure_workspace(executor)
+        ms = (C.c_float * 64)()
+        n = C.c_int32()
+        _check(lib().acc_run_timed(self._h, C.c_void_p(ws.data_ptr()), ws.numel(), self._stream(), executor, ms, 64, C.byref(n)))
+        return [ms[k] for k in range(min(n.value, 64))]
+
+    def check_gather_indices(self):
+        """Raises AccError(ACC_ERR_INDEX_RANGE) if an input index array of a gather points outside its source."""
+        ws = self.ensure_workspace(FUSED)
+        _check(lib().acc_check_gather_indices(self._h, C.c_void_p(ws.data_ptr()), ws.numel(), self._stream()))
 
     def launch_count(self):
         return lib().acc_launch_count(self._h)

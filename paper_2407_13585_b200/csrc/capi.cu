@@ -222,6 +222,37 @@ int acc_run(acc_graph* g, void* workspace, size_t workspace_bytes, void* cuda_st
   return run_schedule(*g, *sch, workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
 }
 
+int acc_run_timed(acc_graph* g, void* workspace, size_t workspace_bytes, void* cuda_stream, int executor,
+                  float* ms_out, int32_t cap, int32_t* n_out) {
+  clear_error();
+  if (!g) return set_error(ACC_ERR_ARG, "graph is null");
+  Schedule* sch = nullptr;
+  int rc = schedule_for(g, executor, &sch);
+  if (rc != ACC_OK) return rc;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  std::vector<cudaEvent_t> marks;
+  rc = run_schedule(*g, *sch, workspace, workspace_bytes, stream, &marks);
+  if (rc == ACC_OK) rc = finish(*g, workspace, stream);
+  if (rc == ACC_OK) {
+    const int n = (int)marks.size() - 1;
+    for (int k = 0; k < n && k < cap && ms_out; ++k) {
+      float ms = 0;
+      if (cudaEventElapsedTime(&ms, marks[k], marks[k + 1]) != cudaSuccess) ms = -1.0f;
+      ms_out[k] = ms;
+    }
+    if (n_out) *n_out = n < 0 ? 0 : n;
+  }
+  for (cudaEvent_t e : marks) cudaEventDestroy(e);
+  cudaGetLastError();
+  return rc;
+}
+
+int acc_check_gather_indices(acc_graph* g, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  clear_error();
+  if (!g) return set_error(ACC_ERR_ARG, "graph is null");
+  return check_gather_indices(*g, workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
 int acc_finish(acc_graph* g, void* workspace, void* cuda_stream) {
   clear_error();
   if (!g) return set_error(ACC_ERR_ARG, "graph is null");

@@ -154,7 +154,15 @@ static void* buffer_of(const Graph& g, const Schedule& sch, char* ws, int node) 
   return ws + sch.ctrl_bytes + sch.array_off[node];
 }
 
-int run_schedule(Graph& g, Schedule& sch, void* workspace, size_t ws_bytes, cudaStream_t stream) {
+static bool mark(std::vector<cudaEvent_t>* marks, cudaStream_t stream) {
+  if (!marks) return true;
+  cudaEvent_t e;
+  if (cudaEventCreate(&e) != cudaSuccess) return false;
+  marks->push_back(e);
+  return cudaEventRecord(e, stream) == cudaSuccess;
+}
+
+int run_schedule(Graph& g, Schedule& sch, void* workspace, size_t ws_bytes, cudaStream_t stream, std::vector<cudaEvent_t>* marks) {
   if (!workspace) return set_error(ACC_ERR_WORKSPACE, "workspace is null, %zu bytes needed", sch.total_bytes);
   if (reinterpret_cast<uintptr_t>(workspace) & 255) return set_error(ACC_ERR_WORKSPACE, "workspace is not 256-byte aligned");
   if (ws_bytes < sch.total_bytes) return set_error(ACC_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", ws_bytes, sch.total_bytes);
@@ -163,6 +171,7 @@ int run_schedule(Graph& g, Schedule& sch, void* workspace, size_t ws_bytes, cuda
     return set_error(ACC_ERR_CUDA, "clearing the control region failed: %s", cudaGetErrorString(cudaGetLastError()));
   g.launches = 0;
   g.schedule.clear();
+  if (!mark(marks, stream)) return set_error(ACC_ERR_CUDA, "recording an event failed: %s", cudaGetErrorString(cudaGetLastError()));
   for (ClusterStep& st : sch.steps) {
     for (int li = 0; li < st.cc.n; ++li) {
       const int node = st.cc.source[li];
@@ -177,12 +186,39 @@ int run_schedule(Graph& g, Schedule& sch, void* workspace, size_t ws_bytes, cuda
     st.launch.stream = stream;
     const int rc = st.kernel->launch(st.launch);
     if (rc != ACC_OK) return rc;
+    if (!mark(marks, stream)) return set_error(ACC_ERR_CUDA, "recording an event failed: %s", cudaGetErrorString(cudaGetLastError()));
     g.launches += 1;
     char item[48];
     snprintf(item, sizeof item, "%s%d:%d", g.schedule.empty() ? "" : " ", st.first_node, st.n_members);
     g.schedule += item;
   }
   return ACC_OK;
+}
+
+// One word per index: out of range (as unsigned, so negative ones too) sets the index bit of the status word.
+__global__ void k_index_range(const uint32_t* idx, int64_t n, uint32_t bound, uint32_t* status) {
+  bool bad = false;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) bad = bad || idx[i] >= bound;
+  if (__syncthreads_or(bad) && threadIdx.x == 0) atomicOr(status, 2u);
+}
+
+int check_gather_indices(Graph& g, void* workspace, size_t ws_bytes, cudaStream_t stream) {
+  if (!workspace || ws_bytes < 256 || (reinterpret_cast<uintptr_t>(workspace) & 255))
+    return set_error(ACC_ERR_WORKSPACE, "the check needs a 256-byte aligned workspace of 256 bytes");
+  if (cudaMemsetAsync(workspace, 0, 256, stream) != cudaSuccess)
+    return set_error(ACC_ERR_CUDA, "clearing the status word failed: %s", cudaGetErrorString(cudaGetLastError()));
+  for (const Node& nd : g.nodes) {
+    if (nd.d.kind != ACC_GATHER) continue;
+    const Node& idx = g.nodes[nd.d.inputs[0]];
+    const Node& src = g.nodes[nd.d.inputs[1]];
+    if (!is_input(idx) || !idx.dev || idx.count == 0) continue;
+    const uint32_t bound = (uint32_t)std::min<int64_t>(src.count, 0x7FFFFFFF);
+    const int grid = (int)std::min<int64_t>((idx.count + 255) / 256, (int64_t)sm_count() * 8);
+    k_index_range<<<grid, 256, 0, stream>>>(static_cast<const uint32_t*>(idx.dev), idx.count, bound, static_cast<uint32_t*>(workspace));
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return set_error(ACC_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+  }
+  return finish(g, workspace, stream);
 }
 
 int finish(Graph& g, void* workspace, cudaStream_t stream) {
@@ -193,7 +229,7 @@ int finish(Graph& g, void* workspace, cudaStream_t stream) {
   if (e != cudaSuccess) return set_error(ACC_ERR_CUDA, "stream failed: %s", cudaGetErrorString(e));
   g.host_status = status;
   if (status & 1u) return set_error(ACC_ERR_DEVICE_TIMEOUT, "a device-side wait ran out of iterations");
-  if (status & 2u) return set_error(ACC_ERR_INDEX_RANGE, "a scatter index or a segment offset fell outside its array");
+  if (status & 2u) return set_error(ACC_ERR_INDEX_RANGE, "a scatter index, a segment offset or a checked gather index fell outside its array");
   if (status & 4u) return set_error(ACC_ERR_SHAPE, "an empty segment has no value: segment offsets must increase");
   return ACC_OK;
 }

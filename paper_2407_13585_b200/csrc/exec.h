@@ -28,7 +28,10 @@ struct Schedule {
 };
 
 int build_schedule(Graph& g, int executor, Schedule& sch);
-int run_schedule(Graph& g, Schedule& sch, void* workspace, size_t ws_bytes, cudaStream_t stream);
+// `marks`, if given, receives one recorded event before the first launch and one after each launch
+int run_schedule(Graph& g, Schedule& sch, void* workspace, size_t ws_bytes, cudaStream_t stream,
+                 std::vector<cudaEvent_t>* marks = nullptr);
+int check_gather_indices(Graph& g, void* workspace, size_t ws_bytes, cudaStream_t stream);
 int finish(Graph& g, void* workspace, cudaStream_t stream);
 
 }  // namespace acc

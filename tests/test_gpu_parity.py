@@ -313,3 +313,31 @@ def test_exclusive_seeded_scans(n):
 @pytest.mark.parametrize("rows,cols", [(3, 10), (5, 4096), (2, 9000), (64, 301)])
 def test_exclusive_row_scans(rows, cols):
     check_program(W.exclusive_row_scans(rows, cols))
+
+
+def test_gather_indices_are_checked_on_request_and_clusters_are_timed():
+    import torch
+    from paper_2407_13585_b200 import binding as B
+    prog = W.config3(1 << 16)
+    inputs = W.make_inputs(prog)
+    g = B.Graph(prog.nodes, prog.outputs)
+    g.set_partition([-1, -1, 0, 1, 1, 1])
+    dev = {i: t.cuda() for i, t in inputs.items()}
+    for i, t in dev.items():
+        g.bind(i, t)
+    out = torch.empty(1 << 16, dtype=torch.int32, device="cuda")
+    g.bind(prog.outputs[0], out)
+    g.check_gather_indices()                               # every index below 2^16
+    ms = g.run_timed(B.FUSED)
+    assert len(ms) == 2 and all(0.0 < t < 50.0 for t in ms) and g.launch_count() == 2
+    ref = oracle_run(prog, np_inputs(inputs))
+    assert np.array_equal(out.cpu().numpy().view(np.uint32), ref.values[prog.outputs[0]])
+    # one index just past the end, one negative: reported by the check (the program is not run on them)
+    idx = [i for i in prog.input_ids() if prog.nodes[i].name == "idx"][0]
+    for bad in (1 << 16, -1):
+        dev[idx][12345] = bad
+        with pytest.raises(B.AccError) as err:
+            g.check_gather_indices()
+        assert err.value.status == "ACC_ERR_INDEX_RANGE"
+    dev[idx][12345] = 7
+    g.check_gather_indices()
