@@ -245,6 +245,21 @@ int64_t acc_enumerate_recompute(acc_graph* g, int32_t max_depth, int32_t* out_pi
 int acc_partition_cost_recompute(acc_graph* g, const int32_t* cluster_of_node, int32_t n_nodes, int32_t max_depth, int cost,
                                  double* out);
 
+/* A clustering in which some nodes are evaluated in several clusters: besides
+ * cluster_of_node (each node's own cluster), n_copies pairs (copy_node[k],
+ * copy_cluster[k]) put a copy of a node into a further cluster.  Every reader of
+ * the node that lies in such a cluster reads the copy (fused, recomputed there)
+ * instead of the stored array; the copy itself reads, input by input, what its
+ * cluster holds of the input (the input's own node or its copy there) and
+ * otherwise the stored array.  A copy must be fused away: it is an error if it
+ * has no reader in its cluster or would have to be stored.  The clustering with
+ * the copies written out as nodes is checked like any other (max_depth as
+ * above; 0: the paper's rules).  acc_get_partition and acc_manifest keep
+ * speaking of the original nodes.  Example: the total of the histogram program
+ * can regenerate `vals` in its own kernel instead of reading them from memory. */
+int acc_set_partition_copies(acc_graph* g, const int32_t* cluster_of_node, int32_t n_nodes, const int32_t* copy_node,
+                             const int32_t* copy_cluster, int32_t n_copies, int32_t max_depth);
+
 /* ---- running ------------------------------------------------------------------ */
 
 /* Binds a caller-owned DEVICE buffer to a node.  Required for INPUT nodes and

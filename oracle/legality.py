@@ -379,3 +379,50 @@ def traffic(nodes, outputs, pi, weight=lambda nd: 1):
     r = sum(weight(nodes[a]) for a, _, _ in reads)
     w = sum(weight(nodes[a]) for a in man if nodes[a].kind != "input")
     return r, w
+
+
+def unfold_copies(nodes, outputs, pi, copies):
+    """A clustering with copies, written out: (nodes2, outputs2, pi2, home, copy_ids).
+
+    `copies` are (node, cluster) pairs: readers of the node inside that cluster read a copy that
+    is evaluated there.  Every copy becomes a node of its own right after the node it copies; a
+    node instance in cluster c reads, input by input, the instance of the input that lives in c
+    (the input itself or its copy there), else the input itself.  home[i] is where node i went.
+    """
+    import copy as _copy
+    nodes2, pi2, home, copy_ids = [], [], {}, {}
+
+    def instance(x, cluster):
+        if nodes[x].kind != "input" and pi[x] != cluster and (x, cluster) in copy_ids:
+            return copy_ids[(x, cluster)]
+        return home[x]
+
+    for i, nd in enumerate(nodes):
+        places = [None] + [c for a, c in copies if a == i]
+        for c in places:
+            cluster = (-1 if nd.kind == "input" else pi[i]) if c is None else c
+            m = _copy.copy(nd)
+            m.inputs = tuple(instance(x, cluster) for x in nd.inputs)
+            nodes2.append(m)
+            pi2.append(cluster)
+            if c is None:
+                home[i] = len(nodes2) - 1
+            else:
+                copy_ids[(i, c)] = len(nodes2) - 1
+    return nodes2, [home[o] for o in outputs], pi2, home, copy_ids
+
+
+def check_with_copies(nodes, outputs, pi, copies, recompute=0):
+    """Legality of a clustering with copies: the written-out clustering is legal and no copy is stored."""
+    for a, c in copies:
+        if nodes[a].kind == "input" or c == pi[a] or copies.count((a, c)) > 1:
+            return False, "bad copy"
+    nodes2, outputs2, pi2, home, copy_ids = unfold_copies(nodes, outputs, pi, copies)
+    ok, why = check(nodes2, outputs2, pi2, recompute)
+    if not ok:
+        return False, why
+    man = manifest_set(nodes2, outputs2, pi2, edges_of(nodes2))
+    for key, j in copy_ids.items():
+        if j in man:
+            return False, f"the copy of node {key[0]} in cluster {key[1]} would be stored"
+    return True, ""

@@ -91,6 +91,7 @@ def load_library(path=LIB_PATH):
         "acc_enumerate_recompute": (i64, [p, i32, pi32, i64]),
         "acc_partition_cost_recompute": (C.c_int, [p, pi32, i32, i32, C.c_int, C.POINTER(C.c_double)]),
         "acc_plan_info": (C.c_int, [p, C.POINTER(i64), C.POINTER(i32)]),
+        "acc_set_partition_copies": (C.c_int, [p, pi32, i32, pi32, pi32, i32, i32]),
         "acc_bind": (C.c_int, [p, i32, p, sz]),
         "acc_bind_host": (C.c_int, [p, i32, p, sz]),
         "acc_workspace_bytes": (C.c_int, [p, C.c_int, C.POINTER(sz)]),
@@ -235,6 +236,12 @@ class Graph:
         out = C.c_double()
         _check(lib().acc_partition_cost_recompute(self._h, _i32_array(pi), len(pi), max_depth, COST[cost], C.byref(out)))
         return out.value
+
+    def set_partition_copies(self, pi, copies, max_depth=0):
+        """copies: (node, cluster) pairs; readers of the node in that cluster read a copy recomputed there."""
+        nodes = _i32_array([a for a, _ in copies])
+        clusters = _i32_array([c for _, c in copies])
+        _check(lib().acc_set_partition_copies(self._h, _i32_array(pi), len(pi), nodes, clusters, len(copies), max_depth))
 
     def get_partition(self):
         out = (C.c_int32 * self.n)()

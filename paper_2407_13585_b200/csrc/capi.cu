@@ -21,13 +21,29 @@ std::map<const acc_graph*, std::unique_ptr<Cache[]>>& caches() {
   return c;
 }
 
+// The graph a run works on: the caller's, or, for the fused executor under a clustering with
+// copies, the graph in which the copies are nodes (buffers and output marks carried over).
+Graph& run_target(acc_graph* g, int executor) {
+  if (executor != ACC_EXEC_FUSED || !g->unfolded) return *g;
+  Graph& u = *g->unfolded;
+  for (size_t i = 0; i < g->nodes.size(); ++i) {
+    Node& to = u.nodes[g->home_in_unfolded[i]];
+    const Node& from = g->nodes[i];
+    to.dev = from.dev;
+    to.dev_bytes = from.dev_bytes;
+    to.host = from.host;
+    to.host_bytes = from.host_bytes;
+  }
+  return u;
+}
+
 int schedule_for(acc_graph* g, int executor, Schedule** out) {
   if (executor != ACC_EXEC_FUSED && executor != ACC_EXEC_UNFUSED) return set_error(ACC_ERR_ARG, "unknown executor %d", executor);
   auto& slot = caches()[g];
   if (!slot) slot.reset(new Cache[2]);
   Cache& c = slot[executor];
   if (c.serial != g->run_serial) {
-    const int rc = build_schedule(*g, executor, c.sch);
+    const int rc = build_schedule(run_target(g, executor), executor, c.sch);
     if (rc != ACC_OK) return rc;
     c.serial = g->run_serial;
   }
@@ -60,6 +76,7 @@ acc_node acc_add_node(acc_graph* g, const acc_node_desc* d) {
   clear_error();
   if (!g || !d) return set_error(ACC_ERR_ARG, "null argument");
   g->run_serial++;
+  g->unfolded.reset();
   return add_node(*g, *d);
 }
 
@@ -69,6 +86,7 @@ int acc_mark_output(acc_graph* g, acc_node n) {
   if (is_input(g->nodes[n])) return set_error(ACC_ERR_ARG, "an input cannot be an output");
   g->nodes[n].output = true;
   g->has_pi = false;
+  g->unfolded.reset();
   g->run_serial++;
   return ACC_OK;
 }
@@ -111,11 +129,77 @@ int acc_set_partition_recompute(acc_graph* g, const int32_t* pi, int32_t n_nodes
   manifest_of(*g, g->pi.data(), g->manifest);
   g->has_pi = true;
   g->recompute_depth = max_depth;
+  g->unfolded.reset();
   g->run_serial++;
   return ACC_OK;
 }
 
 int acc_set_partition(acc_graph* g, const int32_t* pi, int32_t n_nodes) { return acc_set_partition_recompute(g, pi, n_nodes, 0); }
+
+int acc_set_partition_copies(acc_graph* g, const int32_t* pi, int32_t n_nodes, const int32_t* copy_node, const int32_t* copy_cluster,
+                             int32_t n_copies, int32_t max_depth) {
+  clear_error();
+  if (!g || !pi || n_copies < 0 || (n_copies > 0 && (!copy_node || !copy_cluster))) return set_error(ACC_ERR_ARG, "null argument");
+  if (max_depth < 0) return set_error(ACC_ERR_ARG, "max_depth %d is negative", max_depth);
+  const int n = (int)g->nodes.size();
+  if (n_nodes != n) return set_error(ACC_ERR_ARG, "clustering has %d entries, graph has %d nodes", n_nodes, n);
+  for (int i = 0; i < n; ++i)
+    if (!is_input(g->nodes[i]) && (pi[i] < 0 || pi[i] > n)) return set_error(ACC_ERR_ARG, "cluster number %d of node %d outside 0..n", pi[i], i);
+  for (int k = 0; k < n_copies; ++k) {
+    const int a = copy_node[k], c = copy_cluster[k];
+    if (a < 0 || a >= n || is_input(g->nodes[a])) return set_error(ACC_ERR_ARG, "copy %d: node %d cannot be copied", k, a);
+    if (c < 0 || c > n || c == pi[a]) return set_error(ACC_ERR_ARG, "copy %d: cluster %d is node %d's own or outside 0..n", k, c, a);
+    for (int j = 0; j < k; ++j)
+      if (copy_node[j] == a && copy_cluster[j] == c) return set_error(ACC_ERR_ARG, "copy %d repeats copy %d", k, j);
+  }
+  // the graph with every copy as a node, right after the node it copies (so inputs still come first)
+  auto u = std::make_shared<Graph>();
+  std::vector<int> home(n, -1);
+  std::vector<int32_t> upi;
+  std::vector<int> copy_id(n_copies, -1);
+  auto instance = [&](int x, int cluster) {            // what a reader in `cluster` reads of node x
+    if (!is_input(g->nodes[x]) && pi[x] != cluster)
+      for (int k = 0; k < n_copies; ++k)
+        if (copy_node[k] == x && copy_cluster[k] == cluster) return copy_id[k];
+    return home[x];
+  };
+  for (int i = 0; i < n; ++i) {
+    for (int k = -1; k < n_copies; ++k) {
+      if (k >= 0 && copy_node[k] != i) continue;
+      const int cluster = k < 0 ? (is_input(g->nodes[i]) ? -1 : pi[i]) : copy_cluster[k];
+      acc_node_desc d = g->nodes[i].d;
+      for (int s = 0; s < d.n_inputs; ++s) d.inputs[s] = instance(d.inputs[s], cluster);
+      const int id = add_node(*u, d);
+      if (id < 0) return id;
+      upi.push_back(cluster);
+      if (k < 0) { home[i] = id; u->nodes[id].output = g->nodes[i].output; }
+      else copy_id[k] = id;
+    }
+  }
+  const int rc = check_partition(*u, upi.data(), nullptr, false, max_depth);
+  if (rc != ACC_OK) return rc;
+  std::vector<uint8_t> uman;
+  manifest_of(*u, upi.data(), uman);
+  for (int k = 0; k < n_copies; ++k)
+    if (uman[copy_id[k]])
+      return set_error(ACC_ERR_ARG, "the copy of node %d in cluster %d has no reader there or would have to be stored", copy_node[k], copy_cluster[k]);
+  u->pi = upi;
+  u->manifest = uman;
+  u->has_pi = true;
+  u->recompute_depth = max_depth;
+  g->pi.assign(pi, pi + n);
+  g->manifest.assign(n, 0);
+  for (int i = 0; i < n; ++i) {
+    if (is_input(g->nodes[i])) g->pi[i] = -1;
+    g->manifest[i] = uman[home[i]];
+  }
+  g->has_pi = true;
+  g->recompute_depth = max_depth;
+  g->unfolded = u;
+  g->home_in_unfolded = home;
+  g->run_serial++;
+  return ACC_OK;
+}
 
 int acc_get_partition(const acc_graph* g, int32_t* out, int32_t n_nodes) {
   clear_error();
@@ -217,9 +301,13 @@ int acc_run(acc_graph* g, void* workspace, size_t workspace_bytes, void* cuda_st
   clear_error();
   if (!g) return set_error(ACC_ERR_ARG, "graph is null");
   Schedule* sch = nullptr;
-  const int rc = schedule_for(g, executor, &sch);
+  int rc = schedule_for(g, executor, &sch);
   if (rc != ACC_OK) return rc;
-  return run_schedule(*g, *sch, workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+  Graph& target = run_target(g, executor);
+  rc = run_schedule(target, *sch, workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+  g->launches = target.launches;
+  g->schedule = target.schedule;
+  return rc;
 }
 
 int acc_run_timed(acc_graph* g, void* workspace, size_t workspace_bytes, void* cuda_stream, int executor,
@@ -231,7 +319,10 @@ int acc_run_timed(acc_graph* g, void* workspace, size_t workspace_bytes, void* c
   if (rc != ACC_OK) return rc;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   std::vector<cudaEvent_t> marks;
-  rc = run_schedule(*g, *sch, workspace, workspace_bytes, stream, &marks);
+  Graph& target = run_target(g, executor);
+  rc = run_schedule(target, *sch, workspace, workspace_bytes, stream, &marks);
+  g->launches = target.launches;
+  g->schedule = target.schedule;
   if (rc == ACC_OK) rc = finish(*g, workspace, stream);
   if (rc == ACC_OK) {
     const int n = (int)marks.size() - 1;

@@ -3,6 +3,7 @@
 #pragma once
 #include <cstdarg>
 #include <cstdint>
+#include <memory>
 #include <string>
 #include <vector>
 
@@ -33,6 +34,11 @@ struct Graph {
   std::vector<int32_t> pi;         // stored clustering, -1 for inputs
   bool has_pi = false;
   int recompute_depth = 0;         // the rules the stored clustering was checked under
+  // A clustering with nodes copied into further clusters is run on a graph of its own in which
+  // every copy is a node: `unfolded` (its own clustering stored in it), and where each node of
+  // this graph went (`home_in_unfolded`).  Null for every other clustering.
+  std::shared_ptr<Graph> unfolded;
+  std::vector<int> home_in_unfolded;
   std::vector<uint8_t> manifest;   // under the stored clustering
   // bookkeeping of the last run
   int64_t plan_visited = 0;        // partial clusterings the last planner call looked at

@@ -18,4 +18,7 @@ ACC_CLUSTER(kHistogram, 0x1C, hist_k_vals_hist)
 ACC_CLUSTER(kHistogram, 0x34, hist_k_hist_total)
 ACC_CLUSTER(kHistogram, 0x38, hist_vals_hist_total)
 ACC_CLUSTER(kHistogram, 0x3C, hist_all)
+// with a copy of `vals` in the cluster of `total`
+ACC_CLUSTER(programs::kHistogramScatterOnly, 0x1C, hist_k_vals_hist_private)
+ACC_CLUSTER(programs::kGeneratedTotal, 0x3, hist_vals_copy_total)
 }  // namespace acc

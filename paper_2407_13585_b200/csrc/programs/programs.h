@@ -90,12 +90,33 @@ constexpr CProgram histogram_diamond() {
   return p;
 }
 
+// The histogram program when `total` regenerates `vals` in a kernel of its own (a clustering with a
+// copy of `vals`): the scatter's cluster, in which `vals` now has no outside reader, and the copy
+// with the fold.
+constexpr CProgram histogram_scatter_only() {
+  CProgram p{5, 1ull << 4, {}};
+  p.nodes[0] = input(ACC_U32, 1);
+  p.nodes[1] = input(ACC_F32, 1);
+  p.nodes[2] = pnode(ACC_MAP, ACC_U32, 1, ACC_FN_MUL_MOD, 0, 1, 0);
+  p.nodes[3] = pnode(ACC_GENERATE, ACC_F32, 1, ACC_FN_IMOD_TO_F32, 0, 0);
+  p.nodes[4] = pnode(ACC_PERMUTE, ACC_F32, 1, ACC_FN_ADD, 0, 3, 1, 2, 3);
+  return p;
+}
+constexpr CProgram generated_total() {
+  CProgram p{2, 1ull << 1, {}};
+  p.nodes[0] = pnode(ACC_GENERATE, ACC_F32, 1, ACC_FN_IMOD_TO_F32, 0, 0);
+  p.nodes[1] = pnode(ACC_FOLD, ACC_F32, 0, ACC_FN_ADD, 0, 1, 0);
+  return p;
+}
+
 inline constexpr CProgram kChain1d = chain1d();
 inline constexpr CProgram kTransposeReduce = transpose_reduce();
 inline constexpr CProgram kGatherScan = gather_scan();
 inline constexpr CProgram kJacobi = jacobi_iteration();
 inline constexpr CProgram kJacobiChain = jacobi_chain(4);
 inline constexpr CProgram kHistogram = histogram_diamond();
+inline constexpr CProgram kHistogramScatterOnly = histogram_scatter_only();
+inline constexpr CProgram kGeneratedTotal = generated_total();
 
 }  // namespace programs
 }  // namespace acc

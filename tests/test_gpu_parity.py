@@ -341,3 +341,34 @@ def test_gather_indices_are_checked_on_request_and_clusters_are_timed():
         assert err.value.status == "ACC_ERR_INDEX_RANGE"
     dev[idx][12345] = 7
     g.check_gather_indices()
+
+
+@pytest.mark.parametrize("n,bins", [(1 << 12, 64), (100003, 1000), (1 << 20, 1 << 12)])
+def test_histogram_total_regenerates_vals_in_its_own_kernel(n, bins):
+    # a clustering with a copy: {k, vals, hist} | {vals', total} | {frac}: three kernels, vals never stored
+    import torch
+    from paper_2407_13585_b200 import binding as B
+    prog = W.config5(n, bins)
+    inputs_t = W.make_inputs(prog)
+    ref = oracle_run(prog, np_inputs(inputs_t))
+    g = B.Graph(prog.nodes, prog.outputs)
+    g.set_partition_copies([-1, -1, 0, 0, 0, 1, 2], [(3, 1)])
+    assert not g.manifest()[3]
+    bufs = {}
+    for i, nd in enumerate(prog.nodes):
+        if nd.kind == "input":
+            bufs[i] = inputs_t[i].cuda()
+            g.bind(i, bufs[i])
+        elif i in prog.outputs:
+            cnt = int(np.prod(nd.shape, dtype=np.int64)) if nd.shape else 1
+            bufs[i] = torch.full((max(cnt, 4),), -1, dtype=torch.int32, device="cuda")
+            g.bind(i, bufs[i])
+    g.run(B.FUSED)
+    g.run(B.FUSED)
+    assert g.launch_count() == 3
+    got = {}
+    for o in prog.outputs:
+        nd = prog.nodes[o]
+        cnt = int(np.prod(nd.shape, dtype=np.int64)) if nd.shape else 1
+        got[o] = bufs[o][:cnt].cpu().numpy().view(np.float32).reshape(tuple(nd.shape))
+    compare(prog, ref, got, "config5 with a copy of vals")

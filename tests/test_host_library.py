@@ -204,6 +204,36 @@ def test_branch_and_bound_proves_the_jacobi_chain():
     assert pi == [-1] + [0] * 18 + [1] * 18
 
 
+def test_clusterings_with_copies_equal_oracle():
+    # every single copy (node, cluster) on top of every legal clustering, and some pairs of copies, of three programs
+    progs = [W.config5(64, 8), W.config1(16), W.simple5()]
+    agreed = accepted = 0
+    for p in progs:
+        g = B.Graph(p.nodes, p.outputs)
+        ops = [i for i, nd in enumerate(p.nodes) if nd.kind != "input"]
+        for pi in L.enumerate_partitions(p.nodes, p.outputs):
+            clusters = sorted({c for c in pi if c >= 0})
+            singles = [(a, c) for a in ops + [0] for c in clusters]
+            for copies in [[s] for s in singles] + [[singles[i], singles[j]] for i in range(0, len(singles), 3) for j in range(i + 1, len(singles), 4)]:
+                want = L.check_with_copies(p.nodes, p.outputs, pi, copies)[0]
+                try:
+                    g.set_partition_copies(pi, copies)
+                    got = True
+                except B.AccError:
+                    got = False
+                assert got == want, (p.name, pi, copies)
+                agreed += 1
+                accepted += want
+    assert agreed > 300 and accepted >= 5
+    # the accepted one of the histogram program: vals is no longer stored
+    p = progs[0]
+    g = B.Graph(p.nodes, p.outputs)
+    g.set_partition_copies([-1, -1, 0, 0, 0, 1, 2], [(3, 1)])
+    assert g.manifest() == [True, True, False, False, True, True, True] and g.get_partition() == [-1, -1, 0, 0, 0, 1, 2]
+    g.set_partition([-1, -1, 0, 0, 0, 1, 2])
+    assert g.manifest()[3]
+
+
 def test_check_partition_names_the_broken_rule():
     p = W.scatter_example_paper_graph()
     g = B.Graph(p.nodes, p.outputs)

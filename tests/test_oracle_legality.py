@@ -288,3 +288,31 @@ def test_recomputing_clusters_compute_the_same_arrays():
     want = interp.run(p.nodes, {0: x}).values[p.outputs[0]]
     got = cluster_loop.run(p.nodes, p.outputs, [-1] + [0] * 18, {0: x})
     assert np.array_equal(got[p.outputs[0]].view(np.uint32), want.view(np.uint32))
+
+
+# ---- nodes copied into further clusters ----
+
+def test_a_copy_lets_the_total_regenerate_its_values():
+    import numpy as np
+    from oracle import cluster_loop, interp
+    p = W.config5(64, 8)                                    # keys, zeros, k, vals, hist, total, frac
+    pi = [-1, -1, 0, 0, 0, 1, 2]
+    # without the copy, `vals` (3) is stored for `total`; with a copy of it in cluster 1 nothing reads the stored one
+    nodes2, outputs2, pi2, home, copy_ids = L.unfold_copies(p.nodes, p.outputs, pi, [(3, 1)])
+    assert len(nodes2) == len(p.nodes) + 1 and pi2[copy_ids[(3, 1)]] == 1
+    assert nodes2[home[5]].inputs == (copy_ids[(3, 1)],) and nodes2[home[4]].inputs[2] == home[3]
+    assert L.check_with_copies(p.nodes, p.outputs, pi, [(3, 1)])[0]
+    edges = L.edges_of(nodes2)
+    assert home[3] not in L.manifest_set(nodes2, outputs2, pi2, edges)
+    assert 3 in L.manifest_set(p.nodes, p.outputs, pi, L.edges_of(p.nodes))
+    # the arrays are those of the program itself
+    inputs = {k: t.numpy() for k, t in W.make_inputs(p).items()}
+    want = interp.run(p.nodes, inputs)
+    got = cluster_loop.run(nodes2, outputs2, pi2, {home[k]: v for k, v in inputs.items()})
+    for o in p.outputs:
+        assert np.allclose(got[home[o]], want.values[o], rtol=1e-6, atol=0)
+    # what a copy cannot be: of an input, in the node's own cluster, without a reader, or a scatter's result
+    assert not L.check_with_copies(p.nodes, p.outputs, pi, [(0, 1)])[0]
+    assert not L.check_with_copies(p.nodes, p.outputs, pi, [(3, 0)])[0]
+    assert not L.check_with_copies(p.nodes, p.outputs, pi, [(3, 2)])[0]          # nobody in cluster 2 reads vals
+    assert not L.check_with_copies(p.nodes, p.outputs, pi, [(4, 2)])[0]          # frac reads hist through an infusible edge: not inside one cluster
