@@ -82,6 +82,13 @@ __device__ __forceinline__ void red_add_global(double* p, double v) {
   asm volatile("red.global.add.f64 [%0], %1;" ::"l"(p), "d"(v) : "memory");
 }
 
+// Whether member I can only take integer values in [0, iparam[0]), known from its function alone
+// (then a scatter of it needs no per-value test of what the integer bins can hold).
+template <class CL> constexpr bool yields_small_integers(int i) {
+  const CNode& n = CL::c.nodes[i];
+  return n.member && n.kind == ACC_GENERATE && n.dtype == ACC_F32 && n.fn == ACC_FN_IMOD_TO_F32;
+}
+
 template <class CL> constexpr int the_f32_add_permute() {
   for (int i = 0; i < CL::c.n; ++i)
     if (is_f32_add_permute(CL::c.nodes[i])) return i;
@@ -154,11 +161,14 @@ k_hist(const __grid_constant__ Args<CL::c.n> a, const HistPlan plan, int* overfl
   // a bin receives at most `mine` addends of magnitude < cap each: |sum| < 2^31
   const uint32_t mine = ((total + n_teams - 1) / n_teams + 1) * W;
   const int cap_log2 = min(30 - (32 - __clz(mine)), 22);      // 2^cap_log2 * mine < 2^30
+  constexpr bool INTS = yields_small_integers<CL>(pn.in[2]);
+  // values known to be integers below m: m - 1 is the magnitude to scale for, whatever the sample says
+  const float largest = INTS ? (float)max(a.n[pn.in[2]].ip0 - 1, 0) : sample_max;
   int S = 0;
-  if (sample_max > 0.0f) {
+  if (largest > 0.0f) {
     int e;
-    frexpf(sample_max, &e);                                    // sample_max = f * 2^e, f in [0.5, 1)
-    S = min(max(cap_log2 - 1 - e, -100), 100);                 // sample_max * 2^S < cap / 2
+    frexpf(largest, &e);                                       // largest = f * 2^e, f in [0.5, 1)
+    S = min(max(cap_log2 - 1 - e, -100), 100);                 // largest * 2^S < cap / 2
   }
   const float cap = exp2f((float)cap_log2);
   const float up = exp2f((float)S);
@@ -249,6 +259,17 @@ k_hist(const __grid_constant__ Args<CL::c.n> a, const HistPlan plan, int* overfl
         // all four values exact integers below `cap` after scaling.  (With up >= 1 a non-zero x
         // cannot underflow to a zero product; otherwise the careful path below is taken.)
         const uint32_t kmax = max(max(key[u].v[0], key[u].v[1]), max(key[u].v[2], key[u].v[3]));
+        if constexpr (INTS) {
+          // integers below m, and (m - 1) * 2^S below cap / 2 by the choice of S: every product is an
+          // exact integer the bins can take, so only the indices are looked at
+          if (fast_ok & (kmax < n_bins)) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              red_add_bin(key[u].v[j], (uint32_t)per_cta, bins_addr, spill - per_cta,
+                          __float_as_int(__fadd_rn(__fmul_rn(f_(val[u].v[j]), up), 12582912.0f)) - 0x4B400000);
+            continue;
+          }
+        }
         float t[4], shifted[4], off = 0.0f, big = 0.0f;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
