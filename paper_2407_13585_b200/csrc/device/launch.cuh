@@ -173,11 +173,11 @@ struct Launcher {
       dev::TileMaps maps;
       for (int i = 0; i < N; ++i)
         if (dev::is_staged_external<CL>(i) &&
-            !make_tensor_map_2d(&maps.m[dev::tile_slot<CL>(i)], L.nodes[i].ptr, n, n, dev::kTile, dev::kTpBoxCols, true))
+            !make_tensor_map_2d(&maps.m[dev::tile_slot<CL>(i)], L.nodes[i].ptr, n, n, dev::kTile, dev::kTile))
           return 1;
       auto kern = dev::k_tile_pair_tma<CL>;
       constexpr int E = dev::staged_externals<CL>();
-      const size_t smem = (size_t)dev::tp_stages<E>() * E * dev::kTpSlotWords * 4 + 1024;   // + room to align to the swizzle
+      const size_t smem = (size_t)dev::tp_stages<E>() * E * dev::kTpSlotWords * 4 + 128;   // + room to align the copies
       static int fit_on[64];                               // blocks of this kernel per SM, + 1, by device (asked once each)
       int device = 0;
       if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) { cudaGetLastError(); return 1; }

@@ -57,7 +57,7 @@ using EncodeTiled = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, 
 // Describes a row-major rows x cols array of 4-byte elements for copies of box_rows x box_cols
 // boxes (out-of-range parts of a box read as zero).  `out` points to a CUtensorMap.
 // The driver entry point is looked up through the runtime, so libcuda is not linked.
-bool make_tensor_map_2d(void* out, const void* base, int rows, int cols, int box_rows, int box_cols, bool swizzle_128b) {
+bool make_tensor_map_2d(void* out, const void* base, int rows, int cols, int box_rows, int box_cols) {
   static EncodeTiled encode = nullptr;
   if (!encode) {
     void* fn = nullptr;
@@ -70,14 +70,12 @@ bool make_tensor_map_2d(void* out, const void* base, int rows, int cols, int box
     encode = reinterpret_cast<EncodeTiled>(fn);
   }
   if (rows < 1 || cols < 1 || cols % 4 || (reinterpret_cast<uintptr_t>(base) & 15)) return false;
-  if (swizzle_128b && box_cols * 4 != 128) return false;                // a swizzled box row spans exactly the swizzle
   const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   const cuuint64_t strides[1] = {(cuuint64_t)cols * 4};                 // bytes between rows: a multiple of 16
   const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
   const cuuint32_t step[2] = {1, 1};
   return encode(static_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(base), dims, strides, box,
-                step, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_128b ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
-                swizzle_128b ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                step, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 

@@ -35,6 +35,6 @@ int sm_count();
 bool cooperative_launch_ok();   // the current device can run a grid with all blocks resident
 // Fills the CUtensorMap at `out` for box copies from a row-major rows x cols array of 4-byte
 // elements; false if the driver call is unavailable or the array is not 16-byte friendly.
-bool make_tensor_map_2d(void* out, const void* base, int rows, int cols, int box_rows, int box_cols, bool swizzle_128b = false);
+bool make_tensor_map_2d(void* out, const void* base, int rows, int cols, int box_rows, int box_cols);
 
 }  // namespace acc
