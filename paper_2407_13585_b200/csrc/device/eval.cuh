@@ -277,11 +277,11 @@ __device__ __forceinline__ uint32_t free_of(const A& a) {
   else return 0u;
 }
 
-template <class CL, int I, class A>
-__device__ __forceinline__ uint32_t eval_member1(const A& a, const Ix& ix) {
+template <class CL, int I, class A, class IX>
+__device__ __forceinline__ uint32_t eval_member1(const A& a, const IX& ix) {     // IX: any one-element index kind
   constexpr CNode nd = CL::c.nodes[I];
   if constexpr (nd.kind == ACC_GENERATE) {
-    return generate1<nd.fn, nd.dtype>(a.n[I], ix, free_of<CL, I>(a));
+    return generate1<nd.fn, nd.dtype>(a.n[I], lane(ix, 0), free_of<CL, I>(a));
   } else if constexpr (nd.kind == ACC_MAP) {
     return apply1<nd.fn>(a.n[I], eval<CL, nd.in[0]>(a, ix), free_of<CL, I>(a));
   } else if constexpr (nd.kind == ACC_ZIPWITH && nd.narr == 2) {

@@ -237,6 +237,28 @@ struct Launcher {
     }
     dev::Args<N> a;
     fill(L, a, R, C);
+    if constexpr (dev::rowfold_then_eligible<CL>()) {
+      // row folds consumed by element-wise members: the block walks the folds' source rows
+      int src = -1;
+      for (int i = 0; i < N && src < 0; ++i)
+        if (dev::is_inner_row_fold(CL::c.nodes[i])) src = CL::c.nodes[i].in[0];
+      bool same = true;                                  // every fold reduces an array of one shape
+      for (int i = 0; i < N; ++i)
+        if (dev::is_inner_row_fold(CL::c.nodes[i]))
+          same = same && L.nodes[CL::c.nodes[i].in[0]].R == L.nodes[src].R && L.nodes[CL::c.nodes[i].in[0]].C == L.nodes[src].C;
+      if (same && L.nodes[src].C >= 64) {                // short rows are as well off pulled through
+        a.R = L.nodes[src].R;
+        a.C = L.nodes[src].C;
+        if (a.R == 0) return ACC_OK;
+        const int grid = std::min(a.R, sm_count() * 16);
+        const bool v4 = vec_ok(L, a.C);
+        if (v4) dev::k_rowfold_then<CL, true><<<grid, dev::kBlock, 0, L.stream>>>(a);
+        else dev::k_rowfold_then<CL, false><<<grid, dev::kBlock, 0, L.stream>>>(a);
+        const cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return set_error(ACC_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+        return ACC_OK;
+      }
+    }
     if (use_tiles(L, R, C)) {
       if constexpr (kTileShape) {
         const int rc = launch_tiles_tma(L, a, R, vec);

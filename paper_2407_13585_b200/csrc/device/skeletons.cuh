@@ -269,6 +269,128 @@ __global__ void __launch_bounds__(kBlock) k_rowfold(const __grid_constant__ Args
 }
 
 // =========================================================================================
+// k_rowfold_then: row folds whose results are consumed, row for row, by element-wise members of
+// the same cluster (a map of a fold: normalisations, the paper's greedyBottomUpBad).  Pulled
+// through, each output element would walk its whole row in one thread; here a block reduces
+// the rows of all such folds together, one thread then evaluates the consumers of that row with
+// the reduced values in place of the folds (IxAfter), and folds that are manifest are stored on
+// the way.
+struct IxAfter { int r, c; const uint32_t* folded; };    // element c of a rank-1 result; folded[k]: value of the k-th fold at c
+template <> struct width_of<IxAfter> { static constexpr int value = 1; };
+__device__ __forceinline__ Ix lane(const IxAfter& i, int) { return Ix{i.r, i.c}; }
+__device__ __forceinline__ uint32_t ld(const uint32_t* p, int C, const IxAfter& i) { return ld1(p, C, Ix{i.r, i.c}); }
+template <int F, int P0 = kRunTime, int P1 = kRunTime>
+__device__ __forceinline__ auto map_index(const IxAfter& i, const NodeArg& self, const NodeArg& src) {
+  if constexpr (F == ACC_IDX_IDENTITY) return i;
+  else return map1<F>(Ix{i.r, i.c}, self, src);            // behind any other map the folds are pulled through again
+}
+
+constexpr bool is_inner_row_fold(const CNode& n) { return n.member && n.kind == ACC_FOLD && n.rank == 1; }
+template <class CL> constexpr int fold_slot(int i) {
+  int k = 0;
+  for (int j = 0; j < i; ++j) k += is_inner_row_fold(CL::c.nodes[j]) ? 1 : 0;
+  return k;
+}
+template <class CL, int I> struct reads_staged<CL, I, IxAfter> { static constexpr bool value = is_inner_row_fold(CL::c.nodes[I]); };
+template <class CL, int I, class A>
+__device__ __forceinline__ uint32_t ld_staged(const A&, const IxAfter& ix) { return ix.folded[fold_slot<CL>(I)]; }
+
+// does node i depend on a fold member (through members)?
+template <class CL> constexpr bool below_fold(int i) {
+  const CNode& n = CL::c.nodes[i];
+  if (!n.member) return false;
+  if (n.kind == ACC_FOLD) return true;
+  for (int s = 0; s < n.nin; ++s)
+    if (below_fold<CL>(n.in[s])) return true;
+  return false;
+}
+// element-wise members on top of row folds: rank-1 maps / zipWiths / generates of rank-1 arrays and folds
+template <class CL> constexpr bool only_elementwise_above_folds(int i) {
+  const CNode& n = CL::c.nodes[i];
+  if (!n.member) return n.rank <= 1;
+  if (n.kind == ACC_FOLD) return true;
+  if (n.rank != 1 || (n.kind != ACC_MAP && n.kind != ACC_ZIPWITH && n.kind != ACC_GENERATE)) return false;
+  for (int s = 0; s < n.narr; ++s)
+    if (!only_elementwise_above_folds<CL>(n.in[s])) return false;
+  return true;
+}
+template <class CL> constexpr bool rowfold_then_eligible() {
+  int inner = 0, consumers = 0;
+  for (int i = 0; i < CL::c.n; ++i) {
+    const CNode& n = CL::c.nodes[i];
+    if (!n.member) continue;
+    if (n.kind == ACC_FOLD) {
+      if (n.rank != 1 || CL::c.nodes[n.in[0]].rank != 2 || below_fold<CL>(n.in[0])) return false;
+      ++inner;
+    } else if (n.kind == ACC_SCANL || n.kind == ACC_SCANR || n.kind == ACC_PERMUTE || n.kind == ACC_FOLDSEG) {
+      return false;
+    } else if (is_store_root(n)) {
+      if (below_fold<CL>(i)) {
+        if (!only_elementwise_above_folds<CL>(i)) return false;
+        ++consumers;
+      } else {
+        return false;                                      // a root beside the folds: another skeleton's job
+      }
+    }
+  }
+  return inner >= 1 && inner <= 4 && consumers >= 1;
+}
+
+template <class CL, bool VEC>
+__global__ void __launch_bounds__(kBlock) k_rowfold_then(const __grid_constant__ Args<CL::c.n> a) {
+  constexpr int N = CL::c.n;
+  constexpr int W = VEC ? 4 : 1;
+  constexpr int NFOLD = count_if<CL>(is_inner_row_fold);
+  using IX = std::conditional_t<VEC, Ix4, Ix>;
+  __shared__ uint32_t red[kBlock / 32];
+  __shared__ uint32_t folded[NFOLD];
+  for (int r = blockIdx.x; r < a.R; r += gridDim.x) {     // a.R x a.C: the shape the folds reduce
+    uint32_t acc[N];
+    static_for<0, N>([&](auto ic) {
+      constexpr int i = decltype(ic)::value;
+      constexpr CNode nd = CL::c.nodes[i];
+      if constexpr (is_inner_row_fold(nd)) acc[i] = identity_of<nd.fn, nd.dtype>();
+    });
+    for (int c = threadIdx.x * W; c < a.C; c += kBlock * W) {
+      const IX ix{r, c};
+      static_for<0, N>([&](auto ic) {
+        constexpr int i = decltype(ic)::value;
+        constexpr CNode nd = CL::c.nodes[i];
+        if constexpr (is_inner_row_fold(nd)) {
+          const auto v = eval<CL, nd.in[0]>(a, ix);
+          if constexpr (VEC) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i] = combine<nd.fn, nd.dtype>(acc[i], v.v[j]);
+          } else {
+            acc[i] = combine<nd.fn, nd.dtype>(acc[i], v);
+          }
+        }
+      });
+    }
+    static_for<0, N>([&](auto ic) {
+      constexpr int i = decltype(ic)::value;
+      constexpr CNode nd = CL::c.nodes[i];
+      if constexpr (is_inner_row_fold(nd)) {
+        const uint32_t v = block_reduce<nd.fn, nd.dtype>(acc[i], red);
+        if (threadIdx.x == 0) {
+          folded[fold_slot<CL>(i)] = v;
+          if constexpr (nd.manifest) reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr))[r] = v;
+        }
+      }
+    });
+    if (threadIdx.x == 0) {
+      const IxAfter ix{0, r, folded};
+      static_for<0, N>([&](auto ic) {
+        constexpr int i = decltype(ic)::value;
+        if constexpr (is_store_root(CL::c.nodes[i]))
+          reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr))[r] = eval<CL, i>(a, ix);
+      });
+    }
+    __syncthreads();                                       // `folded` is rewritten for the next row
+  }
+}
+
+// =========================================================================================
 // Scratch layout of k_scan: word [0] ticket; from byte 16 one 64-bit tile state per tile:
 // (flag << 32) | value, flag 0 = nothing yet, 1 = the tile's own total, 2 = inclusive prefix.
 constexpr int kScanRows = 4;                     // 128-bit chunks per thread

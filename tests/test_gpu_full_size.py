@@ -99,3 +99,7 @@ def test_greedy_bottom_up_bad_at_paper_scale():
     assert g.partition_cost(pi, "bytes") < g.partition_cost(g.plan("greedy_bottomup", "bytes"), "bytes") / 1000
     ref = oracle_run(prog, {k: v.cpu().numpy() for k, v in inputs.items()})
     compare(prog, ref, got, "greedy_bottom_up_bad, m = 10^6")
+    # the bottom-up greedy clustering itself: a map of a row fold in one kernel
+    got, inputs, pi, g = run_full(prog, "greedy_bottomup")
+    assert pi == [-1, 0, 0, 1, 0, 1] and g.launch_count() == 2
+    compare(prog, ref, got, "greedy_bottom_up_bad, m = 10^6, bottom-up greedy")

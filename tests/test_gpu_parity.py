@@ -372,3 +372,11 @@ def test_histogram_total_regenerates_vals_in_its_own_kernel(n, bins):
         cnt = int(np.prod(nd.shape, dtype=np.int64)) if nd.shape else 1
         got[o] = bufs[o][:cnt].cpu().numpy().view(np.float32).reshape(tuple(nd.shape))
     compare(prog, ref, got, "config5 with a copy of vals")
+
+
+# row folds consumed by a map of the same cluster (the clustering the bottom-up greedy finds for the paper's
+# trap program, and every other clustering of it): rows reduced by a block, the map applied to the reduced
+# values; rows of several block strides, ragged, with and without 128-bit accesses, and short rows (pulled)
+@pytest.mark.parametrize("n,m", [(64, 1000), (7, 4099), (3, 40), (300, 256)])
+def test_maps_of_row_folds(n, m):
+    assert check_program(W.greedy_bottom_up_bad(n, m)) >= 8
