@@ -439,7 +439,7 @@ __global__ void __launch_bounds__(kTpThreads) k_tile_pair_tma(const __grid_const
   volatile uint32_t* const v_abort = &abort_walk;
 
   if (threadIdx.x >= kTpConsumers) {
-    // ---------------- copy warp: one lane keeps kStages - 1 pairs in flight ---------------------
+    // ---------------- copy warp: one lane keeps up to kStages pairs in flight -------------------
     if (lane_id != 0) return;
     auto issue = [&](uint32_t pair, int stage) {
       int I, J;

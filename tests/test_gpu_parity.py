@@ -380,3 +380,9 @@ def test_histogram_total_regenerates_vals_in_its_own_kernel(n, bins):
 @pytest.mark.parametrize("n,m", [(64, 1000), (7, 4099), (3, 40), (300, 256)])
 def test_maps_of_row_folds(n, m):
     assert check_program(W.greedy_bottom_up_bad(n, m)) >= 8
+
+
+# two arrays staged as tile pairs, one read as it lies and one transposed; sizes as for config 2
+@pytest.mark.parametrize("rows", [4, 64, 100, 130, 256, 1600])
+def test_diagonal_of_a_product(rows):
+    assert check_program(W.diagonal_of_product(rows)) == 4

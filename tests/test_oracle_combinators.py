@@ -330,3 +330,16 @@ def test_foldseg_rejects_empty_and_stray_segments():
         run(nodes, {0: np.zeros(5, F32), 1: np.array([0, 2, 2], I32)})       # no seed: an empty segment has no value
     with pytest.raises(IndexError):
         run(nodes, {0: np.zeros(5, F32), 1: np.array([0, 2, 6], I32)})
+
+
+def test_diagonal_of_a_product_against_matmul():
+    # d[i] = sum_j A[i][j] * B[j][i] is the diagonal of the matrix product; the products are rounded to fp32
+    # (one rounding of at most 2^-24 relative each), the sums carried in fp64
+    p = W.diagonal_of_product(37)
+    inp = {k: v.numpy() for k, v in W.make_inputs(p).items()}
+    res = interp.run(p.nodes, inp)
+    a, b = inp[0].astype(np.float64), inp[1].astype(np.float64)
+    want = np.diag(a @ b)
+    bound = 2.0 ** -24 * np.einsum("ij,ji->i", np.abs(a), np.abs(b)) + 1e-12
+    assert (np.abs(res.exact[4] - want) <= bound).all()
+    assert (np.abs(res.values[4] - want) <= bound + 2.0 ** -24 * np.abs(want)).all()

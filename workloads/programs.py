@@ -305,4 +305,17 @@ def exclusive_row_scans(rows=64, cols=300):
     return Program("exclusive_row_scans", nodes, [1])
 
 
+def diagonal_of_product(rows=256):
+    """d[i] = sum_j A[i][j] * B[j][i], the diagonal of A B: two square arrays, one of them read transposed."""
+    sh = (rows, rows)
+    nodes = [
+        _inp("A", "f32", sh),
+        _inp("B", "f32", sh),
+        Node("backpermute", "f32", sh, (1,), 1, idx_fn="transpose", name="Bt"),
+        Node("zipwith", "f32", sh, (0, 2), 2, fn="mul", name="P"),
+        Node("fold", "f32", (rows,), (3,), 1, fn="add", name="d"),
+    ]
+    return Program("diagonal_of_product", nodes, [4])
+
+
 CONFIGS = {1: config1, 2: config2, 3: config3, 4: config4, 5: config5}
