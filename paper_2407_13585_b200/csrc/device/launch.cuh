@@ -347,10 +347,105 @@ int Launcher<CL>::launch_hist(const ClusterLaunch& L, dev::Args<N>& a, int R, in
   }
 }
 
+// A cluster whose accumulating roots no single skeleton walks together (two scans; a scan beside a
+// fold or a scatter; row folds beside a scatter) runs as several passes over the same description.
+// Each pass keeps one group of those roots and treats the others as absent; only the first pass writes
+// the element-wise roots.  Producers that the groups share are evaluated again in every pass, from
+// the cluster's inputs: nothing beyond the cluster's own manifest arrays reaches memory.
+constexpr int kMaxPasses = 6;
+struct PassPlan {
+  int n = 0;
+  uint64_t keep[kMaxPasses] = {};     // bit i: accumulating root i runs in this pass
+};
+
+constexpr bool is_accumulating_root(const CNode& n) {
+  return dev::is_fold_root(n) || dev::is_scan_root(n) || dev::is_permute_root(n);
+}
+
+template <class CL> constexpr PassPlan pass_plan() {
+  PassPlan p;
+  uint64_t folds = 0, permutes = 0;
+  for (int i = 0; i < CL::c.n; ++i) {
+    const CNode& n = CL::c.nodes[i];
+    if (dev::is_scan_root(n)) p.keep[p.n++] = 1ull << i;             // a scan walks alone
+    else if (dev::is_fold_root(n)) folds |= 1ull << i;
+    else if (dev::is_permute_root(n)) permutes |= 1ull << i;
+  }
+  // whole-array folds and scatters share the streaming kernel; row folds have a kernel of their own
+  const bool together = dev::domain_rank<CL>() <= 1 || !folds || !permutes;
+  if (together) {
+    if (p.n == 0 || (folds | permutes)) p.keep[p.n++] = folds | permutes;
+  } else {
+    p.keep[p.n++] = folds;
+    p.keep[p.n++] = permutes;
+  }
+  return p;
+}
+
+constexpr CCluster pass_cluster(CCluster c, uint64_t keep, bool stores) {
+  for (int i = 0; i < c.n; ++i) {
+    CNode& n = c.nodes[i];
+    if (is_accumulating_root(n) && !((keep >> i) & 1))
+      n = CNode{ACC_INPUT, n.dtype, n.rank, 0, 0, 0, 0, {-1, -1, -1, -1, -1, -1}, false, true};   // an array nobody reads
+    else if (!stores && dev::is_store_root(n))
+      n.manifest = false;
+  }
+  return c;
+}
+
+template <class CL, int P>
+struct PassOf {
+  static constexpr CCluster c = pass_cluster(CL::c, pass_plan<CL>().keep[P], P == 0);
+};
+
+template <class CL>
+struct Passes {
+  static constexpr PassPlan plan = pass_plan<CL>();
+
+  template <int P>
+  static int64_t scratch_from(const ClusterLaunch& L) {
+    if constexpr (P < plan.n) {
+      const int64_t here = Launcher<PassOf<CL, P>>::scratch_bytes(L);
+      if (here < 0) return here;
+      const int64_t rest = scratch_from<P + 1>(L);
+      return rest < 0 ? rest : ((here + 255) & ~int64_t(255)) + rest;
+    } else {
+      return 0;
+    }
+  }
+  static int64_t scratch_bytes(const ClusterLaunch& L) {
+    if constexpr (plan.n <= 1) return Launcher<CL>::scratch_bytes(L);
+    else return scratch_from<0>(L);
+  }
+
+  template <int P>
+  static int launch_from(ClusterLaunch& L) {
+    if constexpr (P < plan.n) {
+      const int64_t here = Launcher<PassOf<CL, P>>::scratch_bytes(L);
+      if (here < 0) return (int)here;
+      const int rc = Launcher<PassOf<CL, P>>::launch(L);
+      if (rc != ACC_OK) return rc;
+      L.scratch += ((here + 255) & ~int64_t(255)) / 4;
+      return launch_from<P + 1>(L);
+    } else {
+      return ACC_OK;
+    }
+  }
+  static int launch(const ClusterLaunch& L) {
+    if constexpr (plan.n <= 1) {
+      return Launcher<CL>::launch(L);
+    } else {
+      ClusterLaunch pass = L;
+      return launch_from<0>(pass);
+    }
+  }
+};
+
 template <class CL>
 struct Registrar {
   explicit Registrar(const char* name) {
-    register_kernel(KernelEntry{signature(CL::c), name, &Launcher<CL>::scratch_bytes, &Launcher<CL>::launch});
+    register_kernel(KernelEntry{signature(CL::c), name, &Passes<CL>::scratch_bytes, &Passes<CL>::launch,
+                                Passes<CL>::plan.n > 1 ? Passes<CL>::plan.n : 1});
   }
 };
 

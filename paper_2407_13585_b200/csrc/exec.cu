@@ -187,7 +187,7 @@ int run_schedule(Graph& g, Schedule& sch, void* workspace, size_t ws_bytes, cuda
     const int rc = st.kernel->launch(st.launch);
     if (rc != ACC_OK) return rc;
     if (!mark(marks, stream)) return set_error(ACC_ERR_CUDA, "recording an event failed: %s", cudaGetErrorString(cudaGetLastError()));
-    g.launches += 1;
+    g.launches += st.kernel->passes;
     char item[48];
     snprintf(item, sizeof item, "%s%d:%d", g.schedule.empty() ? "" : " ", st.first_node, st.n_members);
     g.schedule += item;

@@ -26,6 +26,7 @@ struct KernelEntry {
   const char* name;
   int64_t (*scratch_bytes)(const ClusterLaunch&);   // >= 0, or a negative acc_status
   int (*launch)(const ClusterLaunch&);               // acc_status; asynchronous
+  int passes = 1;                                    // launches per run (see Passes in device/launch.cuh)
 };
 
 void register_kernel(const KernelEntry& e);

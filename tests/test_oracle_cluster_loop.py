@@ -53,6 +53,13 @@ def test_both_evaluators_agree_on_every_legal_clustering(prog, count):
         assert n == count
 
 
+@pytest.mark.parametrize("seed", range(14))
+def test_both_evaluators_agree_on_random_programs(seed):
+    # seeded random DAGs of element-wise nodes, reversals, gathers, folds, scans and scatters, rank 1 and rank 2
+    agree_everywhere(W.random_program(seed, 37), max_partitions=60)
+    agree_everywhere(W.random_program(seed, 9, 4), max_partitions=30)
+
+
 def test_config1_full_size_all_clusterings():
     assert agree_everywhere(W.config1(1 << 16)) == 8
 

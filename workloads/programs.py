@@ -319,3 +319,69 @@ def diagonal_of_product(rows=256):
 
 
 CONFIGS = {1: config1, 2: config2, 3: config3, 4: config4, 5: config5}
+
+
+# --------------------------------------------------------------------------
+# Seeded random DAGs (test programs nobody drew by hand)
+# --------------------------------------------------------------------------
+
+def random_program(seed, n=4099, rows=None, steps=None):
+    """A seeded random DAG: a body of element-wise nodes, reversals and gathers over arrays of one shape
+    ((n,) or (rows, n)), then accumulating nodes (folds, scans, a scatter) at the leaves and possibly a map
+    that reads a fold's result.  Every node without a consumer is an output.  The draws come from the
+    counter-based generator of the input arrays, so the same seed names the same program everywhere."""
+    from .inputs import counter_bits
+    shape = (n,) if rows is None else (rows, n)
+    count = n if rows is None else rows * n
+    draws = iter(counter_bits(seed, 63, 96).tolist())
+
+    def pick(k):
+        return ((next(draws) & ((1 << 63) - 1)) >> 20) % k
+
+    nodes = [_inp("x", "f32", shape), _inp("v", "f32", shape), _inp("idx", "i32", shape)]
+    arrays = [0, 1]
+    affine = [(2.0, 1.0), (-0.5, 0.25), (1.0, -3.0), (0.125, 0.0)]
+
+    def add(node):
+        nodes.append(node)
+        node.name = "%s%d" % (node.kind[0], len(nodes) - 1)
+        return len(nodes) - 1
+
+    def some():
+        return arrays[pick(len(arrays))]
+
+    for _ in range(3 + pick(3) if steps is None else steps):
+        k = pick(6)
+        if k == 0:
+            i = add(Node("map", "f32", shape, (some(),), 1, fn="affine", fparam=affine[pick(4)]))
+        elif k in (1, 2):
+            i = add(Node("zipwith", "f32", shape, (some(), some()), 2, fn=("add", "mul", "mul_add_const", "add_scale")[pick(4)],
+                         fparam=(0.75,)))
+        elif k == 3:
+            i = add(Node("backpermute", "f32", shape, (some(),), 1, idx_fn="reverse"))
+        elif k == 4:
+            i = add(Node("gather", "f32", shape, (2, some()), 2))
+        else:
+            i = add(Node("zipwith", "f32", shape, (some(), some(), some()), 3, fn="add3"))
+        arrays.append(i)
+    folded = shape[:-1]
+    fold = None
+    for _ in range(1 + pick(2)):
+        k = pick(6)
+        if k == 0:
+            fold = add(Node("fold", "f32", folded, (some(),), 1, fn="add"))
+        elif k == 1:
+            fold = add(Node("fold", "f32", folded, (some(),), 1, fn="max"))
+        elif k == 2:
+            add(Node("scanl", "f32", shape, (some(),), 1, fn="add"))
+        elif k == 3:
+            add(Node("scanr", "f32", shape, (some(),), 1, fn="max"))
+        elif k == 4:
+            add(Node("scanl", "f32", shape, (some(),), 1, fn="add", fparam=(0.5,), exclusive=True))
+        else:
+            add(Node("permute", "f32", shape, (some(), 2, some()), 3, fn="add"))
+    if fold is not None and pick(2):
+        add(Node("map", "f32", shape, (some(), fold), 1, fn="add_free"))
+    used = {s for nd in nodes for s in nd.inputs}
+    outputs = [i for i, nd in enumerate(nodes) if nd.kind != "input" and i not in used]
+    return Program("random%s_%d" % ("" if rows is None else "2d", seed), nodes, outputs, index_bound={"idx": count})
