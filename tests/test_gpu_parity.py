@@ -133,6 +133,20 @@ def test_random_rank2_programs_all_partitions(seed, rows, n):
     check_program(W.random_program(seed, n, rows), passes=True)
 
 
+# the integer counterparts (wrapping arithmetic, generated arrays, clamped shifts by up to three cells, folds,
+# scans and scatters with +, min and max): every array bit for bit
+@pytest.mark.parametrize("n", [1, 4099, 70000])
+@pytest.mark.parametrize("seed", [1, 3, 4, 5, 8, 10, 11])
+def test_random_integer_programs_all_partitions(seed, n):
+    check_program(W.random_int_program(seed, n), passes=True)
+
+
+@pytest.mark.parametrize("rows,n", [(3, 5), (37, 300), (64, 1024)])
+@pytest.mark.parametrize("seed", [2, 3, 4, 5, 7, 10])
+def test_random_integer_rank2_programs_all_partitions(seed, rows, n):
+    check_program(W.random_int_program(seed, n, rows), passes=True)
+
+
 def test_runs_are_repeatable():
     # a racy fold, scan or scatter would differ between runs; integer outputs must be identical
     check_program(W.config3(1 << 16), runs=3)

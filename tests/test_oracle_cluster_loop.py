@@ -58,6 +58,8 @@ def test_both_evaluators_agree_on_random_programs(seed):
     # seeded random DAGs of element-wise nodes, reversals, gathers, folds, scans and scatters, rank 1 and rank 2
     agree_everywhere(W.random_program(seed, 37), max_partitions=60)
     agree_everywhere(W.random_program(seed, 9, 4), max_partitions=30)
+    agree_everywhere(W.random_int_program(seed, 37), max_partitions=40)
+    agree_everywhere(W.random_int_program(seed, 9, 4), max_partitions=30)
 
 
 def test_config1_full_size_all_clusterings():

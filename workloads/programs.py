@@ -385,3 +385,65 @@ def random_program(seed, n=4099, rows=None, steps=None):
     used = {s for nd in nodes for s in nd.inputs}
     outputs = [i for i, nd in enumerate(nodes) if nd.kind != "input" and i not in used]
     return Program("random%s_%d" % ("" if rows is None else "2d", seed), nodes, outputs, index_bound={"idx": count})
+
+
+def random_int_program(seed, n=4099, rows=None):
+    """The integer counterpart of `random_program`: wrapping int32 arithmetic, hashes and masks, generated
+    arrays, reversals, gathers and (rank 2) clamped shifts by up to three cells; folds, scans and scatters with
+    +, min and max at the leaves.  Every result is exact, so every array compares bit for bit."""
+    from .inputs import counter_bits
+    shape = (n,) if rows is None else (rows, n)
+    count = n if rows is None else rows * n
+    draws = iter(counter_bits(seed, 62, 96).tolist())
+
+    def pick(k):
+        return ((next(draws) & ((1 << 63) - 1)) >> 20) % k
+
+    nodes = [_inp("x", "i32", shape), _inp("v", "i32", shape), _inp("idx", "i32", shape)]
+    arrays = [0, 1]
+    unary = [("hash_mul_xorshift", (2654435761, 13)), ("and_mask", (0xFFFF,)), ("mul_const", (3,)), ("add_const", (-7,)),
+             ("identity", ())]
+
+    def add(node):
+        nodes.append(node)
+        node.name = "%s%d" % (node.kind[0], len(nodes) - 1)
+        return len(nodes) - 1
+
+    def some():
+        return arrays[pick(len(arrays))]
+
+    for _ in range(3 + pick(3)):
+        k = pick(7)
+        if k == 0:
+            fn, ip = unary[pick(len(unary))]
+            i = add(Node("map", "i32", shape, (some(),), 1, fn=fn, iparam=ip))
+        elif k in (1, 2):
+            i = add(Node("zipwith", "i32", shape, (some(), some()), 2, fn=("add", "mul")[pick(2)]))
+        elif k == 3:
+            i = add(Node("backpermute", "i32", shape, (some(),), 1, idx_fn="reverse"))
+        elif k == 4:
+            i = add(Node("gather", "i32", shape, (2, some()), 2))
+        elif k == 5:
+            i = add(Node("generate", "i32", shape, (), 0, fn="iota"))
+        elif rows is None:
+            i = add(Node("map", "i32", shape, (some(),), 1, fn="and_mask", iparam=(0xFF,)))
+        else:
+            i = add(Node("backpermute", "i32", shape, (some(),), 1, idx_fn="shift_clamp", iparam=(pick(7) - 3, pick(7) - 3)))
+        arrays.append(i)
+    folded = shape[:-1]
+    ops = ("add", "min", "max")
+    for _ in range(1 + pick(3)):
+        k = pick(5)
+        if k == 0:
+            add(Node("fold", "i32", folded, (some(),), 1, fn=ops[pick(3)]))
+        elif k == 1:
+            add(Node("scanl", "i32", shape, (some(),), 1, fn=ops[pick(3)]))
+        elif k == 2:
+            add(Node("scanr", "i32", shape, (some(),), 1, fn=ops[pick(3)]))
+        elif k == 3:
+            add(Node("scanr", "i32", shape, (some(),), 1, fn="add", iparam=(1000,), exclusive=True))
+        else:
+            add(Node("permute", "i32", shape, (some(), 2, some()), 3, fn=ops[pick(3)]))
+    used = {s for nd in nodes for s in nd.inputs}
+    outputs = [i for i, nd in enumerate(nodes) if nd.kind != "input" and i not in used]
+    return Program("random_int%s_%d" % ("" if rows is None else "2d", seed), nodes, outputs, index_bound={"idx": count})
