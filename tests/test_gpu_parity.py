@@ -147,6 +147,13 @@ def test_random_integer_rank2_programs_all_partitions(seed, rows, n):
     check_program(W.random_int_program(seed, n, rows), passes=True)
 
 
+# square arrays, so that transposes join in: below one 64 x 64 tile, ragged tiles without 128-bit rows, whole tiles
+@pytest.mark.parametrize("rows", [5, 70, 256])
+@pytest.mark.parametrize("seed", [3, 7, 14, 23, 39])
+def test_random_integer_square_programs_all_partitions(seed, rows):
+    check_program(W.random_int_program(seed, rows, rows), passes=True)
+
+
 def test_runs_are_repeatable():
     # a racy fold, scan or scatter would differ between runs; integer outputs must be identical
     check_program(W.config3(1 << 16), runs=3)

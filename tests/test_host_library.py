@@ -36,7 +36,7 @@ PROGRAMS = [W.config1(64), W.config2(8), W.config3(64), W.config4(8, 8, iters=1)
             W.scatter_example(16), W.scatter_example_paper_graph(), W.single_loop(16), W.simple1(), W.simple2(),
             W.simple3(), W.simple4(), W.simple5(), W.greedy_bottom_up_bad(4, 5), W.greedy_top_down_bad(16),
             W.segmented_sums(64, 5)] + [W.random_program(s, 16) for s in range(14)] + [W.random_program(s, 8, 3) for s in (0, 3, 5, 8)] + [
-                W.random_int_program(s, 16) for s in range(12)] + [W.random_int_program(s, 8, 3) for s in range(12)]
+                W.random_int_program(s, 16) for s in range(12)] + [W.random_int_program(s, 8, 3) for s in range(12)] + [W.random_int_program(s, 6, 6) for s in (2, 3, 7, 14, 16, 17, 20, 23, 31, 39)]
 
 
 @pytest.mark.parametrize("prog", PROGRAMS, ids=lambda p: p.name)

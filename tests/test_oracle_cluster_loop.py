@@ -60,6 +60,7 @@ def test_both_evaluators_agree_on_random_programs(seed):
     agree_everywhere(W.random_program(seed, 9, 4), max_partitions=30)
     agree_everywhere(W.random_int_program(seed, 37), max_partitions=40)
     agree_everywhere(W.random_int_program(seed, 9, 4), max_partitions=30)
+    agree_everywhere(W.random_int_program(seed + 10, 6, 6), max_partitions=30)      # square: with transposes
 
 
 def test_config1_full_size_all_clusterings():

@@ -389,7 +389,7 @@ def random_program(seed, n=4099, rows=None, steps=None):
 
 def random_int_program(seed, n=4099, rows=None):
     """The integer counterpart of `random_program`: wrapping int32 arithmetic, hashes and masks, generated
-    arrays, reversals, gathers and (rank 2) clamped shifts by up to three cells; folds, scans and scatters with
+    arrays, reversals, gathers, (rank 2) clamped shifts by up to three cells and (square) transposes; folds, scans and scatters with
     +, min and max at the leaves.  Every result is exact, so every array compares bit for bit."""
     from .inputs import counter_bits
     shape = (n,) if rows is None else (rows, n)
@@ -427,6 +427,8 @@ def random_int_program(seed, n=4099, rows=None):
             i = add(Node("generate", "i32", shape, (), 0, fn="iota"))
         elif rows is None:
             i = add(Node("map", "i32", shape, (some(),), 1, fn="and_mask", iparam=(0xFF,)))
+        elif rows == n and pick(2):                      # square arrays only: read across the diagonal
+            i = add(Node("backpermute", "i32", shape, (some(),), 1, idx_fn="transpose"))
         else:
             i = add(Node("backpermute", "i32", shape, (some(),), 1, idx_fn="shift_clamp", iparam=(pick(7) - 3, pick(7) - 3)))
         arrays.append(i)
@@ -446,4 +448,5 @@ def random_int_program(seed, n=4099, rows=None):
             add(Node("permute", "i32", shape, (some(), 2, some()), 3, fn=ops[pick(3)]))
     used = {s for nd in nodes for s in nd.inputs}
     outputs = [i for i, nd in enumerate(nodes) if nd.kind != "input" and i not in used]
-    return Program("random_int%s_%d" % ("" if rows is None else "2d", seed), nodes, outputs, index_bound={"idx": count})
+    return Program("random_int%s_%d" % ("" if rows is None else "sq" if rows == n else "2d", seed), nodes, outputs,
+                   index_bound={"idx": count})
