@@ -141,7 +141,7 @@ def test_random_integer_programs_all_partitions(seed, n):
     check_program(W.random_int_program(seed, n), passes=True)
 
 
-@pytest.mark.parametrize("rows,n", [(3, 5), (37, 300), (64, 1024)])
+@pytest.mark.parametrize("rows,n", [(3, 5), (37, 300), (64, 1024), (520, 1284)])
 @pytest.mark.parametrize("seed", [2, 3, 4, 5, 7, 10])
 def test_random_integer_rank2_programs_all_partitions(seed, rows, n):
     check_program(W.random_int_program(seed, n, rows), passes=True)
