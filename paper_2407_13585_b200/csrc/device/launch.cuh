@@ -382,14 +382,43 @@ template <class CL> constexpr PassPlan pass_plan() {
   return p;
 }
 
-constexpr CCluster pass_cluster(CCluster c, uint64_t keep, bool stores) {
+// The scan whose values element-wise member i consumes inside the cluster, -1 if none.
+constexpr int scan_needed_by(const CCluster& c, int i) {
+  for (int s = 0; s < c.n; ++s)
+    if (dev::is_scan_root(c.nodes[s]) && dev::needs_scan(c, i, s)) return s;
+  return -1;
+}
+
+constexpr CNode unread_array(const CNode& n) {
+  return CNode{ACC_INPUT, n.dtype, n.rank, 0, 0, 0, 0, {-1, -1, -1, -1, -1, -1}, false, true};
+}
+
+// The description of one pass: the accumulating roots in `keep` stay; element-wise roots that consume a
+// scan are written by that scan's pass, the other element-wise roots by the first pass; members that no
+// root of the pass reaches any more, and the roots of other passes, become arrays nobody reads.
+constexpr CCluster pass_cluster(CCluster c, uint64_t keep, bool first) {
+  const CCluster whole = c;
+  int scan = -1;
+  for (int i = 0; i < c.n; ++i)
+    if (((keep >> i) & 1) && dev::is_scan_root(whole.nodes[i])) scan = i;
   for (int i = 0; i < c.n; ++i) {
-    CNode& n = c.nodes[i];
-    if (is_accumulating_root(n) && !((keep >> i) & 1))
-      n = CNode{ACC_INPUT, n.dtype, n.rank, 0, 0, 0, 0, {-1, -1, -1, -1, -1, -1}, false, true};   // an array nobody reads
-    else if (!stores && dev::is_store_root(n))
-      n.manifest = false;
+    if (is_accumulating_root(whole.nodes[i]) && !((keep >> i) & 1)) {
+      c.nodes[i] = unread_array(whole.nodes[i]);
+    } else if (dev::is_store_root(whole.nodes[i])) {
+      const int needs = scan_needed_by(whole, i);
+      if (needs >= 0 ? needs != scan : !first) c.nodes[i].manifest = false;
+    }
   }
+  bool live[kMaxCluster] = {};
+  for (int i = c.n - 1; i >= 0; --i) {
+    const CNode& n = c.nodes[i];
+    if (!n.member) continue;
+    if (is_accumulating_root(n) || dev::is_store_root(n) || dev::is_segfold_root(n)) live[i] = true;
+    if (live[i])
+      for (int k = 0; k < n.nin; ++k) live[n.in[k]] = true;
+  }
+  for (int i = 0; i < c.n; ++i)
+    if (c.nodes[i].member && !live[i]) c.nodes[i] = unread_array(c.nodes[i]);
   return c;
 }
 

@@ -408,6 +408,26 @@ __device__ __forceinline__ void st(uint32_t* p, int C, const IxR4& i, const V4& 
   *reinterpret_cast<uint4*>(p + (i.r * C + i.c - 3)) = make_uint4(v.v[3], v.v[2], v.v[1], v.v[0]);
 }
 
+// Element-wise members that consume the scan inside its cluster are evaluated where the scanned values
+// are final, at an index that carries them: IxSc<B> is the plain index B plus the scan's values there,
+// and the scan member reads as those values.  Only index-preserving paths (array operands of map and
+// zipWith, the index operand of a gather) may lead from such a member to the scan; behind an index map
+// the values would be lost, and no such cluster is instantiated.
+template <class B> struct IxSc : B { val_of<B> sv; };
+template <class B> struct width_of<IxSc<B>> { static constexpr int value = width_of<B>::value; };
+template <class CL, int I, class B> struct reads_staged<CL, I, IxSc<B>> { static constexpr bool value = I == first_scan<CL>(); };
+template <class CL, int I, class A, class B>
+__device__ __forceinline__ val_of<B> ld_staged(const A&, const IxSc<B>& ix) { return ix.sv; }
+
+// Whether member i needs the value of scan s (through any chain of operands inside the cluster).
+constexpr bool needs_scan(const CCluster& c, int i, int s) {
+  const CNode& n = c.nodes[i];
+  if (!n.member) return false;
+  for (int k = 0; k < n.nin; ++k)
+    if (n.in[k] == s || needs_scan(c, n.in[k], s)) return true;
+  return false;
+}
+
 // Rows of a rank-2 array are scanned independently: a row is cut into tiles of its own, the
 // look-back of a tile stops at the first tile of its row.  A right-to-left scan walks its row
 // from the far end: position p of the walk is element C-1-p of the row.
@@ -464,7 +484,7 @@ __global__ void __launch_bounds__(kBlock) k_scan(const __grid_constant__ Args<CL
         }
         static_for<0, N>([&](auto ic) {
           constexpr int i = decltype(ic)::value;
-          if constexpr (is_store_root(CL::c.nodes[i]))
+          if constexpr (is_store_root(CL::c.nodes[i]) && !needs_scan(CL::c, i, S))
             st(reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr)), a.n[i].C, ix, eval<CL, i>(a, ix));
         });
       } else {
@@ -547,12 +567,20 @@ __global__ void __launch_bounds__(kBlock) k_scan(const __grid_constant__ Args<CL
       const int c = warp_base + (j * 32 + lane) * W;
       if (c < n) {
         const IX ix = index_at(row, c);
+        IxSc<IX> scanned;
+        static_cast<IX&>(scanned) = ix;
         if constexpr (VEC) {
-          st(out, n, ix, V4{{combine<FN, DT>(base, val[j][0]), combine<FN, DT>(base, val[j][1]),
-                             combine<FN, DT>(base, val[j][2]), combine<FN, DT>(base, val[j][3])}});
+          scanned.sv = V4{{combine<FN, DT>(base, val[j][0]), combine<FN, DT>(base, val[j][1]),
+                           combine<FN, DT>(base, val[j][2]), combine<FN, DT>(base, val[j][3])}};
         } else {
-          st(out, n, ix, combine<FN, DT>(base, val[j][0]));
+          scanned.sv = combine<FN, DT>(base, val[j][0]);
         }
+        if constexpr (sn.manifest) st(out, n, ix, scanned.sv);
+        static_for<0, N>([&](auto ic) {
+          constexpr int i = decltype(ic)::value;
+          if constexpr (is_store_root(CL::c.nodes[i]) && needs_scan(CL::c, i, S))
+            st(reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr)), a.n[i].C, ix, eval<CL, i>(a, scanned));
+        });
       }
     }
   }

@@ -11,7 +11,7 @@ the library's own legality checker), plus every node alone.
 (`module:function[:int,...]` names a program; the integers are the function's arguments.)
 
 Clusters the kernel skeletons cannot express are skipped and listed in a comment: a
-scan that is consumed inside its own cluster, and a fold
+scan whose values are consumed inside its own cluster other than element for element, and a fold
 that is both written to memory and consumed inside its own cluster.
 """
 import importlib
@@ -38,14 +38,39 @@ def clusters_of(prog):
     return sorted(found, key=lambda s: (len(s), sorted(s)))
 
 
+def scans_consumed_in_place(prog, members):
+    """Whether every scan of the cluster that is consumed inside it is consumed element for element: only
+    array operands of map and zipWith and the index operand of a gather lead from a consumer to the scan,
+    and no consumer needs two scans or is itself a fold, a scan or a scatter."""
+    nodes = prog.nodes
+    needs = {}                                   # member -> scans of the cluster it consumes
+    for i in sorted(members):
+        nd = nodes[i]
+        mine = set()
+        for slot, j in enumerate(nd.inputs):
+            if j not in members:
+                continue
+            got = {j} if nodes[j].kind in ("scanl", "scanr") else needs[j]
+            if not got:
+                continue
+            in_place = (nd.kind in ("map", "zipwith") and slot < nd.n_array) or (nd.kind == "gather" and slot == 0)
+            if not in_place:
+                return False
+            mine |= got
+        if len(mine) > 1:
+            return False
+        needs[i] = mine
+    return True
+
+
 def expressible(prog, members):
     nodes = prog.nodes
+    if not scans_consumed_in_place(prog, members):
+        return False
     for i in members:
         k = nodes[i].kind
         inside = [j for j in members if i in nodes[j].inputs]
         outside = i in prog.outputs or any(i in nodes[j].inputs for j in range(len(nodes)) if j not in members)
-        if k in ("scanl", "scanr") and inside:
-            return False
         if k == "fold" and inside and outside:
             return False
         if k == "foldseg" and outside:

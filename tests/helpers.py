@@ -55,18 +55,54 @@ def gpu_run(prog, inputs_t, pi=None, executor=None, bind_all=True, runs=1, recom
     return out, g
 
 
+def error_bounds(prog, ref):
+    """Per element, how far an fp32 array may lie from the oracle's: for a fold, scan or scatter the stated
+    tolerance; for maps and zipWiths of such arrays that tolerance carried through the function to first
+    order (plus the second-order term of a product) and two roundings of the result."""
+    nodes, b = prog.nodes, {}
+    for i, nd in enumerate(nodes):
+        if nd.dtype != "f32":
+            continue
+        if accumulating(nd):
+            b[i] = TOL * ref.abs_sum[i] + np.abs(ref.exact[i]) * 2.0 ** -24 + 1e-30
+            continue
+        ins = nd.inputs[:nd.n_array]
+        if nd.kind not in ("map", "zipwith") or not any(j in b for j in nd.inputs):
+            continue
+        mag = lambda j: np.abs(ref.values[j].astype(np.float64))
+        eb = lambda j: b.get(j, 0.0)
+        if nd.fn == "affine":
+            e = abs(nd.fparam[0]) * eb(ins[0])
+        elif nd.fn == "identity":
+            e = eb(ins[0])
+        elif nd.fn in ("add", "add3"):
+            e = sum(eb(j) for j in ins)
+        elif nd.fn in ("mul", "mul_add_const"):
+            e = mag(ins[0]) * eb(ins[1]) + mag(ins[1]) * eb(ins[0]) + eb(ins[0]) * eb(ins[1])
+        elif nd.fn == "add_scale":
+            e = abs(nd.fparam[0]) * (eb(ins[0]) + eb(ins[1]))
+        elif nd.fn == "add_free":
+            e = eb(ins[0]) + np.max(eb(nd.inputs[1]))
+        else:
+            continue
+        b[i] = e * (1 + 2.0 ** -20) + np.abs(ref.values[i].astype(np.float64)) * 2.0 ** -22 + 1e-30
+    return b
+
+
 def compare(prog, ref, got, what=""):
     """Element-by-element comparison of every array in `got` with the oracle result `ref`.
 
     Integer arrays and fp32 element chains: bit-exact.  fp32 fold/scan/scatter outputs:
     |gpu - fp64 reference| <= 1e-5 * sum|x_i| (+ half an ulp of the result for the final
-    rounding).  A map that divides such an output by such a total inherits both bounds.
+    rounding).  A map that divides such an output by such a total inherits both bounds, and so do other
+    maps and zipWiths of such outputs (error_bounds).
     """
     nodes = prog.nodes
     loose = set()
     for i, nd in enumerate(nodes):
         if accumulating(nd) or any(s in loose for s in nd.inputs):
             loose.add(i)
+    bounds = error_bounds(prog, ref)
     for i, a in got.items():
         nd = nodes[i]
         r = ref.values[i]
@@ -93,6 +129,9 @@ def compare(prog, ref, got, what=""):
             undefined = np.isnan(frac)             # 0/0 when the total is zero: both sides must say so
             assert np.array_equal(np.isnan(a), undefined), (what, i, nd.name)
             assert np.all((err <= bound) | undefined), (what, i, nd.name, float(np.nanmax(err / bound)))
+        elif i in bounds:
+            err = np.abs(a.astype(np.float64) - r.astype(np.float64))
+            assert np.all(err <= bounds[i]), (what, i, nd.name, float((err / bounds[i]).max()))
         else:
             assert np.allclose(a, r, rtol=1e-4, atol=1e-6), (what, i, nd.name)
 

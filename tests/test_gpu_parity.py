@@ -154,6 +154,23 @@ def test_random_integer_square_programs_all_partitions(seed, rows):
     check_program(W.random_int_program(seed, rows, rows), passes=True)
 
 
+# scans consumed element for element inside their cluster (a map of a running sum, offsets used as indices):
+# the consumers are evaluated where the scanned values are final; several scans per cluster take a pass each
+@pytest.mark.parametrize("n", [1, 5, 4099, 4096 * 3, 70000])
+def test_scans_consumed_inside_their_cluster(n):
+    assert check_program(W.scan_consumers(n), passes=True) == 152
+
+
+@pytest.mark.parametrize("rows,n", [(3, 5), (37, 300), (16, 8192)])
+def test_row_scans_consumed_inside_their_cluster(rows, n):
+    assert check_program(W.scan_consumers(n, rows), passes=True) == 152
+
+
+@pytest.mark.parametrize("n", [1, 4, 4096, 1 << 17])
+def test_offsets_used_as_indices_in_the_same_cluster(n):
+    assert check_program(W.offsets_then_gather(n), passes=True) == 20
+
+
 def test_runs_are_repeatable():
     # a racy fold, scan or scatter would differ between runs; integer outputs must be identical
     check_program(W.config3(1 << 16), runs=3)

@@ -318,6 +318,40 @@ def diagonal_of_product(rows=256):
     return Program("diagonal_of_product", nodes, [4])
 
 
+def scan_consumers(n=4099, rows=None):
+    """Scans whose values feed element-wise nodes: a running sum that is only consumed (never an output), a
+    right-to-left running maximum that is both written and consumed, and a seeded exclusive sum."""
+    sh = (n,) if rows is None else (rows, n)
+    nodes = [
+        _inp("x", "f32", sh),
+        _inp("w", "f32", sh),
+        Node("scanl", "f32", sh, (0,), 1, fn="add", name="s"),
+        Node("map", "f32", sh, (2,), 1, fn="affine", fparam=(0.5, 1.0), name="m"),
+        Node("zipwith", "f32", sh, (3, 1), 2, fn="mul", name="z"),
+        Node("scanr", "f32", sh, (1,), 1, fn="max", name="r"),
+        Node("zipwith", "f32", sh, (5, 0), 2, fn="add", name="q"),
+        Node("scanl", "f32", sh, (1,), 1, fn="add", fparam=(0.25,), exclusive=True, name="e"),
+        Node("zipwith", "f32", sh, (7, 0, 1), 3, fn="add3", name="t"),
+    ]
+    return Program("scan_consumers" + ("" if rows is None else "_2d"), nodes, [4, 5, 6, 8])
+
+
+def offsets_then_gather(n=1 << 12):
+    """Offsets from counts, used as indices in the same cluster: c = x & 3; o = exclusive running sum of c;
+    y = src[o & (n-1)] (n a power of two); total = fold(+) c."""
+    assert n & (n - 1) == 0
+    nodes = [
+        _inp("x", "i32", (n,)),
+        _inp("src", "i32", (n,)),
+        Node("map", "i32", (n,), (0,), 1, fn="and_mask", iparam=(3,), name="c"),
+        Node("scanl", "i32", (n,), (2,), 1, fn="add", iparam=(0,), exclusive=True, name="o"),
+        Node("map", "i32", (n,), (3,), 1, fn="and_mask", iparam=(n - 1,), name="k"),
+        Node("gather", "i32", (n,), (4, 1), 2, name="y"),
+        Node("fold", "i32", (), (2,), 1, fn="add", name="total"),
+    ]
+    return Program("offsets_then_gather", nodes, [5, 6], index_bound={"x": 1 << 30, "src": 1 << 30})
+
+
 CONFIGS = {1: config1, 2: config2, 3: config3, 4: config4, 5: config5}
 
 
