@@ -207,6 +207,16 @@ int acc_manifest(const acc_graph* g, int32_t* manifest_out, int32_t n_nodes);
  * reaches the best clustering known, and gives up the proof, not the result,
  * after 2^22 partial clusterings. */
 int acc_plan(acc_graph* g, int mode, int cost, int32_t* cluster_of_node_out);
+/* Makes the stored clustering runnable.  Kernels are instantiated at build
+ * time per cluster shape, and the rules of Figure 3 know nothing of that: a
+ * planner may return a legal cluster nobody built a kernel for (ACC_ERR_NO_KERNEL
+ * from acc_run).  While such a cluster exists, its latest node (in program
+ * order) that can leave it with the clustering still legal becomes a cluster of
+ * its own; if no single node can, the cluster falls apart into its nodes.
+ * Stores the result, writes it to cluster_of_node_out (may be null) and returns
+ * the number of splits (0: every cluster had a kernel), or a negative
+ * acc_status (ACC_ERR_NO_KERNEL if a node alone has none).  Host only. */
+int acc_refine_to_kernels(acc_graph* g, int32_t* cluster_of_node_out);
 /* Every legal clustering, each as n_nodes int32 with canonical numbering
  * (clusters numbered in an execution order, ties by smallest node id), in
  * lexicographic order.  Returns the count (also when out_pi is null or

@@ -91,6 +91,7 @@ def load_library(path=LIB_PATH):
         "acc_enumerate_recompute": (i64, [p, i32, pi32, i64]),
         "acc_partition_cost_recompute": (C.c_int, [p, pi32, i32, i32, C.c_int, C.POINTER(C.c_double)]),
         "acc_plan_info": (C.c_int, [p, C.POINTER(i64), C.POINTER(i32)]),
+        "acc_refine_to_kernels": (C.c_int, [p, pi32]),
         "acc_set_partition_copies": (C.c_int, [p, pi32, i32, pi32, pi32, i32, i32]),
         "acc_bind": (C.c_int, [p, i32, p, sz]),
         "acc_bind_host": (C.c_int, [p, i32, p, sz]),
@@ -263,6 +264,12 @@ class Graph:
         visited, proven = C.c_int64(), C.c_int32()
         _check(lib().acc_plan_info(self._h, C.byref(visited), C.byref(proven)))
         return visited.value, bool(proven.value)
+
+    def refine_to_kernels(self):
+        """Splits clusters that have no instantiated kernel; returns (splits made, the clustering now stored)."""
+        buf = (C.c_int32 * self.n)()
+        splits = _check(lib().acc_refine_to_kernels(self._h, buf))
+        return splits, list(buf)
 
     def enumerate(self):
         cnt = _check(lib().acc_enumerate(self._h, None, 0))

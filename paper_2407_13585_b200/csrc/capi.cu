@@ -230,6 +230,24 @@ int acc_plan_recompute(acc_graph* g, int mode, int cost, int32_t max_depth, int3
 
 int acc_plan(acc_graph* g, int mode, int cost, int32_t* out) { return acc_plan_recompute(g, mode, cost, 0, out); }
 
+int acc_refine_to_kernels(acc_graph* g, int32_t* out) {
+  clear_error();
+  if (!g) return set_error(ACC_ERR_ARG, "graph is null");
+  if (!g->has_pi) return set_error(ACC_ERR_NO_PARTITION, "no clustering set: call acc_set_partition or acc_plan first");
+  if (g->unfolded) return set_error(ACC_ERR_ARG, "a clustering with copies is not refined");
+  std::vector<int32_t> pi(g->pi);
+  int splits = 0;
+  const int depth = g->recompute_depth;
+  int rc = refine_to_kernels(*g, pi, depth, splits);
+  if (rc != ACC_OK) return rc;
+  if (splits > 0) {
+    rc = acc_set_partition_recompute(g, pi.data(), (int32_t)pi.size(), depth);
+    if (rc != ACC_OK) return rc;
+  }
+  if (out) memcpy(out, g->pi.data(), sizeof(int32_t) * g->pi.size());
+  return splits;
+}
+
 int acc_plan_info(const acc_graph* g, int64_t* visited, int32_t* proven) {
   clear_error();
   if (!g) return set_error(ACC_ERR_ARG, "graph is null");

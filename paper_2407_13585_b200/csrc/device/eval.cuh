@@ -253,6 +253,21 @@ __device__ __forceinline__ Ix gather1(uint32_t k, const NodeArg& src) {
   else return Ix{(int)(k / (uint32_t)src.C), (int)(k % (uint32_t)src.C)};
 }
 
+// One step of a thread's running fold.  An fp32 sum carries a compensation term (Kahan's summation): one
+// thread may add thousands of elements, and where their rounding errors do not cancel (equal addends) a
+// plain running sum drifts beyond 1e-5 of the sum of magnitudes; with the term it stays within a few ulp.
+template <int FN, int DT>
+__device__ __forceinline__ void fold_step(uint32_t& acc, float& comp, uint32_t x) {
+  if constexpr (FN == ACC_FN_ADD && DT == ACC_F32) {
+    const float y = __fsub_rn(f_(x), comp);
+    const float t = __fadd_rn(f_(acc), y);
+    comp = __fsub_rn(__fsub_rn(t, f_(acc)), y);
+    acc = u_(t);
+  } else {
+    acc = combine<FN, DT>(acc, x);
+  }
+}
+
 // ---- the evaluator ----------------------------------------------------------------------
 template <class CL, int I, class A, class IX>
 __device__ __forceinline__ val_of<IX> eval(const A& a, const IX& ix);
@@ -335,7 +350,8 @@ __device__ __forceinline__ val_of<IX> eval_here(const A& a, const IX& ix) {
     auto row_value = [&](const Ix& o) {
       const int row = o.r * a.n[I].C + o.c;
       uint32_t acc = identity_of<nd.fn, nd.dtype>();
-      for (int j = 0; j < s.C; ++j) acc = combine<nd.fn, nd.dtype>(acc, eval<CL, nd.in[0]>(a, Ix{row, j}));
+      float comp = 0.0f;
+      for (int j = 0; j < s.C; ++j) fold_step<nd.fn, nd.dtype>(acc, comp, eval<CL, nd.in[0]>(a, Ix{row, j}));
       return acc;
     };
     if constexpr (W == 1) {
@@ -354,7 +370,8 @@ __device__ __forceinline__ val_of<IX> eval_here(const A& a, const IX& ix) {
     auto seg_value = [&](const Ix& o) {
       const int lo = max(__ldg(off + o.c), 0), hi = min(__ldg(off + o.c + 1), s.R * s.C);
       uint32_t acc = identity_of<nd.fn, nd.dtype>();
-      for (int j = lo; j < hi; ++j) acc = combine<nd.fn, nd.dtype>(acc, eval<CL, nd.in[0]>(a, Ix{0, j}));
+      float comp = 0.0f;
+      for (int j = lo; j < hi; ++j) fold_step<nd.fn, nd.dtype>(acc, comp, eval<CL, nd.in[0]>(a, Ix{0, j}));
       return acc;
     };
     if constexpr (W == 1) {

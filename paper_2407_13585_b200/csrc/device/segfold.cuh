@@ -69,6 +69,7 @@ __global__ void __launch_bounds__(kBlock) k_segfold(const __grid_constant__ Args
         if (lane == 0) long_list[atomicAdd(&n_long, 1)] = s;
       } else {
         uint32_t acc[N];
+        float comp[N] = {};                              // see fold_step
         static_for<0, N>([&](auto ic) {
           constexpr int i = decltype(ic)::value;
           constexpr CNode nd = CL::c.nodes[i];
@@ -78,7 +79,7 @@ __global__ void __launch_bounds__(kBlock) k_segfold(const __grid_constant__ Args
           static_for<0, N>([&](auto ic) {
             constexpr int i = decltype(ic)::value;
             constexpr CNode nd = CL::c.nodes[i];
-            if constexpr (is_segfold_root(nd)) acc[i] = combine<nd.fn, nd.dtype>(acc[i], eval<CL, nd.in[0]>(a, Ix{0, j}));
+            if constexpr (is_segfold_root(nd)) fold_step<nd.fn, nd.dtype>(acc[i], comp[i], eval<CL, nd.in[0]>(a, Ix{0, j}));
           });
         }
         static_for<0, N>([&](auto ic) {
@@ -97,6 +98,7 @@ __global__ void __launch_bounds__(kBlock) k_segfold(const __grid_constant__ Args
       const int t = long_list[k];
       const int lo = __ldg(off + t), hi = __ldg(off + t + 1);
       uint32_t acc[N];
+      float comp[N] = {};
       static_for<0, N>([&](auto ic) {
         constexpr int i = decltype(ic)::value;
         constexpr CNode nd = CL::c.nodes[i];
@@ -106,7 +108,7 @@ __global__ void __launch_bounds__(kBlock) k_segfold(const __grid_constant__ Args
         static_for<0, N>([&](auto ic) {
           constexpr int i = decltype(ic)::value;
           constexpr CNode nd = CL::c.nodes[i];
-          if constexpr (is_segfold_root(nd)) acc[i] = combine<nd.fn, nd.dtype>(acc[i], eval<CL, nd.in[0]>(a, Ix{0, j}));
+          if constexpr (is_segfold_root(nd)) fold_step<nd.fn, nd.dtype>(acc[i], comp[i], eval<CL, nd.in[0]>(a, Ix{0, j}));
         });
       }
       static_for<0, N>([&](auto ic) {

@@ -126,6 +126,7 @@ __global__ void __launch_bounds__(kBlock) k_stream(const __grid_constant__ Args<
   __shared__ bool last_block;
 
   uint32_t acc[N];
+  float comp[N] = {};                                    // see fold_step
   static_for<0, N>([&](auto ic) {
     constexpr int i = decltype(ic)::value;
     constexpr CNode nd = CL::c.nodes[i];
@@ -167,9 +168,9 @@ __global__ void __launch_bounds__(kBlock) k_stream(const __grid_constant__ Args<
         const auto v = eval<CL, nd.in[0]>(a, ix);
         if constexpr (VEC) {
 #pragma unroll
-          for (int j = 0; j < 4; ++j) acc[i] = combine<nd.fn, nd.dtype>(acc[i], v.v[j]);
+          for (int j = 0; j < 4; ++j) fold_step<nd.fn, nd.dtype>(acc[i], comp[i], v.v[j]);
         } else {
-          acc[i] = combine<nd.fn, nd.dtype>(acc[i], v);
+          fold_step<nd.fn, nd.dtype>(acc[i], comp[i], v);
         }
       } else if constexpr (is_permute_root(nd)) {
         const auto k = eval<CL, nd.in[1]>(a, ix);
@@ -234,6 +235,7 @@ __global__ void __launch_bounds__(kBlock) k_rowfold(const __grid_constant__ Args
   __shared__ uint32_t red[kBlock / 32];
   for (int r = blockIdx.x; r < a.R; r += gridDim.x) {
     uint32_t acc[N];
+    float comp[N] = {};                                  // see fold_step
     static_for<0, N>([&](auto ic) {
       constexpr int i = decltype(ic)::value;
       constexpr CNode nd = CL::c.nodes[i];
@@ -250,9 +252,9 @@ __global__ void __launch_bounds__(kBlock) k_rowfold(const __grid_constant__ Args
           const auto v = eval<CL, nd.in[0]>(a, ix);
           if constexpr (VEC) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) acc[i] = combine<nd.fn, nd.dtype>(acc[i], v.v[j]);
+            for (int j = 0; j < 4; ++j) fold_step<nd.fn, nd.dtype>(acc[i], comp[i], v.v[j]);
           } else {
-            acc[i] = combine<nd.fn, nd.dtype>(acc[i], v);
+            fold_step<nd.fn, nd.dtype>(acc[i], comp[i], v);
           }
         }
       });
@@ -346,6 +348,7 @@ __global__ void __launch_bounds__(kBlock) k_rowfold_then(const __grid_constant__
   __shared__ uint32_t folded[NFOLD];
   for (int r = blockIdx.x; r < a.R; r += gridDim.x) {     // a.R x a.C: the shape the folds reduce
     uint32_t acc[N];
+    float comp[N] = {};                                  // see fold_step
     static_for<0, N>([&](auto ic) {
       constexpr int i = decltype(ic)::value;
       constexpr CNode nd = CL::c.nodes[i];
@@ -360,9 +363,9 @@ __global__ void __launch_bounds__(kBlock) k_rowfold_then(const __grid_constant__
           const auto v = eval<CL, nd.in[0]>(a, ix);
           if constexpr (VEC) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) acc[i] = combine<nd.fn, nd.dtype>(acc[i], v.v[j]);
+            for (int j = 0; j < 4; ++j) fold_step<nd.fn, nd.dtype>(acc[i], comp[i], v.v[j]);
           } else {
-            acc[i] = combine<nd.fn, nd.dtype>(acc[i], v);
+            fold_step<nd.fn, nd.dtype>(acc[i], comp[i], v);
           }
         }
       });

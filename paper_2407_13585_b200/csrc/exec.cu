@@ -76,6 +76,61 @@ static dev::NodeArg node_arg(const Node& n, const void* ptr) {
   return a;
 }
 
+// The kernel instantiated for a cluster: for its very constants, else the one that takes them at run time.
+static const KernelEntry* lookup(CCluster& cc, std::string& sig) {
+  sig = signature(cc);
+  const KernelEntry* k = find_kernel(sig);
+  if (!k) {
+    for (int li = 0; li < cc.n; ++li)
+      if (cc.nodes[li].kind == ACC_BACKPERMUTE) cc.nodes[li].p0 = cc.nodes[li].p1 = kRunTime;
+    sig = signature(cc);
+    k = find_kernel(sig);
+  }
+  return k;
+}
+
+int refine_to_kernels(const Graph& g, std::vector<int32_t>& pi, int recompute_depth, int& splits) {
+  const int n = (int)g.nodes.size();
+  splits = 0;
+  for (;;) {
+    std::vector<uint8_t> man;
+    manifest_of(g, pi.data(), man);
+    std::map<int, std::vector<int>> clusters;
+    for (int i = 0; i < n; ++i)
+      if (!is_input(g.nodes[i])) clusters[pi[i]].push_back(i);
+    const std::vector<int>* bad = nullptr;
+    std::string sig;
+    for (auto& kv : clusters) {
+      CCluster cc;
+      if (!extract_runtime(g, kv.second, man, cc) || !lookup(cc, sig)) { bad = &kv.second; break; }
+    }
+    if (!bad) return ACC_OK;
+    if (bad->size() == 1)
+      return set_error(ACC_ERR_NO_KERNEL, "no kernel instantiated for node %d alone [%s]", bad->front(), sig.c_str());
+    // the latest member that may leave and still leave a legal clustering becomes a cluster of its own;
+    // failing that the whole cluster falls apart into its nodes
+    const int n_blocks = (int)clusters.size();
+    std::vector<int> block_of(pi.begin(), pi.end());
+    std::vector<int32_t> trial;
+    bool done = false;
+    for (auto it = bad->rbegin(); it != bad->rend() && !done; ++it) {
+      std::vector<int> b(block_of);
+      b[*it] = n_blocks;
+      done = canonical_numbering(g, b, n_blocks + 1, trial) && check_partition(g, trial.data(), nullptr, true, recompute_depth) == ACC_OK;
+    }
+    if (!done) {
+      std::vector<int> b(block_of);
+      int next = n_blocks;
+      for (size_t k = 1; k < bad->size(); ++k) b[(*bad)[k]] = next++;
+      if (!canonical_numbering(g, b, next, trial) || check_partition(g, trial.data(), nullptr, true, recompute_depth) != ACC_OK)
+        return set_error(ACC_ERR_NO_KERNEL, "the cluster at node %d has no kernel and cannot be split legally [%s]", bad->front(), sig.c_str());
+    }
+    clear_error();
+    pi = trial;
+    ++splits;
+  }
+}
+
 int build_schedule(Graph& g, int executor, Schedule& sch) {
   const int n = (int)g.nodes.size();
   sch = Schedule{};
@@ -120,14 +175,8 @@ int build_schedule(Graph& g, int executor, Schedule& sch) {
     st.n_members = (int)kv.second.size();
     if (!extract_runtime(g, kv.second, man, st.cc))
       return set_error(ACC_ERR_NO_KERNEL, "cluster at node %d has more than %d local nodes", st.first_node, kMaxCluster);
-    std::string sig = signature(st.cc);
-    st.kernel = find_kernel(sig);
-    if (!st.kernel) {                                   // none for these constants: the one that takes them at run time
-      for (int li = 0; li < st.cc.n; ++li)
-        if (st.cc.nodes[li].kind == ACC_BACKPERMUTE) st.cc.nodes[li].p0 = st.cc.nodes[li].p1 = kRunTime;
-      sig = signature(st.cc);
-      st.kernel = find_kernel(sig);
-    }
+    std::string sig;
+    st.kernel = lookup(st.cc, sig);
     if (!st.kernel)
       return set_error(ACC_ERR_NO_KERNEL, "no kernel instantiated for the cluster of %d nodes starting at node %d [%s]",
                        st.n_members, st.first_node, sig.c_str());

@@ -28,6 +28,8 @@ struct Schedule {
 };
 
 int build_schedule(Graph& g, int executor, Schedule& sch);
+// Splits clusters of `pi` that have no instantiated kernel until every cluster has one (see acc_refine_to_kernels).
+int refine_to_kernels(const Graph& g, std::vector<int32_t>& pi, int recompute_depth, int& splits);
 // `marks`, if given, receives one recorded event before the first launch and one after each launch
 int run_schedule(Graph& g, Schedule& sch, void* workspace, size_t ws_bytes, cudaStream_t stream,
                  std::vector<cudaEvent_t>* marks = nullptr);

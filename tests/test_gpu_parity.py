@@ -14,9 +14,9 @@ def np_inputs(inputs_t):
     return {k: v.cpu().numpy() for k, v in inputs_t.items()}
 
 
-def check_program(prog, partitions="all", runs=1, passes=False):
+def check_program(prog, partitions="all", runs=1, passes=False, inputs_t=None):
     from paper_2407_13585_b200 import binding as B
-    inputs_t = W.make_inputs(prog)
+    inputs_t = W.make_inputs(prog) if inputs_t is None else inputs_t
     ref = oracle_run(prog, np_inputs(inputs_t))
     got, g = gpu_run(prog, inputs_t, None, B.UNFUSED)
     assert g.launch_count() == sum(nd.kind != "input" for nd in prog.nodes)
@@ -169,6 +169,35 @@ def test_row_scans_consumed_inside_their_cluster(rows, n):
 @pytest.mark.parametrize("n", [1, 4, 4096, 1 << 17])
 def test_offsets_used_as_indices_in_the_same_cluster(n):
     assert check_program(W.offsets_then_gather(n), passes=True) == 20
+
+
+def test_a_plan_without_kernels_is_refined_and_runs():
+    from paper_2407_13585_b200 import binding as B
+    for n in (1, 4099, 70000):
+        prog = W.fold_of_scan(n)
+        g = B.Graph(prog.nodes, prog.outputs)
+        g.plan("enumerate", "bytes")
+        splits, pi = g.refine_to_kernels()
+        assert (splits, pi) == (1, [-1, 0, 1])
+        check_program(prog, [pi])
+
+
+def test_equal_addends_stay_within_tolerance():
+    # rounding errors of a running fp32 sum cancel on random data and pile up when every addend is the same
+    # number: the per-thread sums are compensated, so long folds, row folds, segmented folds and scans of a
+    # constant still meet 1e-5 * sum|x|
+    import torch
+    from paper_2407_13585_b200 import binding as B
+
+    def constant(prog, value=0.1):
+        inputs = W.make_inputs(prog)
+        return {i: (torch.full_like(t, value) if t.dtype == torch.float32 else t) for i, t in inputs.items()}
+
+    for prog in (W.config1(1 << 22), W.greedy_bottom_up_bad(4, 1 << 20), W.segmented_sums(1 << 20, 16),
+                 W.scan_consumers(1 << 22), W.scan_consumers(1 << 20, 4)):
+        g = B.Graph(prog.nodes, prog.outputs)
+        pi = g.plan("enumerate", "bytes")
+        check_program(prog, [pi], passes=True, inputs_t=constant(prog))
 
 
 def test_runs_are_repeatable():

@@ -386,3 +386,22 @@ def test_generated_sources_match_their_programs():
         finally:
             instantiate.sys.stdout = stdout
         assert out.getvalue() == text, f
+
+
+def test_refine_to_kernels_splits_only_clusters_nobody_built():
+    # the cheapest clustering of a fold of a scan is one cluster, which no kernel walks: the fold leaves it
+    prog = W.fold_of_scan(64)
+    g = B.Graph(prog.nodes, prog.outputs)
+    assert g.plan("enumerate", "bytes") == [-1, 0, 0]
+    assert g.refine_to_kernels() == (1, [-1, 0, 1])
+    assert g.refine_to_kernels() == (0, [-1, 0, 1])
+    assert L.check(prog.nodes, prog.outputs, [-1, 0, 1])
+    # plans whose clusters all have kernels stay as they are
+    for prog in (W.config1(64), W.config2(8), W.config3(64), W.config5(256, 16), W.scan_consumers(16)):
+        g = B.Graph(prog.nodes, prog.outputs)
+        pi = g.plan("enumerate", "bytes")
+        assert g.refine_to_kernels() == (0, pi)
+    # without a clustering there is nothing to refine
+    g = B.Graph(prog.nodes, prog.outputs)
+    with pytest.raises(B.AccError):
+        g.refine_to_kernels()

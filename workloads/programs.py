@@ -352,6 +352,16 @@ def offsets_then_gather(n=1 << 12):
     return Program("offsets_then_gather", nodes, [5, 6], index_bound={"x": 1 << 30, "src": 1 << 30})
 
 
+def fold_of_scan(n=4099):
+    """The largest prefix sum: a fold that consumes a scan.  Legal as one cluster; no kernel walks it so."""
+    nodes = [
+        _inp("x", "f32", (n,)),
+        Node("scanl", "f32", (n,), (0,), 1, fn="add", name="s"),
+        Node("fold", "f32", (), (1,), 1, fn="max", name="f"),
+    ]
+    return Program("fold_of_scan", nodes, [2])
+
+
 CONFIGS = {1: config1, 2: config2, 3: config3, 4: config4, 5: config5}
 
 
