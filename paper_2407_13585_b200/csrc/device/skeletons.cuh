@@ -395,15 +395,30 @@ __global__ void __launch_bounds__(kBlock) k_rowfold_then(const __grid_constant__
 
 // =========================================================================================
 // Scratch layout of k_scan: word [0] ticket; from byte 16 one 64-bit tile state per tile:
-// (flag << 32) | value, flag 0 = nothing yet, 1 = the tile's own total, 2 = inclusive prefix.
+// (value << 32) | low, the two lowest bits of `low` being the flag: 0 = nothing yet, 1 = the tile's
+// own total, 2 = inclusive prefix.  The prefix of an fp32 sum is carried as two floats, hi in `value`
+// and lo (its two lowest mantissa bits dropped) in the rest of `low`: the chain of tile prefixes is a
+// running sum over up to 2^31 / 4096 tiles, and in plain fp32 its rounding errors pile up on inputs
+// where they do not cancel.
 constexpr int kScanRows = 4;                     // 128-bit chunks per thread
-constexpr uint64_t kFlagAggregate = 1, kFlagPrefix = 2;
+constexpr uint32_t kFlagAggregate = 1, kFlagPrefix = 2;
 
 __device__ __forceinline__ uint64_t ld_state(const uint64_t* p) {
   return *reinterpret_cast<const volatile uint64_t*>(p);
 }
-__device__ __forceinline__ void st_state(uint64_t* p, uint64_t flag, uint32_t v) {
-  *reinterpret_cast<volatile uint64_t*>(p) = (flag << 32) | v;
+__device__ __forceinline__ void st_state(uint64_t* p, uint32_t flag, uint32_t v, uint32_t low = 0u) {
+  *reinterpret_cast<volatile uint64_t*>(p) = ((uint64_t)v << 32) | (low & ~3u) | flag;
+}
+__device__ __forceinline__ uint32_t flag_of(uint64_t s) { return (uint32_t)s & 3u; }
+__device__ __forceinline__ uint32_t value_of(uint64_t s) { return (uint32_t)(s >> 32); }
+// hi + lo of a state of an fp32 sum (lo is zero for a tile's own total)
+__device__ __forceinline__ double wide_of(uint64_t s) {
+  return (double)__uint_as_float(value_of(s)) + (double)__uint_as_float((uint32_t)s & ~3u);
+}
+__device__ __forceinline__ void st_wide(uint64_t* p, double prefix) {
+  const float hi = (float)prefix;
+  const float lo = isfinite(hi) ? (float)(prefix - (double)hi) : 0.0f;     // an overflowed sum stays infinite
+  st_state(p, kFlagPrefix, __float_as_uint(hi), __float_as_uint(lo));
 }
 
 // stores at a descending chunk: the lanes go back into ascending memory order
@@ -529,6 +544,7 @@ __global__ void __launch_bounds__(kBlock) k_scan(const __grid_constant__ Args<CL
     }
 
     if (warp == 0) {
+      constexpr bool WIDE = FN == ACC_FN_ADD && DT == ACC_F32;
       uint32_t exclusive = identity_of<FN, DT>();
       if (in_row == 0) {
         if (lane == 0) st_state(states + tile, kFlagPrefix, tile_total);
@@ -537,27 +553,40 @@ __global__ void __launch_bounds__(kBlock) k_scan(const __grid_constant__ Args<CL
         int look = in_row - 1;                             // tiles of this row before this one
         uint32_t spins = 0;
         bool gave_up = false;
+        double wide = 0.0;                                 // WIDE: the sum of the tiles before this one
         for (;;) {
           const int idx = look - lane;
           const uint64_t* at = states + (tile - in_row) + idx;
-          uint64_t s = idx >= 0 ? ld_state(at) : (kFlagPrefix << 32) | identity_of<FN, DT>();
-          while (__any_sync(0xFFFFFFFFu, (s >> 32) == 0)) {
+          uint64_t s = idx >= 0 ? ld_state(at) : ((uint64_t)identity_of<FN, DT>() << 32) | kFlagPrefix;
+          while (__any_sync(0xFFFFFFFFu, flag_of(s) == 0)) {
             if (++spins > a.spin_limit) { gave_up = true; break; }
             __nanosleep(20);
             if (idx >= 0) s = ld_state(at);
           }
           if (gave_up) break;
-          const unsigned done = __ballot_sync(0xFFFFFFFFu, (s >> 32) == kFlagPrefix);
+          const unsigned done = __ballot_sync(0xFFFFFFFFu, flag_of(s) == kFlagPrefix);
           const int stop = done ? __ffs(done) - 1 : 31;
-          uint32_t part = lane <= stop ? (uint32_t)s : identity_of<FN, DT>();
+          if constexpr (WIDE) {
+            double part = lane <= stop ? wide_of(s) : 0.0;
 #pragma unroll
-          for (int o = 16; o > 0; o >>= 1) part = combine<FN, DT>(part, __shfl_xor_sync(0xFFFFFFFFu, part, o));
-          exclusive = combine<FN, DT>(part, exclusive);
+            for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
+            wide += part;
+          } else {
+            uint32_t part = lane <= stop ? value_of(s) : identity_of<FN, DT>();
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) part = combine<FN, DT>(part, __shfl_xor_sync(0xFFFFFFFFu, part, o));
+            exclusive = combine<FN, DT>(part, exclusive);
+          }
           if (done) break;
           look -= 32;
         }
         if (gave_up && lane == 0) atomicOr(a.status, kStatusTimeout);
-        if (lane == 0) st_state(states + tile, kFlagPrefix, combine<FN, DT>(exclusive, tile_total));
+        if constexpr (WIDE) {
+          exclusive = u_((float)wide);
+          if (lane == 0) st_wide(states + tile, wide + (double)f_(tile_total));
+        } else {
+          if (lane == 0) st_state(states + tile, kFlagPrefix, combine<FN, DT>(exclusive, tile_total));
+        }
       }
       if (lane == 0) tile_prefix = exclusive;
     }
