@@ -392,7 +392,7 @@ def run_ours(args):
              5: "k_hist<hash+generate+permute+fold>", 1: "k_stream<chain>"}
     # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
     # summarised under profiles/, taken at these sizes; null for a kernel without a capture
-    ncu_traffic = {3: 6.267e9 + 0.2570e9, 4: 268.5e6 + 217.4e6, 2: 270.8e6 + 6.6e6, 5: 542.6e6 + 3.6e6}
+    ncu_traffic = {3: 6.267e9 + 0.2590e9, 4: 268.5e6 + 217.4e6, 2: 270.8e6 + 6.6e6, 5: 542.6e6 + 3.6e6}
     traffic = ncu_traffic.get(top) if args.shrink == 0 else None
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": traffic, "kernel": names[top], "of": peak_kind,
