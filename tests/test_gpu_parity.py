@@ -200,6 +200,40 @@ def test_equal_addends_stay_within_tolerance():
         check_program(prog, [pi], passes=True, inputs_t=constant(prog))
 
 
+# random DAGs around a scan in the middle.  Clusterings in which something other than an element-wise chain reads
+# the scan inside its cluster (a reversal, a fold, a second scan) have no kernel: the run must say so, not guess
+def around_a_scan(prog):
+    from paper_2407_13585_b200 import binding as B
+    from paper_2407_13585_b200 import instantiate
+    built, missing = [], []
+    for pi in all_partitions(prog):
+        blocks = {}
+        for i, c in enumerate(pi):
+            if c >= 0:
+                blocks.setdefault(c, set()).add(i)
+        (built if all(instantiate.expressible(prog, b) for b in blocks.values()) else missing).append(pi)
+    assert built
+    check_program(prog, built, passes=True)
+    inputs_t = W.make_inputs(prog)
+    for pi in missing:
+        with pytest.raises(B.AccError) as err:
+            gpu_run(prog, inputs_t, pi, B.FUSED)
+        assert err.value.status == "ACC_ERR_NO_KERNEL"
+    return len(missing)
+
+
+@pytest.mark.parametrize("n", [1, 4099, 70000])
+@pytest.mark.parametrize("seed", [1, 3, 4, 7, 10, 13, 14])
+def test_random_programs_around_a_scan(seed, n):
+    assert (around_a_scan(W.random_scan_program(seed, n)) > 0) == (seed in (4, 7, 10, 14))
+
+
+@pytest.mark.parametrize("rows,n", [(3, 5), (37, 1024)])
+@pytest.mark.parametrize("seed", [4, 7, 12])
+def test_random_rank2_programs_around_a_scan(seed, rows, n):
+    around_a_scan(W.random_scan_program(seed, n, rows))
+
+
 def test_runs_are_repeatable():
     # a racy fold, scan or scatter would differ between runs; integer outputs must be identical
     check_program(W.config3(1 << 16), runs=3)

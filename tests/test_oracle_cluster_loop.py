@@ -62,6 +62,8 @@ def test_both_evaluators_agree_on_random_programs(seed):
     agree_everywhere(W.random_int_program(seed, 37), max_partitions=40)
     agree_everywhere(W.random_int_program(seed, 9, 4), max_partitions=30)
     agree_everywhere(W.random_int_program(seed + 10, 6, 6), max_partitions=30)      # square: with transposes
+    agree_everywhere(W.random_scan_program(seed, 37), max_partitions=40)            # a scan in the middle, with readers
+    agree_everywhere(W.random_scan_program(seed, 9, 4), max_partitions=30)
 
 
 def test_config1_full_size_all_clusterings():

@@ -318,6 +318,59 @@ def diagonal_of_product(rows=256):
     return Program("diagonal_of_product", nodes, [4])
 
 
+def random_scan_program(seed, n=4099, rows=0):
+    """A seeded random DAG around a scan in the middle: element-wise nodes and reversals before it, then nodes
+    that may read the scan (directly, or through a reversal, which no kernel follows inside a cluster), then
+    possibly a fold or a second scan of any of them.  rows = 0: rank 1."""
+    from .inputs import counter_bits
+    shape = (n,) if not rows else (rows, n)
+    draws = iter(counter_bits(seed, 61, 96).tolist())
+
+    def pick(k):
+        return ((next(draws) & ((1 << 63) - 1)) >> 20) % k
+
+    nodes = [_inp("x", "f32", shape), _inp("v", "f32", shape)]
+    arrays = [0, 1]
+    affine = [(2.0, 1.0), (-0.5, 0.25), (1.0, -3.0), (0.125, 0.0)]
+
+    def add(node):
+        nodes.append(node)
+        node.name = "%s%d" % (node.kind[0], len(nodes) - 1)
+        arrays.append(len(nodes) - 1)
+        return len(nodes) - 1
+
+    def some():
+        return arrays[pick(len(arrays))]
+
+    def element_wise():
+        k = pick(4)
+        if k == 0:
+            add(Node("map", "f32", shape, (some(),), 1, fn="affine", fparam=affine[pick(4)]))
+        elif k in (1, 2):
+            add(Node("zipwith", "f32", shape, (some(), some()), 2, fn=("add", "mul")[pick(2)]))
+        else:
+            add(Node("backpermute", "f32", shape, (some(),), 1, idx_fn="reverse"))
+
+    for _ in range(1 + pick(2)):
+        element_wise()
+    kind, fn = ("scanl", "scanr")[pick(2)], ("add", "max")[pick(2)]
+    if pick(3) == 0:
+        scan = add(Node(kind, "f32", shape, (some(),), 1, fn=fn, fparam=(0.5,), exclusive=True))
+    else:
+        scan = add(Node(kind, "f32", shape, (some(),), 1, fn=fn))
+    add(Node("map", "f32", shape, (scan,), 1, fn="affine", fparam=affine[pick(4)]))      # at least one reader
+    for _ in range(1 + pick(2)):
+        element_wise()
+    k = pick(3)
+    if k == 1:
+        add(Node("fold", "f32", shape[:-1], (some(),), 1, fn="add"))
+    elif k == 2:
+        add(Node("scanl", "f32", shape, (some(),), 1, fn="add"))
+    used = {s for nd in nodes for s in nd.inputs}
+    outputs = [i for i, nd in enumerate(nodes) if nd.kind != "input" and i not in used]
+    return Program("random_scan%s_%d" % ("2d" if rows else "", seed), nodes, outputs)
+
+
 def scan_consumers(n=4099, rows=None):
     """Scans whose values feed element-wise nodes: a running sum that is only consumed (never an output), a
     right-to-left running maximum that is both written and consumed, and a seeded exclusive sum."""
