@@ -234,6 +234,14 @@ def test_random_rank2_programs_around_a_scan(seed, rows, n):
     around_a_scan(W.random_scan_program(seed, n, rows))
 
 
+# a scatter histogram over rank-2 keys beside per-row totals: few elements per bin (atomics on global accumulators)
+# and many (bins in shared memory, also with the private overflow slice); fused with the row folds, the scatter
+# and the folds take a pass each
+@pytest.mark.parametrize("rows,n,bins", [(1, 1, 1), (3, 5, 4), (37, 300, 16), (64, 4096, 256), (256, 4096, 1 << 16)])
+def test_rank2_histogram_beside_row_totals(rows, n, bins):
+    assert check_program(W.histogram_2d(rows, n, bins), passes=True) == 10
+
+
 def test_runs_are_repeatable():
     # a racy fold, scan or scatter would differ between runs; integer outputs must be identical
     check_program(W.config3(1 << 16), runs=3)

@@ -35,7 +35,8 @@ def test_library_exports_every_declared_symbol():
 PROGRAMS = [W.config1(64), W.config2(8), W.config3(64), W.config4(8, 8, iters=1), W.config5(256, 16),
             W.scatter_example(16), W.scatter_example_paper_graph(), W.single_loop(16), W.simple1(), W.simple2(),
             W.simple3(), W.simple4(), W.simple5(), W.greedy_bottom_up_bad(4, 5), W.greedy_top_down_bad(16),
-            W.segmented_sums(64, 5), W.scan_consumers(16), W.scan_consumers(8, 3), W.offsets_then_gather(16)] + [W.random_program(s, 16) for s in range(14)] + [W.random_program(s, 8, 3) for s in (0, 3, 5, 8)] + [
+            W.segmented_sums(64, 5), W.scan_consumers(16), W.scan_consumers(8, 3), W.offsets_then_gather(16),
+            W.histogram_2d(4, 16, 8), W.fold_of_scan(16)] + [W.random_program(s, 16) for s in range(14)] + [W.random_program(s, 8, 3) for s in (0, 3, 5, 8)] + [
                 W.random_int_program(s, 16) for s in range(12)] + [W.random_int_program(s, 8, 3) for s in range(12)] + [W.random_int_program(s, 6, 6) for s in (2, 3, 7, 14, 16, 17, 20, 23, 31, 39)] + [
                 W.random_scan_program(s, 16) for s in range(16)] + [W.random_scan_program(s, 8, 3) for s in (4, 7, 12)]
 
@@ -375,8 +376,9 @@ def test_generated_sources_match_their_programs():
     import glob, io, os, re
     from paper_2407_13585_b200 import instantiate
     here = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "paper_2407_13585_b200", "csrc", "programs")
-    files = sorted(glob.glob(os.path.join(here, "prog_random*.cu")) + glob.glob(os.path.join(here, "prog_scan_consumers*.cu")))
-    assert len(files) >= 17
+    files = sorted(glob.glob(os.path.join(here, "prog_random*.cu")) + glob.glob(os.path.join(here, "prog_scan_consumers*.cu")) +
+                   glob.glob(os.path.join(here, "prog_histogram_2d.cu")))
+    assert len(files) >= 18
     for f in files:
         text = open(f).read()
         argv = re.match(r"// Generated by `python -m paper_2407_13585_b200.instantiate (.*)`\.", text).group(1).split()

@@ -47,7 +47,7 @@ def agree_everywhere(p, max_partitions=None):
     (W.scatter_example(24), None), (W.single_loop(33), None), (W.simple1(), 2), (W.simple2(), 2),
     (W.simple3(), 1), (W.simple4(), 2), (W.simple5(), None), (W.greedy_bottom_up_bad(3, 5), None),
     (W.greedy_top_down_bad(17), None), (W.config4(5, 6, iters=1), None), (W.segmented_sums(200, 9), None),
-    (W.scan_consumers(41), None), (W.scan_consumers(7, 3), None), (W.offsets_then_gather(64), 20)])
+    (W.scan_consumers(41), None), (W.scan_consumers(7, 3), None), (W.offsets_then_gather(64), 20), (W.histogram_2d(4, 16, 8), 10), (W.fold_of_scan(33), None)])
 def test_both_evaluators_agree_on_every_legal_clustering(prog, count):
     n = agree_everywhere(prog, max_partitions=40)
     if count is not None:

@@ -130,6 +130,8 @@ def make_inputs(program, seed=0, device="cpu"):
             t = normal_f32(seed, st, cnt, device=device)
         elif name == "config5" and nd.name == "keys":
             t = zipf_keys(seed, st, cnt, device=device)
+        elif name == "histogram_2d" and nd.name == "zeros":
+            t = torch.zeros(cnt, dtype=torch.float32, device=device)
         elif name == "config5" and nd.name == "zeros":
             t = torch.zeros(cnt, dtype=torch.float32, device=device)
         elif nd.dtype == "f32":

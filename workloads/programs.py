@@ -405,6 +405,21 @@ def offsets_then_gather(n=1 << 12):
     return Program("offsets_then_gather", nodes, [5, 6], index_bound={"x": 1 << 30, "src": 1 << 30})
 
 
+def histogram_2d(rows=64, n=4096, bins=256):
+    """The scatter histogram of config 5 over a rank-2 array of keys, with per-row totals beside it: the
+    scatter and the row folds share producers but no kernel walk."""
+    sh = (rows, n)
+    nodes = [
+        _inp("keys", "u32", sh),
+        _inp("zeros", "f32", (bins,)),
+        Node("map", "u32", sh, (0,), 1, fn="mul_mod", iparam=(40503, bins), name="k"),
+        Node("generate", "f32", sh, (), 0, fn="imod_to_f32", iparam=(7,), name="vals"),
+        Node("permute", "f32", (bins,), (1, 2, 3), 3, fn="add", name="hist"),
+        Node("fold", "f32", (rows,), (3,), 1, fn="add", name="row_totals"),
+    ]
+    return Program("histogram_2d", nodes, [4, 5], index_bound={"keys": 1 << 20})
+
+
 def fold_of_scan(n=4099):
     """The largest prefix sum: a fold that consumes a scan.  Legal as one cluster; no kernel walks it so."""
     nodes = [
