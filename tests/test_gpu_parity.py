@@ -242,6 +242,24 @@ def test_rank2_histogram_beside_row_totals(rows, n, bins):
     assert check_program(W.histogram_2d(rows, n, bins), passes=True) == 10
 
 
+def test_launches_count_the_passes_of_a_cluster():
+    from paper_2407_13585_b200 import binding as B
+    # {s, m, z, e, t}: two scans, a pass each; {r, q}: one kernel
+    prog = W.scan_consumers(4099)
+    _, g = gpu_run(prog, W.make_inputs(prog), [-1, -1, 0, 0, 0, 1, 1, 0, 0], B.FUSED)
+    assert g.launch_count() == 3
+    # everything in one cluster on a rank-2 domain: the row folds, then the scatter
+    prog = W.histogram_2d(37, 300, 16)
+    _, g = gpu_run(prog, W.make_inputs(prog), [-1, -1, 0, 0, 0, 0], B.FUSED)
+    assert g.launch_count() == 2
+    # whole-array folds and a scatter share the streaming kernel: config 5 fused stays one launch (+ the map of the total)
+    prog = W.config5(1 << 15, 256)
+    g0 = B.Graph(prog.nodes, prog.outputs)
+    pi = g0.plan("enumerate", "bytes")
+    _, g = gpu_run(prog, W.make_inputs(prog), pi, B.FUSED)
+    assert g.launch_count() == len({c for c in pi if c >= 0})
+
+
 def test_runs_are_repeatable():
     # a racy fold, scan or scatter would differ between runs; integer outputs must be identical
     check_program(W.config3(1 << 16), runs=3)
