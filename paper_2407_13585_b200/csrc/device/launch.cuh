@@ -20,7 +20,8 @@ struct Launcher {
   static constexpr bool kHasScan = dev::count_if<CL>(dev::is_scan_root) > 0;
   static constexpr bool kHasRowFold = dev::count_if<CL>(dev::is_row_fold) > 0;
   static constexpr int kScalarFolds = dev::count_if<CL>(dev::is_scalar_fold);
-  static constexpr int kScanTile = dev::kBlock * 16;
+  static constexpr int kScanBlock = dev::scan_block<CL>();
+  static constexpr int kScanTile = kScanBlock * dev::scan_rows<CL>() * 4;
   static constexpr bool kHasSegFold = dev::count_if<CL>(dev::is_segfold_root) > 0;
   // exactly one scatter, fp32 '+': its bins can live in shared memory (k_hist)
   static constexpr bool kHistShape = !kHasScan && !kHasRowFold && dev::count_if<CL>(dev::is_permute_root) == 1 &&
@@ -295,9 +296,9 @@ struct Launcher {
       const int per_row = (C + kScanTile - 1) / kScanTile;
       const int64_t tiles = (int64_t)R * per_row;
       if (tiles >= (int64_t(1) << 31)) return set_error(ACC_ERR_SHAPE, "too many rows to scan in one launch");
-      const int grid = (int)std::min<int64_t>(tiles, (int64_t)sm_count() * 6);
-      if (vec) dev::k_scan<CL, true><<<grid, dev::kBlock, 0, L.stream>>>(a, per_row, (int)tiles);
-      else dev::k_scan<CL, false><<<grid, dev::kBlock, 0, L.stream>>>(a, per_row, (int)tiles);
+      const int grid = (int)std::min<int64_t>(tiles, (int64_t)sm_count() * (1536 / kScanBlock));
+      if (vec) dev::k_scan<CL, true><<<grid, kScanBlock, 0, L.stream>>>(a, per_row, (int)tiles);
+      else dev::k_scan<CL, false><<<grid, kScanBlock, 0, L.stream>>>(a, per_row, (int)tiles);
     } else if constexpr (kHasRowFold) {
       if (R == 0) return ACC_OK;
       const int grid = std::min(R, sm_count() * 16);

@@ -25,8 +25,8 @@ namespace acc {
 namespace {
 
 constexpr int64_t kMaxElements = ACC_STATIC_SCAN_MAX_ELEMENTS;
-constexpr int kTile = dev::kBlock * 16;
-constexpr int64_t kMaxTiles = (kMaxElements + kTile - 1) / kTile;
+constexpr int kSmallestTile = 256 * 16;                   // the static array holds a state per tile of the smallest tile shape
+constexpr int64_t kMaxTiles = (kMaxElements + kSmallestTile - 1) / kSmallestTile;
 constexpr size_t kHeaderBytes = 256;                      // status word, padded
 constexpr size_t kScratchBytes = kHeaderBytes + 16 + (size_t)kMaxTiles * 8;
 
@@ -80,6 +80,9 @@ extern "C" int acc_scanl_add_i32_static(const int32_t* in, int32_t* out, int64_t
   int rc = scratch_for_current_device(&base);
   if (rc != ACC_OK) return rc;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  constexpr int kScanBlock = dev::scan_block<ScanCluster>();
+  constexpr int kTile = kScanBlock * dev::scan_rows<ScanCluster>() * 4;
+  static_assert(kTile >= kSmallestTile, "the static tile states are sized for tiles of at least 4096 elements");
   const int tiles = (int)((n + kTile - 1) / kTile);
   // the array keeps whatever the previous call left: status, ticket and the states in use start at zero
   cudaError_t e = cudaMemsetAsync(base, 0, kHeaderBytes + 16 + (size_t)tiles * 8, stream);
@@ -99,9 +102,10 @@ extern "C" int acc_scanl_add_i32_static(const int32_t* in, int32_t* out, int64_t
   a.spin_limit = 1u << 22;
   a.grid = 0;
   const bool vec = n % 4 == 0 && ((reinterpret_cast<uintptr_t>(in) | reinterpret_cast<uintptr_t>(out)) & 15) == 0;
-  const int grid = tiles < sm_count() * 6 ? tiles : sm_count() * 6;
-  if (vec) dev::k_scan<ScanCluster, true><<<grid, dev::kBlock, 0, stream>>>(a, tiles, tiles);
-  else dev::k_scan<ScanCluster, false><<<grid, dev::kBlock, 0, stream>>>(a, tiles, tiles);
+  const int resident = sm_count() * (1536 / kScanBlock);
+  const int grid = tiles < resident ? tiles : resident;
+  if (vec) dev::k_scan<ScanCluster, true><<<grid, kScanBlock, 0, stream>>>(a, tiles, tiles);
+  else dev::k_scan<ScanCluster, false><<<grid, kScanBlock, 0, stream>>>(a, tiles, tiles);
   e = cudaGetLastError();
   if (e != cudaSuccess) return set_error(ACC_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
   uint32_t status = 0;
