@@ -329,14 +329,15 @@ int acc_last_schedule(const acc_graph* g, char* buf, size_t cap);
  * the scan kernel, not a combinator or a rule of its own.)
  *
  * Who needs it: code that may not allocate device memory where it calls us --
- * a serving or real-time loop in which cudaMalloc's implicit device-wide
- * synchronisation is unacceptable, a plug-in or callback that receives raw
- * device pointers but no allocator, a process whose memory budget is fixed
- * up front.  acc_run needs a caller-allocated workspace for the scan's tile
- * states; this entry point keeps them in a fixed array inside the library's
- * device image instead (about 128 KiB, resident on every GPU that loads the
- * library until the process exits) and calls no cudaMalloc, cudaFree or any
- * other allocating routine.
+ * a plug-in or callback that receives raw device pointers but no allocator, a
+ * process whose device-memory budget is fixed up front and fully handed out,
+ * a component that must not call cudaMalloc or cudaFree because other work
+ * shares the device with it.  acc_run needs a caller-allocated workspace for
+ * the scan's tile states; this entry point keeps them in a fixed array inside
+ * the library's device image instead (about 128 KiB, resident on every GPU
+ * that loads the library until the process exits) and calls no cudaMalloc,
+ * cudaFree or any other allocating routine.  It is not a low-latency call:
+ * it blocks the host until the scan has finished (see below).
  *
  *   in, out      DEVICE pointers to n int32 each, owned by the caller, not
  *                overlapping; 16-byte alignment and n % 4 == 0 select the
@@ -346,10 +347,12 @@ int acc_last_schedule(const acc_graph* g, char* buf, size_t cap);
  *   cuda_stream  a cudaStream_t of the current device (null = default stream).
  *
  * The call enqueues a clear of the part of the array it uses and the scan, then
- * WAITS for the stream and returns ACC_OK, ACC_ERR_DEVICE_TIMEOUT (a bounded
- * wait between tiles ran out; out is then not valid) or ACC_ERR_CUDA.
- * The first call on each device looks up the array's device address (with
- * that device current); make that first call outside any stream capture.
+ * BLOCKS THE HOST until the stream has finished (it copies the status word
+ * back and synchronises the stream) and returns ACC_OK, ACC_ERR_DEVICE_TIMEOUT
+ * (a bounded wait between tiles ran out; out is then not valid) or
+ * ACC_ERR_CUDA.  Because of that copy and wait, never call it on a stream that
+ * is being captured.  The first call on each device also looks up the array's
+ * device address (with that device current).
  * All calls on one GPU share the one array, which keeps the previous call's
  * contents between calls: two calls whose work overlaps on the same GPU
  * (different streams or threads) race on it and give undefined results --

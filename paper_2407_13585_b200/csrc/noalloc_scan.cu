@@ -3,9 +3,10 @@
 //
 // The regular path takes its tile states and its ticket counter from the caller's workspace,
 // which the caller obtains with cudaMalloc or a framework allocator.  Some callers cannot do
-// that at the point of the call: code running inside a region where device allocation is
-// forbidden or would synchronise the device (a latency-critical serving loop, a callback, a
-// plug-in that was given raw pointers and no allocator).  For them the scratch lives in a
+// that at the point of the call: code running where device allocation is forbidden (a callback
+// or plug-in that was given raw pointers and no allocator, a process whose device memory was
+// handed out completely up front).  The call itself still blocks the host until the scan has
+// finished, so it must never run on a capturing stream.  For such callers the scratch lives in a
 // file-scope device array of fixed size that every GPU loading this library holds until the
 // process exits; the caller passes only the input and the output.
 //

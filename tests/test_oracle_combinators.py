@@ -343,3 +343,126 @@ def test_diagonal_of_a_product_against_matmul():
     bound = 2.0 ** -24 * np.einsum("ij,ji->i", np.abs(a), np.abs(b)) + 1e-12
     assert (np.abs(res.exact[4] - want) <= bound).all()
     assert (np.abs(res.values[4] - want) <= bound + 2.0 ** -24 * np.abs(want)).all()
+
+
+# ---- element functions and operators that no benchmark configuration pins -------------------------
+# Expected values below are worked by hand from Section 2's definitions (generate: ys[i] = f(i);
+# map: ys[i] = f(xs[i]); fold / scan / scatter with an operator other than +).  Integer cases mix
+# signs so that an unsigned comparison where a signed one is meant (or the reverse) gives another answer.
+
+def test_generate_functions_worked():
+    # row_index on a 2 x 3 array: the row of every element; iota on rank 2 counts row-major
+    nodes = [Node("generate", "i32", (2, 3), (), 0, fn="row_index"), Node("generate", "i32", (2, 3), (), 0, fn="iota"),
+             Node("generate", "f32", (2, 3), (), 0, fn="iota")]
+    v = run(nodes, {})
+    assert v[0].tolist() == [[0, 0, 0], [1, 1, 1]]
+    assert v[1].tolist() == [[0, 1, 2], [3, 4, 5]] and v[2].tolist() == [[0.0, 1.0, 2.0], [3.0, 4.0, 5.0]]
+    # iota_plus_free: float(i) + the scalar read from a free-variable slot (element 0 of that array)
+    nodes = [_inp("t", "f32", ()), Node("generate", "f32", (4,), (0,), 0, fn="iota_plus_free")]
+    assert run(nodes, {0: np.array(2.5, F32)})[1].tolist() == [2.5, 3.5, 4.5, 5.5]
+    assert run(nodes, {0: np.array(-1.0, F32)})[1].tolist() == [-1.0, 0.0, 1.0, 2.0]
+    # imod_to_f32: float(i mod m)
+    nodes = [Node("generate", "f32", (9,), (), 0, fn="imod_to_f32", iparam=(7,))]
+    assert run(nodes, {})[0].tolist() == [0, 1, 2, 3, 4, 5, 6, 0, 1]
+
+
+def test_unary_and_free_variable_functions_worked():
+    x = np.array([1.0, 2.0, -4.0], F32)
+    nodes = [_inp("x", "f32", (3,)), _inp("t", "f32", ()),
+             Node("map", "f32", (3,), (0, 1), 1, fn="add_free"), Node("map", "f32", (3,), (0, 1), 1, fn="div_free"),
+             Node("map", "f32", (3,), (0,), 1, fn="identity"),
+             Node("zipwith", "f32", (3,), (0, 0, 2), 3, fn="add3"),
+             Node("zipwith", "f32", (3,), (0, 2), 2, fn="add_scale", fparam=(0.5,))]
+    v = run(nodes, {0: x, 1: np.array(0.5, F32)})
+    assert v[2].tolist() == [1.5, 2.5, -3.5]                   # x + t
+    assert v[3].tolist() == [2.0, 4.0, -8.0]                   # x / t
+    assert v[4].tolist() == [1.0, 2.0, -4.0]
+    assert v[5].tolist() == [3.5, 6.5, -11.5]                  # (x + x) + (x + t)
+    assert v[6].tolist() == [1.25, 2.25, -3.75]                # 0.5 * (x + (x + t))
+    # integer constants act on the 32-bit pattern and wrap
+    xi = np.array([3, -2, 2**31 - 1], I32)
+    nodes = [_inp("x", "i32", (3,)), Node("map", "i32", (3,), (0,), 1, fn="mul_const", iparam=(5,)),
+             Node("map", "i32", (3,), (0,), 1, fn="add_const", iparam=(1,)),
+             Node("map", "i32", (3,), (0,), 1, fn="add_const", iparam=(-7,)),
+             Node("map", "i32", (3,), (0,), 1, fn="mul_const", iparam=(-1,))]
+    v = {k: interp.to_external(a, "i32") for k, a in run(nodes, {0: xi}).items()}
+    assert v[1].tolist() == [15, -10, 2147483643]              # (2^31 - 1) * 5 = 2 * 2^32 + 2147483643
+    assert v[2].tolist() == [4, -1, -2**31]
+    assert v[3].tolist() == [-4, -9, 2**31 - 8]
+    assert v[4].tolist() == [-3, 2, -(2**31 - 1)]
+
+
+def test_folds_with_other_operators_worked():
+    x = np.array([[1, -2, 3], [0.5, 4, -1]], F32)
+    mk = lambda op: Node("fold", "f32", (2,), (0,), 1, fn=op)
+    v = run([_inp("x", "f32", (2, 3)), mk("mul"), mk("min"), mk("max")], {0: x})
+    assert v[1].tolist() == [-6.0, -2.0] and v[2].tolist() == [-2.0, -1.0] and v[3].tolist() == [3.0, 4.0]
+    xi = np.array([[-3, 2, 7], [5, -1, -8]], I32)
+    mk = lambda op: Node("fold", "i32", (2,), (0,), 1, fn=op)
+    v = {k: interp.to_external(a, "i32") for k, a in run([_inp("x", "i32", (2, 3)), mk("mul"), mk("min"), mk("max")], {0: xi}).items()}
+    assert v[1].tolist() == [-42, 40]
+    assert v[2].tolist() == [-3, -8]                           # compared as unsigned patterns these would be 2 and 5
+    assert v[3].tolist() == [7, 5]                             # ... and these -3 and -1
+    # the same bit patterns declared unsigned compare the other way round
+    mk = lambda op: Node("fold", "u32", (2,), (0,), 1, fn=op)
+    v = run([_inp("x", "u32", (2, 3)), mk("min"), mk("max")], {0: xi.view(U32)})
+    assert v[1].tolist() == [2, 5] and v[2].tolist() == [2**32 - 3, 2**32 - 1]
+    # products wrap: 65536 * 65536 = 2^32 -> 0; 65536 * 32768 = 2^31 -> the most negative int32
+    v = run([_inp("x", "i32", (2, 2)), Node("fold", "i32", (2,), (0,), 1, fn="mul")],
+            {0: np.array([[65536, 65536], [65536, 32768]], I32)})
+    assert interp.to_external(v[1], "i32").tolist() == [0, -2**31]
+    # a whole-array fold of a rank-1 array gives a scalar
+    v = run([_inp("x", "i32", (4,)), Node("fold", "i32", (), (0,), 1, fn="min")], {0: np.array([4, -9, 0, 3], I32)})
+    assert int(interp.to_external(v[1], "i32")) == -9
+
+
+def test_scans_with_other_operators_worked():
+    xi = np.array([3, -1, 2, -5, 0], I32)
+    mk = lambda kind, op, dt="i32": Node(kind, dt, (5,), (0,), 1, fn=op)
+    v = {k: interp.to_external(a, "i32") for k, a in
+         run([_inp("x", "i32", (5,)), mk("scanl", "min"), mk("scanl", "max"), mk("scanr", "min"), mk("scanr", "max"),
+              mk("scanl", "mul")], {0: xi}).items()}
+    assert v[1].tolist() == [3, -1, -1, -5, -5]
+    assert v[2].tolist() == [3, 3, 3, 3, 3]
+    assert v[3].tolist() == [-5, -5, -5, -5, 0]
+    assert v[4].tolist() == [3, 2, 2, 0, 0]
+    assert v[5].tolist() == [3, -3, -6, 30, 0]
+    # running maximum that starts negative (an unsigned comparison would keep -4 forever)
+    v = run([_inp("x", "i32", (4,)), Node("scanl", "i32", (4,), (0,), 1, fn="max")], {0: np.array([-4, -2, -3, 1], I32)})
+    assert interp.to_external(v[1], "i32").tolist() == [-4, -2, -2, 1]
+    # unsigned: 2^31 is large, not negative
+    xu = np.array([1, 2**31, 5], U32)
+    v = run([_inp("x", "u32", (3,)), Node("scanl", "u32", (3,), (0,), 1, fn="max"), Node("scanl", "u32", (3,), (0,), 1, fn="min")], {0: xu})
+    assert v[1].tolist() == [1, 2**31, 2**31] and v[2].tolist() == [1, 1, 1]
+    v = run([_inp("x", "i32", (3,)), Node("scanl", "i32", (3,), (0,), 1, fn="max")], {0: xu.view(I32)})
+    assert interp.to_external(v[1], "i32").tolist() == [1, 1, 5]
+    # fp32: product, minimum and maximum, per row, both directions
+    xf = np.array([[0.5, 4, -1], [2, -3, 0.25]], F32)
+    mk = lambda kind, op: Node(kind, "f32", (2, 3), (0,), 1, fn=op)
+    v = run([_inp("x", "f32", (2, 3)), mk("scanl", "mul"), mk("scanl", "min"), mk("scanr", "max"), mk("scanr", "mul")], {0: xf})
+    assert v[1].tolist() == [[0.5, 2.0, -2.0], [2.0, -6.0, -1.5]]
+    assert v[2].tolist() == [[0.5, 0.5, -1.0], [2.0, -3.0, -3.0]]
+    assert v[3].tolist() == [[4.0, 4.0, -1.0], [2.0, 0.25, 0.25]]
+    assert v[4].tolist() == [[-2.0, -4.0, -1.0], [-1.5, -0.75, 0.25]]
+
+
+def test_scatters_with_other_operators_worked():
+    def scatter(dt, op, dest, idx, vals):
+        np_dt = F32 if dt == "f32" else (I32 if dt == "i32" else U32)
+        nodes = [_inp("d", dt, (len(dest),)), _inp("i", "i32", (len(idx),)), _inp("v", dt, (len(vals),)),
+                 Node("permute", dt, (len(dest),), (0, 1, 2), 3, fn=op)]
+        out = run(nodes, {0: np.array(dest, np_dt), 1: np.array(idx, I32), 2: np.array(vals, np_dt)})[3]
+        return interp.to_external(out, dt).tolist()
+    # dest[i] = op(dest[i], x) for every (i, x); untouched bins keep their defaults
+    assert scatter("i32", "min", [10, 10, 10], [0, 0, 2, 2], [-3, 4, 11, 12]) == [-3, 10, 10]
+    assert scatter("i32", "max", [10, 10, 10], [0, 0, 2, 2], [-3, 4, 11, 12]) == [10, 10, 12]
+    assert scatter("i32", "max", [-1, -1], [0, 1], [-2, 3]) == [-1, 3]        # unsigned: -1 would beat 3
+    assert scatter("i32", "min", [-1, -1], [0, 1], [-2, 3]) == [-2, -1]
+    assert scatter("u32", "max", [1, 1], [0, 1, 1], [2**31, 0, 7]) == [2**31, 7]
+    assert scatter("u32", "min", [2**32 - 1, 9], [0, 1, 1], [2**31, 12, 7]) == [2**31, 7]
+    assert scatter("i32", "mul", [2, 3], [0, 0, 1], [5, -1, 4]) == [-10, 12]
+    assert scatter("f32", "min", [1.0, 1.0], [0, 1, 1], [0.5, 2.0, -3.0]) == [0.5, -3.0]
+    assert scatter("f32", "max", [1.0, 1.0], [0, 1, 1], [0.5, 2.0, -3.0]) == [1.0, 2.0]
+    assert scatter("f32", "mul", [1.0, 1.0], [0, 1, 1], [0.5, 2.0, -3.0]) == [0.5, -6.0]
+    with pytest.raises(IndexError):
+        scatter("i32", "min", [0, 0], [0, 2], [1, 1])

@@ -1,16 +1,18 @@
 """The allocation-free prefix sum `acc_scanl_add_i32_static` against the regular path.
 
 Some users of the library call it from places where device memory cannot be allocated
-(a serving loop that must not hit cudaMalloc's device-wide synchronisation, a plug-in that
-only receives raw pointers).  For them the scan's tile states live in a fixed array inside
+(a plug-in that only receives raw pointers, a process whose device memory is handed out
+completely up front).  For them the scan's tile states live in a fixed array inside
 the library.  That array is shared by all calls and keeps its old contents, so the test
-calls the entry point twice in a row, with different data and lengths, and requires each
-result to equal what `acc_run` computes for the same input with a caller-provided
-workspace: bit for bit, as for every integer result in this suite.
+calls the entry point several times in a row, with different data and lengths, and requires
+each result to equal what `acc_run` computes for the same input with a caller-provided
+workspace, and what the CPU oracle computes for it (both paths share a kernel, so their
+agreement alone would prove little): bit for bit, as for every integer result in this suite.
 
 This file sorts last on purpose: a run that stops at the first failure has then already
 exercised every other test.
 """
+import numpy as np
 import pytest
 
 import workloads as W
@@ -33,6 +35,14 @@ def regular_scan(x):
     return out
 
 
+def oracle_scan(x):
+    """The same prefix sum by the oracle's interpreter (wrapping int32 adds, Section 2's scanl)."""
+    from oracle import interp
+    n = x.numel()
+    nodes = [Node("input", "i32", (n,), name="x"), Node("scanl", "i32", (n,), (0,), 1, fn="add", name="out")]
+    return interp.to_external(interp.run(nodes, {0: x.cpu().numpy()}).values[1], "i32")
+
+
 def test_static_scan_matches_regular_scan_twice_in_a_row():
     import torch
     from paper_2407_13585_b200 import binding as B
@@ -44,6 +54,7 @@ def test_static_scan_matches_regular_scan_twice_in_a_row():
         B.scanl_add_i32_static(x, got)
         want = regular_scan(x)
         assert torch.equal(got, want), (seed, n)
+        assert np.array_equal(got.cpu().numpy(), oracle_scan(x)), (seed, n)
     # and the same input again gives the same answer
     B.scanl_add_i32_static(x, got)
     assert torch.equal(got, want)
