@@ -16,7 +16,8 @@
  *     acc_bind / the workspace argument and must stay valid until the work
  *     that uses them has finished on the stream.
  *   - Arrays are dense, row-major, 4-byte elements (fp32, int32, uint32),
- *     rank 0..2, fewer than 2^31 elements, base pointers 16-byte aligned.
+ *     rank 0..2, at most ACC_MAX_ELEMENTS (2^31 - 2^16) elements, base pointers
+ *     16-byte aligned.
  *   - A graph handle is not thread-safe.
  */
 #ifndef ACC_H
@@ -40,7 +41,7 @@ enum acc_kind {
   ACC_INPUT = 0,   /* array supplied by the caller                               */
   ACC_GENERATE,    /* ys[i] = f(i)                                                */
   ACC_MAP,         /* ys[i] = f(xs[i])                       slots {xs, free...}  */
-  ACC_ZIPWITH,     /* ys[i] = f(xs1[i]..xsk[i]), k = 2..5    slots {xs.., free..} */
+  ACC_ZIPWITH,     /* ys[i] = f(xs1[i]..xsk[i]), k = 2..3    slots {xs.., free..} */
   ACC_BACKPERMUTE, /* ys[j] = xs[p(j)], p named by idx_fn    slots {xs}           */
   ACC_GATHER,      /* ys[j] = src[idx[j]] (linear index)     slots {idx, src}     */
   ACC_PERMUTE,     /* out = defaults; out[idx[j]] op= vals[j] slots {defaults, idx, vals} */
@@ -140,6 +141,9 @@ enum acc_status {
 };
 
 #define ACC_MAX_INPUTS 6
+/* Largest array (and largest single extent) acc_add_node accepts: the kernels
+ * index with signed 32-bit arithmetic and keep one tile of head room. */
+#define ACC_MAX_ELEMENTS ((1ll << 31) - (1ll << 16))
 #define ACC_FLAG_FORCE_SLOT(s) (1u << (s)) /* the read of slot s goes through force() */
 /* SCANL / SCANR only.  The paper's scans (Section 2) have no seed and keep the length, which is
  * read as inclusive.  With this flag the scan is seeded and exclusive: element k is the seed
@@ -317,6 +321,15 @@ int acc_run_e2e(acc_graph* g, void* workspace, size_t workspace_bytes, void* cud
  * directions with each other and with the kernels. */
 int acc_run_e2e_async(acc_graph* g, void* workspace, size_t workspace_bytes, void* cuda_stream, int executor,
                       size_t* h2d_bytes, size_t* d2h_bytes);
+/* Bound of the one device-side wait that polls plain memory: a tile of a
+ * single-pass scan (Section 2: "prefix sum", computed with decoupled look-back)
+ * polls the state of the tiles before it until they have published a total.
+ * A tile that has polled max_polls times without success gives up, the run
+ * goes on and ends with ACC_ERR_DEVICE_TIMEOUT (the scan's output is then not
+ * valid); 0 gives up at the first unsuccessful poll.  Default 2^22 (seconds).
+ * Applies to later runs of this graph; the waits on copy barriers in the
+ * tile-staging kernels have a fixed bound and are not affected. */
+int acc_set_spin_limit(acc_graph* g, uint32_t max_polls);
 /* Kernels launched by the last acc_run / acc_run_e2e on this graph. */
 int32_t acc_launch_count(const acc_graph* g);
 /* Clusters of the last run, as "first_node:count" items separated by blanks,

@@ -103,6 +103,7 @@ def load_library(path=LIB_PATH):
         "acc_run_timed": (C.c_int, [p, p, sz, p, C.c_int, C.POINTER(C.c_float), i32, pi32]),
         "acc_check_gather_indices": (C.c_int, [p, p, sz, p]),
         "acc_launch_count": (i32, [p]),
+        "acc_set_spin_limit": (C.c_int, [p, C.c_uint32]),
         "acc_last_schedule": (C.c_int, [p, C.c_char_p, sz]),
         "acc_scanl_add_i32_static": (C.c_int, [p, p, i64, p]),
         "acc_last_error": (C.c_char_p, []),
@@ -342,6 +343,9 @@ class Graph:
         """Raises AccError(ACC_ERR_INDEX_RANGE) if an input index array of a gather points outside its source."""
         ws = self.ensure_workspace(FUSED)
         _check(lib().acc_check_gather_indices(self._h, C.c_void_p(ws.data_ptr()), ws.numel(), self._stream()))
+
+    def set_spin_limit(self, max_polls):
+        _check(lib().acc_set_spin_limit(self._h, max_polls))
 
     def launch_count(self):
         return lib().acc_launch_count(self._h)

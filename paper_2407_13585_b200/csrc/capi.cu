@@ -26,6 +26,7 @@ std::map<const acc_graph*, std::unique_ptr<Cache[]>>& caches() {
 Graph& run_target(acc_graph* g, int executor) {
   if (executor != ACC_EXEC_FUSED || !g->unfolded) return *g;
   Graph& u = *g->unfolded;
+  u.spin_limit = g->spin_limit;
   for (size_t i = 0; i < g->nodes.size(); ++i) {
     Node& to = u.nodes[g->home_in_unfolded[i]];
     const Node& from = g->nodes[i];
@@ -404,6 +405,12 @@ int acc_run_e2e_async(acc_graph* g, void* workspace, size_t workspace_bytes, voi
 }
 
 int32_t acc_launch_count(const acc_graph* g) { return g ? g->launches : ACC_ERR_ARG; }
+
+int acc_set_spin_limit(acc_graph* g, uint32_t max_polls) {
+  if (!g) return set_error(ACC_ERR_ARG, "null graph");
+  g->spin_limit = max_polls;
+  return ACC_OK;
+}
 
 int acc_last_schedule(const acc_graph* g, char* buf, size_t cap) {
   if (!g || !buf || !cap) return ACC_ERR_ARG;

@@ -1,7 +1,6 @@
-// Execution of a program: clusters in ascending cluster number, one kernel launch per
-// cluster on the caller's stream (Section 4.1: "clusters are executed in the ascending
-// order of their cluster numbers").  The unfused executor is the same machinery with
-// every combinator its own cluster.
+// Execution of a program: clusters run by ascending cluster number (Section 4.1), one kernel
+// launch each (or one per pass) on the caller's stream.  The unfused executor is the same
+// machinery with every combinator its own cluster.
 #include <algorithm>
 #include <cstring>
 #include <map>
@@ -233,6 +232,7 @@ int run_schedule(Graph& g, Schedule& sch, void* workspace, size_t ws_bytes, cuda
     st.launch.scratch = reinterpret_cast<uint32_t*>(ws + st.scratch_off);
     st.launch.status = reinterpret_cast<uint32_t*>(ws);
     st.launch.stream = stream;
+    st.launch.spin_limit = g.spin_limit;
     const int rc = st.kernel->launch(st.launch);
     if (rc != ACC_OK) return rc;
     if (!mark(marks, stream)) return set_error(ACC_ERR_CUDA, "recording an event failed: %s", cudaGetErrorString(cudaGetLastError()));

@@ -48,6 +48,20 @@ static int fn_arity(int fn, int* free_slots) {
   }
 }
 
+// What an element function computes on: 1 = fp32 arithmetic, 2 = integer (bit-pattern) arithmetic,
+// 0 = defined for both (identity, +, *).
+static int fn_domain(int fn) {
+  switch (fn) {
+    case ACC_FN_AFFINE: case ACC_FN_DIV_FREE: case ACC_FN_ADD_FREE: case ACC_FN_MUL_ADD_CONST: case ACC_FN_ADD_SCALE:
+    case ACC_FN_ADD3:
+      return 1;
+    case ACC_FN_HASH_MUL_XORSHIFT: case ACC_FN_AND_MASK: case ACC_FN_MUL_MOD: case ACC_FN_MUL_CONST: case ACC_FN_ADD_CONST:
+      return 2;
+    default:
+      return 0;
+  }
+}
+
 int add_node(Graph& g, const acc_node_desc& d) {
   const int id = (int)g.nodes.size();
   if (d.kind < ACC_INPUT || d.kind > ACC_SCANR) return set_error(ACC_ERR_ARG, "node %d: unknown kind %d", id, d.kind);
@@ -57,7 +71,10 @@ int add_node(Graph& g, const acc_node_desc& d) {
   for (int i = 0; i < d.rank; ++i) {
     if (d.shape[i] < 0) return set_error(ACC_ERR_SHAPE, "node %d: negative extent", id);
     count *= d.shape[i];
-    if (count >= (int64_t(1) << 31)) return set_error(ACC_ERR_SHAPE, "node %d: 2^31 elements or more", id);
+    // kernels index with signed 32-bit arithmetic and step past the end of a row by up to one tile
+    // (2^14 elements) before they compare: leave that room
+    if (count > ACC_MAX_ELEMENTS || d.shape[i] > ACC_MAX_ELEMENTS)
+      return set_error(ACC_ERR_SHAPE, "node %d: more than 2^31 - 2^16 elements", id);
   }
   if (d.n_inputs < 0 || d.n_inputs > ACC_MAX_INPUTS || d.n_array_inputs < 0 || d.n_array_inputs > d.n_inputs)
     return set_error(ACC_ERR_ARG, "node %d: bad slot counts %d/%d", id, d.n_array_inputs, d.n_inputs);
@@ -90,9 +107,19 @@ int add_node(Graph& g, const acc_node_desc& d) {
       if (ar < 0) return set_error(ACC_ERR_ARG, "node %d: %d is not an element function", id, d.fn_id);
       if (d.n_array_inputs != ar || n_free != want_free)
         return set_error(ACC_ERR_ARG, "node %d: function %d takes %d array and %d free slots", id, d.fn_id, ar, want_free);
-      if ((d.kind == ACC_MAP) != (ar == 1)) return set_error(ACC_ERR_ARG, "node %d: map takes one array, zipWith two to five", id);
+      if ((d.kind == ACC_MAP) != (ar == 1)) return set_error(ACC_ERR_ARG, "node %d: map takes one array, zipWith two or three", id);
       for (int s = 0; s < ar; ++s)
         if (!same_shape(in(s), d)) return set_error(ACC_ERR_SHAPE, "node %d: slot %d differs in shape", id, s);
+      // element functions are typed: fp32 arithmetic on fp32 arrays, bit arithmetic on integer ones;
+      // the generic ones (identity, +, *) keep the class of their operands
+      const int domain = fn_domain(d.fn_id);               // 1 fp32, 2 integer, 0 either
+      const bool want_int = domain == 2 || (domain == 0 && is_int(d.dtype));
+      if (domain == 1 && d.dtype != ACC_F32) return set_error(ACC_ERR_DTYPE, "node %d: function %d yields fp32", id, d.fn_id);
+      if (domain == 2 && !is_int(d.dtype)) return set_error(ACC_ERR_DTYPE, "node %d: function %d yields an integer", id, d.fn_id);
+      for (int s = 0; s < d.n_inputs; ++s)
+        if (is_int(in(s).dtype) != want_int)
+          return set_error(ACC_ERR_DTYPE, "node %d: slot %d is %s, function %d works on %s", id, s, is_int(in(s).dtype) ? "integer" : "fp32",
+                           d.fn_id, want_int ? "integers" : "fp32");
       if (d.fn_id == ACC_FN_MUL_MOD && d.iparam[1] <= 0) return set_error(ACC_ERR_ARG, "node %d: modulus must be positive", id);
       if (d.fn_id == ACC_FN_HASH_MUL_XORSHIFT && (d.iparam[1] < 0 || d.iparam[1] > 31))
         return set_error(ACC_ERR_ARG, "node %d: shift outside 0..31", id);

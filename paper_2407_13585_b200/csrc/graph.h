@@ -47,6 +47,7 @@ struct Graph {
   std::string schedule;
   uint32_t host_status = 0;
   uint32_t run_serial = 0;         // bumped by every change that invalidates a schedule
+  uint32_t spin_limit = 1u << 22;  // polls a scan tile spends on a predecessor before it gives up (acc_set_spin_limit)
 };
 
 inline bool is_input(const Node& n) { return n.d.kind == ACC_INPUT; }

@@ -530,3 +530,30 @@ def test_maps_of_row_folds(n, m):
 @pytest.mark.parametrize("rows", [4, 64, 100, 130, 256, 1600])
 def test_diagonal_of_a_product(rows):
     assert check_program(W.diagonal_of_product(rows)) == 4
+
+
+def test_lookback_wait_that_runs_out_is_reported():
+    """The one device-side wait that polls plain memory (a scan tile looking back at its predecessors) is given
+    no patience at all: tiles that find a predecessor unfinished give up at once, the kernel ends normally, and
+    the run reports ACC_ERR_DEVICE_TIMEOUT; with the default bound the same graph then gives the oracle's result."""
+    import torch
+    from oracle import interp
+    from paper_2407_13585_b200 import binding as B
+    from workloads import Node
+    n = 1 << 22
+    nodes = [Node("input", "i32", (n,), name="x"), Node("scanl", "i32", (n,), (0,), 1, fn="add", name="out")]
+    x = W.uniform_int(5, 0, n, 1 << 31, device="cuda")
+    out = torch.zeros(n, dtype=torch.int32, device="cuda")
+    g = B.Graph(nodes, [1])
+    g.bind(0, x)
+    g.bind(1, out)
+    g.set_spin_limit(0)
+    with pytest.raises(B.AccError) as e:
+        g.run(B.UNFUSED)
+    assert e.value.status == "ACC_ERR_DEVICE_TIMEOUT"
+    g.set_spin_limit(1 << 22)
+    g.run(B.UNFUSED)
+    want = np.cumsum(x.cpu().numpy().view(np.uint32), dtype=np.uint32).view(np.int32)       # wrapping adds, as Section 2's scanl(+)
+    ref = interp.run(nodes, {0: x.cpu().numpy()}).values[1]
+    assert np.array_equal(interp.to_external(ref, "i32"), want)
+    assert np.array_equal(out.cpu().numpy(), want)

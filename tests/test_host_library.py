@@ -408,3 +408,50 @@ def test_refine_to_kernels_splits_only_clusters_nobody_built():
     g = B.Graph(prog.nodes, prog.outputs)
     with pytest.raises(B.AccError):
         g.refine_to_kernels()
+
+
+def test_element_functions_are_typed():
+    # fp32 arithmetic on integer arrays, bit arithmetic on fp32 arrays and mixed operands are refused when
+    # the node is added (they would otherwise surface as a missing kernel at run time, or as reinterpreted bits)
+    g = B.Graph()
+    xf = g.add_node(_inp("xf", "f32", (8,)))
+    xi = g.add_node(_inp("xi", "i32", (8,)))
+    xu = g.add_node(_inp("xu", "u32", (8,)))
+    bad = [
+        Node("map", "i32", (8,), (xi,), 1, fn="affine", fparam=(2.0, 1.0)),
+        Node("map", "f32", (8,), (xi,), 1, fn="affine", fparam=(2.0, 1.0)),
+        Node("zipwith", "u32", (8,), (xu, xu), 2, fn="mul_add_const"),
+        Node("map", "f32", (8,), (xf,), 1, fn="and_mask", iparam=(255,)),
+        Node("map", "i32", (8,), (xf,), 1, fn="hash_mul_xorshift", iparam=(3, 5)),
+        Node("map", "f32", (8,), (xf,), 1, fn="mul_mod", iparam=(3, 7)),
+        Node("zipwith", "f32", (8,), (xf, xi), 2, fn="add"),
+        Node("zipwith", "i32", (8,), (xi, xf), 2, fn="mul"),
+        Node("map", "i32", (8,), (xf,), 1, fn="identity"),
+    ]
+    for nd in bad:
+        with pytest.raises(B.AccError) as e:
+            g.add_node(nd)
+        assert e.value.status == "ACC_ERR_DTYPE", nd
+    # signed and unsigned integers are the same bit patterns and may meet
+    assert g.add_node(Node("zipwith", "i32", (8,), (xi, xu), 2, fn="add")) == 3
+    assert g.add_node(Node("map", "u32", (8,), (xi,), 1, fn="mul_mod", iparam=(3, 7))) == 4
+    assert g.add_node(Node("map", "f32", (8,), (xf,), 1, fn="identity")) == 5
+
+
+def test_arrays_near_the_index_range_are_refused():
+    # kernels index with signed 32-bit arithmetic and overshoot a row by up to a tile before comparing
+    limit = (1 << 31) - (1 << 16)
+    g = B.Graph()
+    assert g.add_node(_inp("big", "f32", (limit,))) == 0
+    assert g.add_node(_inp("big2", "f32", (2, limit // 2))) == 1
+    for shape in ((limit + 1,), ((1 << 31) - 1,), (2, limit // 2 + 1), (1 << 16, 1 << 15)):
+        with pytest.raises(B.AccError) as e:
+            g.add_node(_inp("too_big", "f32", shape))
+        assert e.value.status == "ACC_ERR_SHAPE", shape
+
+
+def test_spin_limit_is_a_property_of_the_graph():
+    g = B.Graph(W.config3(64).nodes, W.config3(64).outputs)
+    g.set_spin_limit(0)
+    g.set_spin_limit(1 << 22)
+    assert B.lib().acc_set_spin_limit(None, 5) == B.lib().acc_launch_count(None)      # both refuse a null graph with ACC_ERR_ARG
