@@ -125,6 +125,21 @@ def lib():
     return _lib
 
 
+_kernel_libraries = {}
+
+
+def load_kernel_library(path):
+    """Loads a shared object of further kernel instantiations (built by `build.build_kernel_library`); its
+    kernels register themselves with libacc.so while it loads.  Returns how many signatures were new."""
+    path = os.path.abspath(path)
+    before = registry_size()
+    if path not in _kernel_libraries:
+        if not os.path.exists(path):
+            raise ImportError("%s is missing: build it with `python -m paper_2407_13585_b200.build --tests`" % path)
+        _kernel_libraries[path] = C.CDLL(path, mode=C.RTLD_GLOBAL)
+    return registry_size() - before
+
+
 def _check(code):
     if code < 0:
         raise AccError(int(code), lib().acc_last_error().decode())

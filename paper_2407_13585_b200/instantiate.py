@@ -130,7 +130,7 @@ def main(argv):
     out = sys.stdout
     out.write("// Generated by `python -m paper_2407_13585_b200.instantiate %s`.\n" % " ".join(argv))
     out.write("// Every cluster of every legal clustering of the programs named above, and every node alone.\n")
-    out.write('#include "../device/launch.cuh"\n\nnamespace acc {\n\n')
+    out.write('#include "device/launch.cuh"\n\nnamespace acc {\n\n')
     for spec in argv:
         mod, fn, *rest = spec.split(":")                  # module:function[:int,int,...]
         prog = getattr(importlib.import_module(mod), fn)(*[int(v) for v in rest[0].split(",")] if rest else [])

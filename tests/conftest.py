@@ -12,6 +12,15 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu on a B200)")
 
 
+def pytest_sessionstart(session):
+    """The kernels of the seeded random test programs are not part of the product library: they live in a
+    shared object of their own, built from tests/programs/ and loaded into the registry here."""
+    from paper_2407_13585_b200 import binding, build
+    if not os.path.exists(build.TEST_LIB):
+        build.build_test_kernels()
+    binding.load_kernel_library(build.TEST_LIB)
+
+
 def pytest_collection_modifyitems(config, items):
     try:
         import torch

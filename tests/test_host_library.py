@@ -372,11 +372,13 @@ def test_unbound_buffers_are_reported_without_a_device():
 
 
 def test_generated_sources_match_their_programs():
-    # every csrc/programs/prog_random*.cu and prog_scan_consumers*.cu is what the generator prints today for the command in its first line
+    # every tests/programs/prog_random*.cu and the library's prog_scan_consumers*.cu are what the generator prints today for the
+    # command in their first line
     import glob, io, os, re
     from paper_2407_13585_b200 import instantiate
-    here = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "paper_2407_13585_b200", "csrc", "programs")
-    files = sorted(glob.glob(os.path.join(here, "prog_random*.cu")) + glob.glob(os.path.join(here, "prog_scan_consumers*.cu")) +
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    here = os.path.join(root, "paper_2407_13585_b200", "csrc", "programs")
+    files = sorted(glob.glob(os.path.join(root, "tests", "programs", "prog_random*.cu")) + glob.glob(os.path.join(here, "prog_scan_consumers*.cu")) +
                    glob.glob(os.path.join(here, "prog_histogram_2d.cu")))
     assert len(files) >= 18
     for f in files:
