@@ -14,6 +14,21 @@
 
 namespace acc {
 
+// Opt-in to `smem` bytes of dynamic shared memory for a kernel, asked of the driver once per device
+// and size: `granted` (one per kernel, 64 zeroed words) remembers the largest size already granted.
+template <class K>
+inline bool opt_in_shared_memory(K kern, size_t smem, int* granted) {
+  int device = 0;
+  if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) {
+    cudaGetLastError();
+    return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) == cudaSuccess;
+  }
+  if (granted[device] >= (int)smem + 1) return true;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return false;
+  granted[device] = (int)smem + 1;
+  return true;
+}
+
 template <class CL>
 struct Launcher {
   static constexpr int N = CL::c.n;
@@ -151,7 +166,8 @@ struct Launcher {
       auto kern = dev::k_stencil<CL>;
       // two stages of every external's box, one box per member kept on chip
       const size_t smem = (size_t)(dev::kStStages * dev::staged_externals<CL>() + dev::staged_members<CL>()) * dev::st_box_stride(depth) * 4;
-      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      static int granted[64];
+      if (!opt_in_shared_memory(kern, smem, granted))
         return set_error(ACC_ERR_CUDA, "shared-memory opt-in failed: %s", cudaGetErrorString(cudaGetLastError()));
       const int64_t tiles = (int64_t)((C + dev::kStCols - 1) / dev::kStCols) * ((R + dev::kStRows - 1) / dev::kStRows);
       const int per_sm = std::max(1, std::min(3, (int)((size_t)220 * 1024 / (smem + 1024))));
@@ -266,7 +282,8 @@ struct Launcher {
         if (rc != 1) return rc;                          // 1 = no tensor copies here: the threads stage the tiles
         auto kern = vec ? dev::k_tile_pair<CL, true> : dev::k_tile_pair<CL, false>;
         const size_t smem = (size_t)dev::staged_externals<CL>() * 2 * dev::kTileWords * 4;
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        static int granted[2][64];
+        if (!opt_in_shared_memory(kern, smem, granted[vec ? 1 : 0]))
           return set_error(ACC_ERR_CUDA, "shared-memory opt-in failed: %s", cudaGetErrorString(cudaGetLastError()));
         const int blocks = (R + dev::kTile - 1) / dev::kTile;
         kern<<<blocks * (blocks + 1) / 2, dev::kBlock, smem, L.stream>>>(a);
@@ -331,7 +348,8 @@ int Launcher<CL>::launch_hist(const ClusterLaunch& L, dev::Args<N>& a, int R, in
     const int64_t bins = (int64_t)L.nodes[P].R * L.nodes[P].C;
     auto kern = vec ? dev::k_hist<CL, true> : dev::k_hist<CL, false>;
     const size_t smem = (size_t)plan.per_cta * 4;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    static int granted[2][64];
+    if (!opt_in_shared_memory(kern, smem, granted[vec ? 1 : 0]))
       return set_error(ACC_ERR_CUDA, "shared-memory opt-in failed: %s", cudaGetErrorString(cudaGetLastError()));
     const int64_t chunks = (int64_t)R * C / (vec ? 4 : 1);
     const int64_t per_team = (int64_t)dev::kHistBlock * dev::kHistUnroll;

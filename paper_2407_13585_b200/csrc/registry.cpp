@@ -48,6 +48,10 @@ bool cooperative_launch_ok() {
 // ---- tensor maps for cp.async.bulk.tensor copies -------------------------------------------
 #include <cuda.h>
 
+#include <cstring>
+#include <mutex>
+#include <tuple>
+
 namespace acc {
 
 using EncodeTiled = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -70,13 +74,33 @@ bool make_tensor_map_2d(void* out, const void* base, int rows, int cols, int box
     encode = reinterpret_cast<EncodeTiled>(fn);
   }
   if (rows < 1 || cols < 1 || cols % 4 || (reinterpret_cast<uintptr_t>(base) & 15)) return false;
+  // the descriptor depends on nothing but these five values: programs that run again and again
+  // over the same buffers get it from a small table instead of the driver
+  using Key = std::tuple<const void*, int, int, int, int>;
+  static std::map<Key, CUtensorMap> known;
+  static std::mutex guard;
+  const Key key{base, rows, cols, box_rows, box_cols};
+  {
+    std::lock_guard<std::mutex> lock(guard);
+    auto it = known.find(key);
+    if (it != known.end()) {
+      memcpy(out, &it->second, sizeof(CUtensorMap));
+      return true;
+    }
+  }
+  CUtensorMap made;
   const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   const cuuint64_t strides[1] = {(cuuint64_t)cols * 4};                 // bytes between rows: a multiple of 16
   const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
   const cuuint32_t step[2] = {1, 1};
-  return encode(static_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(base), dims, strides, box,
-                step, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  if (encode(&made, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(base), dims, strides, box, step, CU_TENSOR_MAP_INTERLEAVE_NONE,
+             CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return false;
+  memcpy(out, &made, sizeof(CUtensorMap));
+  std::lock_guard<std::mutex> lock(guard);
+  if (known.size() >= 4096) known.clear();
+  known.emplace(key, made);
+  return true;
 }
 
 }  // namespace acc
