@@ -23,9 +23,12 @@ constexpr int kMaxCluster = 40;   // local nodes per cluster
 constexpr int kMaxProgram = 40;   // nodes per build-time program
 
 // Constants of a node that select code instead of being run-time arguments: the row and
-// column offsets of a clamped shift when both lie in -1..1 (kRunTime: not fixed), and
-// p0 = 1 for a seeded exclusive scan.
+// column offsets of a clamped shift when both lie in -1..1 (kRunTime: not fixed), p0 = 1 for a
+// seeded exclusive scan, and p0 = kPow2 for a modulus that is a power of two.  Except for the
+// scan's, a kernel built with kRunTime in their place serves every value.
 constexpr int kRunTime = 9;
+// p0 of a map with ACC_FN_MUL_MOD: the modulus is a power of two (v mod d is one AND in such a kernel).
+constexpr int kPow2 = 1;
 
 struct PNode {                    // node of a build-time program
   int kind = 0, dtype = 0, rank = 0, fn = 0, idxfn = 0, nin = 0, narr = 0;

@@ -27,7 +27,7 @@ struct NodeArg {
   // host (d = iparam[1] for ACC_FN_MUL_MOD, iparam[0] otherwise, 1 <= d < 2^32): for every 32-bit
   // v, with t = umulhi(v, div_mul):  v / d == (t + ((v - t) >> div_sh1)) >> div_sh2
   uint32_t div_mul, div_sh1, div_sh2;
-  uint32_t div_mask;   // d - 1 when d is a power of two (> 1), else 0: then v mod d is one AND
+  uint32_t div_mask;   // d - 1 when d is a power of two, else 0 (kernels built for such divisors use it)
 };
 
 // v / d and v mod d with the host's multiplier for d (see NodeArg).
@@ -35,9 +35,13 @@ __device__ __forceinline__ uint32_t div_by(uint32_t v, const NodeArg& p) {
   const uint32_t t = __umulhi(v, p.div_mul);
   return (t + ((v - t) >> p.div_sh1)) >> p.div_sh2;
 }
+// POW2: the kernel was built for divisors that are powers of two (cluster.h, kPow2): one AND.  Otherwise
+// the multiplier sequence, which is right for every divisor (for d = 2^l its multiplier is 1 and the
+// shifts do the work), with no test of the divisor per call.
+template <bool POW2 = false>
 __device__ __forceinline__ uint32_t mod_by(uint32_t v, uint32_t d, const NodeArg& p) {
-  if (p.div_mask != 0) return v & p.div_mask;             // the same for every thread of the launch
-  return v - div_by(v, p) * d;
+  if constexpr (POW2) return v & p.div_mask;
+  else return v - div_by(v, p) * d;
 }
 
 template <int N>
@@ -176,7 +180,7 @@ template <int F, int P0 = kRunTime, int P1 = kRunTime> __device__ __forceinline_
 __device__ __forceinline__ float f_(uint32_t b) { return __uint_as_float(b); }
 __device__ __forceinline__ uint32_t u_(float f) { return __float_as_uint(f); }
 
-template <int FN>
+template <int FN, int P0 = kRunTime>
 __device__ __forceinline__ uint32_t apply1(const NodeArg& p, uint32_t a, uint32_t free0) {
   if constexpr (FN == ACC_FN_IDENTITY) return a;
   else if constexpr (FN == ACC_FN_AFFINE) return u_(__fadd_rn(__fmul_rn(p.fp0, f_(a)), p.fp1));
@@ -186,7 +190,7 @@ __device__ __forceinline__ uint32_t apply1(const NodeArg& p, uint32_t a, uint32_
   else if constexpr (FN == ACC_FN_AND_MASK) return a & (uint32_t)p.ip0;
   else if constexpr (FN == ACC_FN_MUL_MOD) {
     const uint32_t t = a * (uint32_t)p.ip0;
-    return mod_by(t, (uint32_t)p.ip1, p);
+    return mod_by<P0 == kPow2>(t, (uint32_t)p.ip1, p);
   }
   else if constexpr (FN == ACC_FN_MUL_CONST) return a * (uint32_t)p.ip0;
   else if constexpr (FN == ACC_FN_ADD_CONST) return a + (uint32_t)p.ip0;
@@ -298,7 +302,7 @@ __device__ __forceinline__ uint32_t eval_member1(const A& a, const IX& ix) {    
   if constexpr (nd.kind == ACC_GENERATE) {
     return generate1<nd.fn, nd.dtype>(a.n[I], lane(ix, 0), free_of<CL, I>(a));
   } else if constexpr (nd.kind == ACC_MAP) {
-    return apply1<nd.fn>(a.n[I], eval<CL, nd.in[0]>(a, ix), free_of<CL, I>(a));
+    return apply1<nd.fn, nd.p0>(a.n[I], eval<CL, nd.in[0]>(a, ix), free_of<CL, I>(a));
   } else if constexpr (nd.kind == ACC_ZIPWITH && nd.narr == 2) {
     return apply2<nd.fn, nd.dtype>(a.n[I], eval<CL, nd.in[0]>(a, ix), eval<CL, nd.in[1]>(a, ix));
   } else if constexpr (nd.kind == ACC_ZIPWITH && nd.narr == 3) {
@@ -414,7 +418,7 @@ __device__ __forceinline__ val_of<IX> eval_here(const A& a, const IX& ix) {
     const V4 x = eval<CL, nd.in[0]>(a, ix);
     V4 out;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) out.v[j] = apply1<nd.fn>(a.n[I], x.v[j], f0);
+    for (int j = 0; j < 4; ++j) out.v[j] = apply1<nd.fn, nd.p0>(a.n[I], x.v[j], f0);
     return out;
   } else if constexpr (nd.kind == ACC_ZIPWITH && nd.narr == 2) {
     const V4 x = eval<CL, nd.in[0]>(a, ix), y = eval<CL, nd.in[1]>(a, ix);

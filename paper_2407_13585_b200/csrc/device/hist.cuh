@@ -122,6 +122,7 @@ k_hist(const __grid_constant__ Args<CL::c.n> a, const HistPlan plan, int* overfl
   for (int i = threadIdx.x; i < per_cta; i += kHistBlock) bins_smem[i] = 0;
 
   uint32_t acc[N];
+  float comp[N] = {};                                          // see fold_step
   static_for<0, N>([&](auto ic) {
     constexpr int i = decltype(ic)::value;
     constexpr CNode nd = CL::c.nodes[i];
@@ -245,11 +246,14 @@ k_hist(const __grid_constant__ Args<CL::c.n> a, const HistPlan plan, int* overfl
             if constexpr (nd.in[0] == CL::c.nodes[P].in[2]) v = val[u];
             else if constexpr (nd.in[0] == CL::c.nodes[P].in[1]) v = key[u];
             else v = eval<CL, nd.in[0]>(a, ix);
+            // a thread adds thousands of chunks to its running value: that step is compensated; the four
+            // elements of a chunk are of one magnitude and are combined as a small tree first
             if constexpr (VEC) {
-#pragma unroll
-              for (int j = 0; j < 4; ++j) acc[i] = combine<nd.fn, nd.dtype>(acc[i], v.v[j]);
+              const uint32_t four = combine<nd.fn, nd.dtype>(combine<nd.fn, nd.dtype>(v.v[0], v.v[1]),
+                                                             combine<nd.fn, nd.dtype>(v.v[2], v.v[3]));
+              fold_step<nd.fn, nd.dtype>(acc[i], comp[i], four);
             } else {
-              acc[i] = combine<nd.fn, nd.dtype>(acc[i], v);
+              fold_step<nd.fn, nd.dtype>(acc[i], comp[i], v);
             }
           }
         });

@@ -43,6 +43,8 @@ static bool extract_runtime(const Graph& g, const std::vector<int>& members, con
       n.p1 = (int)d.iparam[1];
     }
     if ((d.kind == ACC_SCANL || d.kind == ACC_SCANR) && (d.flags & ACC_FLAG_SCAN_EXCLUSIVE)) n.p0 = 1;   // other code, not another argument
+    if (d.kind == ACC_MAP && d.fn_id == ACC_FN_MUL_MOD && d.iparam[1] > 0 && (d.iparam[1] & (d.iparam[1] - 1)) == 0)
+      n.p0 = kPow2;                                    // a kernel built for power-of-two moduli is looked up first
     for (int s = 0; s < d.n_inputs; ++s) n.in[s] = local[d.inputs[s]];
     local[m] = c.n;
     c.source[c.n] = m;
@@ -68,7 +70,7 @@ static dev::NodeArg node_arg(const Node& n, const void* ptr) {
     a.div_mul = (uint32_t)((((1ull << l) - d) << 32) / d + 1);
     a.div_sh1 = l < 1 ? l : 1;
     a.div_sh2 = l - a.div_sh1;
-    a.div_mask = (d > 1 && (d & (d - 1)) == 0) ? d - 1 : 0;
+    a.div_mask = (d & (d - 1)) == 0 ? d - 1 : 0;
   }
   a.R = n.d.rank == 2 ? (int32_t)n.d.shape[0] : 1;
   a.C = n.d.rank == 2 ? (int32_t)n.d.shape[1] : (n.d.rank == 1 ? (int32_t)n.d.shape[0] : 1);
@@ -81,7 +83,8 @@ static const KernelEntry* lookup(CCluster& cc, std::string& sig) {
   const KernelEntry* k = find_kernel(sig);
   if (!k) {
     for (int li = 0; li < cc.n; ++li)
-      if (cc.nodes[li].kind == ACC_BACKPERMUTE) cc.nodes[li].p0 = cc.nodes[li].p1 = kRunTime;
+      if (cc.nodes[li].kind == ACC_BACKPERMUTE || (cc.nodes[li].kind == ACC_MAP && cc.nodes[li].fn == ACC_FN_MUL_MOD))
+        cc.nodes[li].p0 = cc.nodes[li].p1 = kRunTime;
     sig = signature(cc);
     k = find_kernel(sig);
   }

@@ -114,8 +114,16 @@ inline constexpr CProgram kTransposeReduce = transpose_reduce();
 inline constexpr CProgram kGatherScan = gather_scan();
 inline constexpr CProgram kJacobi = jacobi_iteration();
 inline constexpr CProgram kJacobiChain = jacobi_chain(4);
+// The same programs for a hash whose modulus is a power of two (as many bins as a power of two).
+constexpr CProgram with_pow2_hash(CProgram p) {
+  p.nodes[2] = fixed(p.nodes[2], kPow2, kRunTime);
+  return p;
+}
+
 inline constexpr CProgram kHistogram = histogram_diamond();
 inline constexpr CProgram kHistogramScatterOnly = histogram_scatter_only();
+inline constexpr CProgram kHistogramPow2 = with_pow2_hash(histogram_diamond());
+inline constexpr CProgram kHistogramScatterOnlyPow2 = with_pow2_hash(histogram_scatter_only());
 inline constexpr CProgram kGeneratedTotal = generated_total();
 
 }  // namespace programs

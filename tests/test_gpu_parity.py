@@ -198,6 +198,17 @@ def test_equal_addends_stay_within_tolerance():
         g = B.Graph(prog.nodes, prog.outputs)
         pi = g.plan("enumerate", "bytes")
         check_program(prog, [pi], passes=True, inputs_t=constant(prog))
+    # a whole-array fold beside a scatter with on-chip bins (the kernel config 5's diamond runs in), fed from memory:
+    # hist = permute(+) zeros (hash keys) vals and total = fold(+) vals share a kernel through their common input
+    from workloads import Node, Program
+    n, bins = 1 << 24, 1 << 10
+    nodes = [Node("input", "u32", (n,), name="keys"), Node("input", "f32", (bins,), name="zeros"), Node("input", "f32", (n,), name="vals"),
+             Node("map", "u32", (n,), (0,), 1, fn="mul_mod", iparam=(40503, bins), name="k"),
+             Node("permute", "f32", (bins,), (1, 3, 2), 3, fn="add", name="hist"),
+             Node("fold", "f32", (), (2,), 1, fn="add", name="total")]
+    prog = Program("weighted_histogram_with_total", nodes, [4, 5])
+    inputs = {0: W.zipf_keys(0, 0, n), 1: torch.zeros(bins), 2: torch.full((n,), 0.1)}
+    check_program(prog, [[-1, -1, -1, 0, 1, 1]], inputs_t=inputs)
 
 
 # random DAGs around a scan in the middle.  Clusterings in which something other than an element-wise chain reads
