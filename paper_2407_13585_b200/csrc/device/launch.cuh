@@ -113,6 +113,31 @@ struct Launcher {
     }
   }
 
+  // blocks of k_segfold: one per run of kSegTilesPerBlock tiles of the folds' source (its records are laid out for them)
+  static int seg_grid(const ClusterLaunch& L) {
+    if constexpr (kHasSegFold) {
+      const int src = CL::c.nodes[dev::first_segfold<CL>()].in[0];
+      const int64_t n_src = (int64_t)L.nodes[src].R * L.nodes[src].C;
+      const int64_t tiles = std::max<int64_t>(1, (n_src + dev::kSegTile - 1) / dev::kSegTile);
+      return (int)((tiles + dev::kSegTilesPerBlock - 1) / dev::kSegTilesPerBlock);
+    } else {
+      return 0;
+    }
+  }
+
+  // 128-bit reads of a segmented fold's operands: every array read as an array has 16-byte rows and base
+  static bool seg_vec_ok(const ClusterLaunch& L) {
+    for (int i = 0; i < N; ++i) {
+      if (CL::c.nodes[i].member) continue;
+      bool as_array = false;
+      for (int j = 0; j < N; ++j)
+        for (int s = 0; s < CL::c.nodes[j].narr; ++s)
+          if (CL::c.nodes[j].member && CL::c.nodes[j].in[s] == i) as_array = true;
+      if (as_array && (L.nodes[i].C % 4 || (reinterpret_cast<uintptr_t>(L.nodes[i].ptr) & 15))) return false;
+    }
+    return true;
+  }
+
   static int64_t scratch_bytes(const ClusterLaunch& L) {
     int R, C;
     if (!domain(L, R, C)) return ACC_ERR_NO_KERNEL;
@@ -121,7 +146,8 @@ struct Launcher {
       return (dev::tile_partials_off(blocks) + (int64_t)kRowFolds * blocks * R) * 4;
     }
     if (kHasScan) return 16 + (int64_t)R * ((C + kScanTile - 1) / kScanTile) * 8;
-    if (kHasRowFold || kHasSegFold) return 0;
+    if (kHasSegFold) return dev::seg_scratch_words(dev::count_if<CL>(dev::is_segfold_root), seg_grid(L)) * 4;
+    if (kHasRowFold) return 0;
     int64_t words = dev::stream_acc64_off(kScalarFolds, sm_count() * 8);
     for (int i = 0; i < N; ++i)
       if (dev::is_f32_add_permute(CL::c.nodes[i])) words += 2 * (int64_t)L.nodes[i].R * L.nodes[i].C;
@@ -295,8 +321,17 @@ struct Launcher {
     if constexpr (kHasSegFold) {
       if constexpr (dev::segfold_eligible<CL>()) {
         if (C == 0) return ACC_OK;
-        const int grid = std::min((C + dev::kBlock / 32 - 1) / (dev::kBlock / 32), sm_count() * 8);
-        dev::k_segfold<CL><<<grid, dev::kBlock, 0, L.stream>>>(a);
+        constexpr int NFOLD = dev::count_if<CL>(dev::is_segfold_root);
+        const int grid = seg_grid(L);
+        const int per_block = dev::kSegTilesPerBlock;
+        const size_t smem = (size_t)NFOLD * dev::kSegTile * 4;
+        const bool v4 = seg_vec_ok(L);
+        auto kern = v4 ? dev::k_segfold<CL, true> : dev::k_segfold<CL, false>;
+        static int granted[2][64];
+        if (smem > 48 * 1024 && !opt_in_shared_memory(kern, smem, granted[v4 ? 1 : 0]))
+          return set_error(ACC_ERR_CUDA, "shared-memory opt-in failed: %s", cudaGetErrorString(cudaGetLastError()));
+        kern<<<grid, dev::kBlock, smem, L.stream>>>(a, per_block);
+        dev::k_segfold_across<CL><<<(grid + dev::kBlock / 32 - 1) / (dev::kBlock / 32), dev::kBlock, 0, L.stream>>>(a, grid);
         const cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return set_error(ACC_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
         return ACC_OK;
@@ -492,8 +527,10 @@ struct Passes {
 template <class CL>
 struct Registrar {
   explicit Registrar(const char* name) {
+    // (a cluster of segmented folds is a walk over the elements and a small second launch for the segments that
+    // cross its blocks)
     register_kernel(KernelEntry{signature(CL::c), name, &Passes<CL>::scratch_bytes, &Passes<CL>::launch,
-                                Passes<CL>::plan.n > 1 ? Passes<CL>::plan.n : 1});
+                                Passes<CL>::plan.n > 1 ? Passes<CL>::plan.n : (dev::count_if<CL>(dev::is_segfold_root) > 0 ? 2 : 1)});
   }
 };
 

@@ -2,24 +2,41 @@
 // array:  ys[s] = fold(op) of xs[off[s] .. off[s+1]),  xs evaluated in registers from the
 // fused producers.
 //
-// A warp takes a segment and walks it with coalesced reads, ending in a shuffle tree; eight
-// consecutive segments go to the eight warps of a block.  A segment longer than kSegLong
-// elements is set aside and reduced by the whole block afterwards, so that one long segment
-// does not hold a single warp for its whole length.  Several segmented folds of one cluster
-// (say a sum and a maximum over the same segments) share the walk and every load their
-// producers have in common.  Results do not depend on timing: the order of combination is
-// fixed by the thread layout.
+// The work is cut by elements, not by segments, so that a few very long segments among many
+// short ones (skewed lengths) cost what their elements cost:
 //
-// Offsets are data, so they are checked here: a segment that leaves the source is skipped
-// and reported as ACC_ERR_INDEX_RANGE, an empty or descending one as ACC_ERR_SHAPE (a fold
-// has no seed, so an empty segment has no value).
+//  * the source range is cut into tiles of kSegTile elements; a block owns a contiguous run of
+//    tiles and walks it in order.  It evaluates a tile's operands with coalesced (128-bit where
+//    the arrays allow) reads into shared memory, one array per fold;
+//  * the pieces of segments inside the tile are reduced from shared memory: a thread per piece
+//    up to kSegShort elements, a warp per piece up to kSegMedium, the whole block beyond;
+//  * a piece that is a whole segment is written at once.  A segment that crosses tiles is carried
+//    by the block from tile to tile (a compensated running value in one thread); one that crosses
+//    blocks leaves a record per block (the part after its start: `tail`; a part that continues
+//    one begun earlier: `head`), and a second, small launch (k_segfold_across) combines the
+//    records in block order.
+//
+// Several segmented folds of one cluster (say a sum and a maximum over the same segments) share
+// the walk.  Results do not depend on timing: every order of combination is fixed by the layout.
+//
+// Offsets are data, so they are checked here, every one of them: a segment that leaves the
+// source is reported as ACC_ERR_INDEX_RANGE, an empty or descending one as ACC_ERR_SHAPE (a fold
+// has no seed, so an empty segment has no value); pieces are clamped to their tile, so bad
+// offsets cannot make the kernel read or write outside its arrays.
 #pragma once
 #include "skeletons.cuh"
 
 namespace acc {
 namespace dev {
 
-constexpr int kSegLong = 1 << 14;
+constexpr int kSegTile = 4096;                 // elements per tile
+constexpr int kSegShort = 16;                  // pieces up to here: one thread
+constexpr int kSegMedium = 1024;               // pieces up to here: one warp; longer ones: the block
+constexpr int kSegListCap = kSegTile / (kSegShort + 1) + 2;
+constexpr int kSegBigCap = kSegTile / (kSegMedium + 1) + 2;    // pieces of a tile the whole block reduces
+constexpr int kSegResident = 4;                // blocks per SM the kernel is built for
+constexpr int kSegTilesPerBlock = 16;          // a block's run of tiles: short enough for the block scheduler to even out slow and fast runs
+constexpr int kSegWindow = 1024;               // offsets kept in shared memory at a time
 constexpr uint32_t kStatusEmptySegment = 4u;
 
 template <class CL> constexpr int first_segfold() {
@@ -40,63 +57,151 @@ template <class CL> constexpr bool segfold_eligible() {
   return true;
 }
 
-template <class CL>
-__global__ void __launch_bounds__(kBlock) k_segfold(const __grid_constant__ Args<CL::c.n> a) {
+// Scratch of k_segfold (32-bit words): from word 4 two records per block, `head`
+// then `tail`, of 2 + NF words each: segment id + 1 (0: no record), unused, one value per fold.
+__host__ __device__ inline int seg_record_words(int n_folds) { return 2 + n_folds; }
+__host__ __device__ inline int64_t seg_scratch_words(int n_folds, int grid) { return 4 + (int64_t)grid * 2 * seg_record_words(n_folds); }
+
+// Largest s in [0, S) with off[s] <= x, for off[0] <= x < off[S] (any s for other x): a 32-way search by one warp.
+__device__ __forceinline__ int seg_containing(const int32_t* off, int S, int x, int lane) {
+  int lo = 0, hi = S;                                          // off[lo] <= x < off[hi]
+  while (hi - lo > 1) {
+    const int step = (hi - lo + 31) / 32;
+    const int p = lo + (lane + 1) * step;
+    const bool ok = p < hi && __ldg(off + p) <= x;             // true for a prefix of the lanes
+    const int k = __popc(__ballot_sync(0xFFFFFFFFu, ok));
+    const int nlo = lo + k * step;
+    hi = min(hi, nlo + step);
+    lo = nlo;
+  }
+  return lo;
+}
+
+template <class CL, bool VEC>
+__global__ void __launch_bounds__(kBlock, kSegResident) k_segfold(const __grid_constant__ Args<CL::c.n> a, int tiles_per_block) {
   constexpr int N = CL::c.n;
   constexpr int F = first_segfold<CL>();
+  constexpr int NF = count_if<CL>(is_segfold_root);
   constexpr int WARPS = kBlock / 32;
+  constexpr int REC = 2 + NF;
+  extern __shared__ uint32_t seg_vals[];                         // NF arrays of kSegTile operand values
   __shared__ uint32_t red[WARPS];
-  __shared__ int long_list[WARPS];
-  __shared__ int n_long;
+  __shared__ int off_win[kSegWindow + 1];                        // offsets of segments win_base .. win_base + kSegWindow
+  __shared__ int long_seg[kSegListCap], long_lo[kSegListCap], long_hi[kSegListCap], long_kind[kSegListCap];
+  __shared__ int big_seg[kSegBigCap], big_lo[kSegBigCap], big_hi[kSegBigCap], big_kind[kSegBigCap];
+  __shared__ int n_long, n_big, next_s, first_open, have_first, have_last, last_seg;
+  __shared__ uint32_t first_val[NF], last_val[NF];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int S = a.C;                                               // segments
+  const int S = a.C;                                             // segments
   constexpr int OFF = CL::c.nodes[F].in[1], SRC = CL::c.nodes[F].in[0];
   const int32_t* off = reinterpret_cast<const int32_t*>(a.n[OFF].ptr);
   const int n_src = a.n[SRC].R * a.n[SRC].C;
+  uint32_t* rec = a.scratch + 4;
 
-  for (int base = blockIdx.x * WARPS; base < S; base += gridDim.x * WARPS) {
-    __syncthreads();
-    if (threadIdx.x == 0) n_long = 0;
-    __syncthreads();
-    const int s = base + warp;
-    if (s < S) {
-      const int lo = __ldg(off + s), hi = __ldg(off + s + 1);
-      if (lo < 0 || hi > n_src) {
-        if (lane == 0) atomicOr(a.status, kStatusIndex);
-      } else if (hi <= lo) {
-        if (lane == 0) atomicOr(a.status, kStatusEmptySegment);
-      } else if (hi - lo > kSegLong) {
-        if (lane == 0) long_list[atomicAdd(&n_long, 1)] = s;
-      } else {
-        uint32_t acc[N];
-        float comp[N] = {};                              // see fold_step
-        static_for<0, N>([&](auto ic) {
-          constexpr int i = decltype(ic)::value;
-          constexpr CNode nd = CL::c.nodes[i];
-          if constexpr (is_segfold_root(nd)) acc[i] = identity_of<nd.fn, nd.dtype>();
-        });
-        for (int j = lo + lane; j < hi; j += 32) {
-          static_for<0, N>([&](auto ic) {
-            constexpr int i = decltype(ic)::value;
-            constexpr CNode nd = CL::c.nodes[i];
-            if constexpr (is_segfold_root(nd)) fold_step<nd.fn, nd.dtype>(acc[i], comp[i], eval<CL, nd.in[0]>(a, Ix{0, j}));
-          });
-        }
-        static_for<0, N>([&](auto ic) {
-          constexpr int i = decltype(ic)::value;
-          constexpr CNode nd = CL::c.nodes[i];
-          if constexpr (is_segfold_root(nd)) {
-            const uint32_t v = warp_reduce<nd.fn, nd.dtype>(acc[i]);
-            if (lane == 0) reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr))[s] = v;
-          }
-        });
+  // every offset is looked at once, whatever the walk below does with it
+  for (int s = blockIdx.x * kBlock + threadIdx.x; s < S; s += gridDim.x * kBlock) {
+    const int lo = __ldg(off + s), hi = __ldg(off + s + 1);
+    if (lo < 0 || hi > n_src) atomicOr(a.status, kStatusIndex);
+    else if (hi <= lo) atomicOr(a.status, kStatusEmptySegment);
+  }
+
+  auto fold_slot_of = [](int i) { return count_if<CL>(is_segfold_root, i); };
+  // kind of a piece: bit 0 = it continues a segment begun before the tile, bit 1 = its segment goes on after the tile
+  auto store_piece = [&](int s, int kind, const uint32_t (&v)[N]) {
+    static_for<0, N>([&](auto ic) {
+      constexpr int i = decltype(ic)::value;
+      if constexpr (is_segfold_root(CL::c.nodes[i])) {
+        const int f = fold_slot_of(i);
+        if (kind & 1) first_val[f] = v[i];
+        else if (kind & 2) last_val[f] = v[i];
+        else reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr))[s] = v[i];
       }
+    });
+    if (kind & 1) { have_first = 1; first_open = kind >> 1; }
+    else if (kind & 2) { have_last = 1; last_seg = s; }
+  };
+  // Inside a tile sums are plain: a thread adds at most 32 staged values and trees do the rest, which
+  // stays far inside the tolerance; what is compensated is the running value a segment keeps from
+  // tile to tile (thousands of steps for a long one).
+  auto reduce_strided = [&](int plo, int phi, int first, int stride, int tile_lo, uint32_t (&v)[N]) {
+    uint32_t w[4][N];
+    static_for<0, N>([&](auto ic) {
+      constexpr int i = decltype(ic)::value;
+      constexpr CNode nd = CL::c.nodes[i];
+      if constexpr (is_segfold_root(nd)) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) w[u][i] = identity_of<nd.fn, nd.dtype>();
+      }
+    });
+    int j = plo + first;
+    for (; j + 3 * stride < phi; j += 4 * stride) {              // four independent running values per fold
+      static_for<0, N>([&](auto ic) {
+        constexpr int i = decltype(ic)::value;
+        constexpr CNode nd = CL::c.nodes[i];
+        if constexpr (is_segfold_root(nd)) {
+          const uint32_t* src = seg_vals + fold_slot_of(i) * kSegTile - tile_lo;
+#pragma unroll
+          for (int u = 0; u < 4; ++u) w[u][i] = combine<nd.fn, nd.dtype>(w[u][i], src[j + u * stride]);
+        }
+      });
     }
-    __syncthreads();
-    const int todo = n_long;
-    for (int k = 0; k < todo; ++k) {                              // long segments: the whole block each
-      const int t = long_list[k];
-      const int lo = __ldg(off + t), hi = __ldg(off + t + 1);
+    for (; j < phi; j += stride) {
+      static_for<0, N>([&](auto ic) {
+        constexpr int i = decltype(ic)::value;
+        constexpr CNode nd = CL::c.nodes[i];
+        if constexpr (is_segfold_root(nd)) w[0][i] = combine<nd.fn, nd.dtype>(w[0][i], (seg_vals + fold_slot_of(i) * kSegTile - tile_lo)[j]);
+      });
+    }
+    static_for<0, N>([&](auto ic) {
+      constexpr int i = decltype(ic)::value;
+      constexpr CNode nd = CL::c.nodes[i];
+      if constexpr (is_segfold_root(nd))
+        v[i] = combine<nd.fn, nd.dtype>(combine<nd.fn, nd.dtype>(w[0][i], w[1][i]), combine<nd.fn, nd.dtype>(w[2][i], w[3][i]));
+    });
+  };
+
+  const int e_lo = max(__ldg(off), 0), e_hi = min(__ldg(off + S), n_src);   // elements that belong to segments
+  const int first_tile = blockIdx.x * tiles_per_block;
+  int s_cur = 0;                                                 // the segment that holds the next element to process (uniform)
+  int win_base = -1;                                             // first segment of the offsets window, -1: not filled (uniform)
+  // the block's carry: the running value of the segment that is open at the end of the last tile (thread 0)
+  int carry_seg = -1;
+  bool carry_from_here = false;
+  uint32_t carry[N];
+  float carry_comp[N] = {};
+
+  for (int t = 0; t < tiles_per_block; ++t) {                    // (a run of tiles inside one segment advances t by its length)
+    const int64_t tile_lo64 = (int64_t)(first_tile + t) * kSegTile;
+    if (tile_lo64 >= e_hi) break;
+    const int tile_lo = (int)tile_lo64;
+    const int tile_hi = (int)(tile_lo64 + kSegTile < (int64_t)e_hi ? tile_lo64 + kSegTile : (int64_t)e_hi);
+    const int lo0 = max(tile_lo, e_lo);
+    if (lo0 >= tile_hi) continue;
+    __syncthreads();                                             // the previous tile's values and flags have been read
+    if (win_base < 0) {                                          // the block's first tile: which segment holds its first element
+      if (warp == 0) {
+        const int s0 = seg_containing(off, S, lo0, lane);
+        if (lane == 0) next_s = s0;
+      }
+      __syncthreads();
+      s_cur = next_s;
+      __syncthreads();
+    }
+    if (win_base < 0 || s_cur + kBlock > win_base + kSegWindow) {  // uniform: the window of offsets moves up to s_cur
+      win_base = s_cur;
+      for (int k = threadIdx.x; k <= kSegWindow; k += kBlock) off_win[k] = s_cur + k <= S ? __ldg(off + s_cur + k) : 0x7FFFFFFF;
+      __syncthreads();
+    }
+    if (threadIdx.x == 0) { n_long = 0; n_big = 0; have_first = 0; have_last = 0; first_open = 0; next_s = s_cur; }
+    // Tiles that lie inside one segment need no staging: the block streams through all of them that are
+    // its own, every thread keeping a compensated running value per fold, and reduces once at the end.
+    const int lo_c = off_win[s_cur - win_base], hi_c = off_win[s_cur - win_base + 1];
+    const bool whole = s_cur < S && lo_c <= lo0 && hi_c >= tile_hi && lo0 == tile_lo && tile_hi - tile_lo == kSegTile;
+    if (whole) {                                                 // uniform
+      const int own_end = first_tile + tiles_per_block;          // first tile that is not this block's
+      const int inside_end = min(hi_c, e_hi) / kSegTile;         // first tile that is not wholly inside the segment
+      const int run = max(1, min(own_end, inside_end) - (first_tile + t));
+      const int run_hi = tile_lo + run * kSegTile;               // (no overflow: run_hi <= e_hi)
       uint32_t acc[N];
       float comp[N] = {};
       static_for<0, N>([&](auto ic) {
@@ -104,22 +209,223 @@ __global__ void __launch_bounds__(kBlock) k_segfold(const __grid_constant__ Args
         constexpr CNode nd = CL::c.nodes[i];
         if constexpr (is_segfold_root(nd)) acc[i] = identity_of<nd.fn, nd.dtype>();
       });
-      for (int j = lo + (int)threadIdx.x; j < hi; j += kBlock) {
-        static_for<0, N>([&](auto ic) {
-          constexpr int i = decltype(ic)::value;
-          constexpr CNode nd = CL::c.nodes[i];
-          if constexpr (is_segfold_root(nd)) fold_step<nd.fn, nd.dtype>(acc[i], comp[i], eval<CL, nd.in[0]>(a, Ix{0, j}));
-        });
+      if constexpr (VEC) {
+        // a tile is four trips of the block, so the run is a whole number of these steps: four chunks in flight per fold
+        for (int c = tile_lo + (int)threadIdx.x * 4; c < run_hi; c += kSegTile) {
+          static_for<0, N>([&](auto ic) {
+            constexpr int i = decltype(ic)::value;
+            constexpr CNode nd = CL::c.nodes[i];
+            if constexpr (is_segfold_root(nd)) {
+              V4 x[kSegTile / (4 * kBlock)];
+#pragma unroll
+              for (int u = 0; u < kSegTile / (4 * kBlock); ++u) x[u] = eval<CL, nd.in[0]>(a, Ix4{0, c + u * kBlock * 4});
+#pragma unroll
+              for (int u = 0; u < kSegTile / (4 * kBlock); ++u)
+                fold_step<nd.fn, nd.dtype>(acc[i], comp[i], combine<nd.fn, nd.dtype>(combine<nd.fn, nd.dtype>(x[u].v[0], x[u].v[1]),
+                                                                                     combine<nd.fn, nd.dtype>(x[u].v[2], x[u].v[3])));
+            }
+          });
+        }
+      } else {
+        for (int q = tile_lo + (int)threadIdx.x; q < run_hi; q += kBlock) {
+          static_for<0, N>([&](auto ic) {
+            constexpr int i = decltype(ic)::value;
+            constexpr CNode nd = CL::c.nodes[i];
+            if constexpr (is_segfold_root(nd)) fold_step<nd.fn, nd.dtype>(acc[i], comp[i], eval<CL, nd.in[0]>(a, Ix{0, q}));
+          });
+        }
       }
+      uint32_t v[N];
       static_for<0, N>([&](auto ic) {
         constexpr int i = decltype(ic)::value;
         constexpr CNode nd = CL::c.nodes[i];
-        if constexpr (is_segfold_root(nd)) {
-          const uint32_t v = block_reduce<nd.fn, nd.dtype>(acc[i], red);
-          if (threadIdx.x == 0) reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr))[t] = v;
-        }
+        if constexpr (is_segfold_root(nd)) v[i] = block_reduce<nd.fn, nd.dtype>(acc[i], red);
       });
+      if (threadIdx.x == 0) {
+        store_piece(s_cur, (lo_c < lo0 ? 1 : 0) | (hi_c > run_hi ? 2 : 0), v);
+        next_s = hi_c > run_hi ? s_cur : s_cur + 1;
+      }
+      t += run - 1;
+    } else {
+    // stage the operands of the tile
+    static_for<0, N>([&](auto ic) {
+      constexpr int i = decltype(ic)::value;
+      constexpr CNode nd = CL::c.nodes[i];
+      if constexpr (is_segfold_root(nd)) {
+        uint32_t* dst = seg_vals + fold_slot_of(i) * kSegTile;
+        if constexpr (VEC) {
+          V4 v[kSegTile / (4 * kBlock)];
+#pragma unroll
+          for (int j = 0; j < kSegTile / (4 * kBlock); ++j) {
+            const int c = tile_lo + (j * kBlock + (int)threadIdx.x) * 4;
+            if (c < tile_hi) v[j] = eval<CL, nd.in[0]>(a, Ix4{0, c});
+          }
+#pragma unroll
+          for (int j = 0; j < kSegTile / (4 * kBlock); ++j) {
+            const int q = (j * kBlock + (int)threadIdx.x) * 4;
+            if (tile_lo + q < tile_hi) *reinterpret_cast<uint4*>(dst + q) = make_uint4(v[j].v[0], v[j].v[1], v[j].v[2], v[j].v[3]);
+          }
+        } else {
+          for (int q = threadIdx.x; q < tile_hi - tile_lo; q += kBlock) dst[q] = eval<CL, nd.in[0]>(a, Ix{0, tile_lo + q});
+        }
+      }
+    });
+
+    // the pieces of the tile, a thread per segment; those beyond kSegShort elements are set aside
+    for (int base = s_cur;; base += kBlock) {
+      if (win_base < 0 || base + kBlock > win_base + kSegWindow) {     // uniform: the window moves up to `base`
+        __syncthreads();
+        win_base = base;
+        for (int k = threadIdx.x; k <= kSegWindow; k += kBlock) off_win[k] = base + k <= S ? __ldg(off + base + k) : 0x7FFFFFFF;
+      }
+      __syncthreads();
+      const int s = base + (int)threadIdx.x;
+      const int lo_s = off_win[s - win_base], hi_s = off_win[s - win_base + 1];
+      const bool beyond = s >= S || lo_s >= tile_hi;
+      if (!beyond) {
+        const int plo = max(lo_s, lo0), phi = min(hi_s, tile_hi);
+        if (hi_s >= tile_hi) next_s = hi_s > tile_hi ? s : s + 1;      // the segment that holds the tile's last element
+        if (phi > plo) {
+          const int kind = (lo_s < lo0 ? 1 : 0) | (hi_s > tile_hi ? 2 : 0);
+          if (phi - plo <= kSegShort) {
+            uint32_t v[N];
+            reduce_strided(plo, phi, 0, 1, tile_lo, v);
+            store_piece(s, kind, v);
+          } else if (phi - plo <= kSegMedium) {
+            const int at = atomicAdd(&n_long, 1);
+            if (at < kSegListCap) { long_seg[at] = s; long_lo[at] = plo; long_hi[at] = phi; long_kind[at] = kind; }
+          } else {
+            const int at = atomicAdd(&n_big, 1);
+            if (at < kSegBigCap) { big_seg[at] = s; big_lo[at] = plo; big_hi[at] = phi; big_kind[at] = kind; }
+          }
+        }
+      }
+      if (__syncthreads_or(beyond)) break;
     }
+    const int todo = min(n_long, kSegListCap);
+    // a warp per piece of medium length
+    for (int k = warp; k < todo; k += WARPS) {
+      const int plo = long_lo[k], phi = long_hi[k];
+      uint32_t v[N];
+      reduce_strided(plo, phi, lane, 32, tile_lo, v);
+      static_for<0, N>([&](auto ic) {
+        constexpr int i = decltype(ic)::value;
+        constexpr CNode nd = CL::c.nodes[i];
+        if constexpr (is_segfold_root(nd)) v[i] = warp_reduce<nd.fn, nd.dtype>(v[i]);
+      });
+      if (lane == 0) store_piece(long_seg[k], long_kind[k], v);
+    }
+    // the whole block per piece beyond that (at most three of them in a tile)
+    const int todo_big = min(n_big, kSegBigCap);
+    for (int k = 0; k < todo_big; ++k) {
+      const int plo = big_lo[k], phi = big_hi[k];
+      uint32_t v[N];
+      reduce_strided(plo, phi, (int)threadIdx.x, kBlock, tile_lo, v);
+      static_for<0, N>([&](auto ic) {
+        constexpr int i = decltype(ic)::value;
+        constexpr CNode nd = CL::c.nodes[i];
+        if constexpr (is_segfold_root(nd)) v[i] = block_reduce<nd.fn, nd.dtype>(v[i], red);
+      });
+      if (threadIdx.x == 0) store_piece(big_seg[k], big_kind[k], v);
+    }
+    }
+    __syncthreads();
+
+    // segments that cross the tile's ends: the block's running value
+    if (threadIdx.x == 0) {
+      if (have_first) {
+        if (carry_seg != s_cur) {                              // begun before this block: nothing carried yet
+          carry_seg = s_cur;
+          carry_from_here = false;
+          static_for<0, N>([&](auto ic) {
+            constexpr int i = decltype(ic)::value;
+            if constexpr (is_segfold_root(CL::c.nodes[i])) { carry[i] = first_val[fold_slot_of(i)]; carry_comp[i] = 0.0f; }
+          });
+        } else {
+          static_for<0, N>([&](auto ic) {
+            constexpr int i = decltype(ic)::value;
+            constexpr CNode nd = CL::c.nodes[i];
+            if constexpr (is_segfold_root(nd)) fold_step<nd.fn, nd.dtype>(carry[i], carry_comp[i], first_val[fold_slot_of(i)]);
+          });
+        }
+        if (!first_open) {                                     // the segment ends in this tile
+          uint32_t* head = rec + (size_t)blockIdx.x * 2 * REC;
+          if (!carry_from_here) head[0] = (uint32_t)carry_seg + 1u;
+          static_for<0, N>([&](auto ic) {
+            constexpr int i = decltype(ic)::value;
+            if constexpr (is_segfold_root(CL::c.nodes[i])) {
+              if (carry_from_here) reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr))[carry_seg] = carry[i];
+              else head[2 + fold_slot_of(i)] = carry[i];
+            }
+          });
+          carry_seg = -1;
+        }
+      }
+      if (have_last) {
+        carry_seg = last_seg;
+        carry_from_here = true;
+        static_for<0, N>([&](auto ic) {
+          constexpr int i = decltype(ic)::value;
+          if constexpr (is_segfold_root(CL::c.nodes[i])) { carry[i] = last_val[fold_slot_of(i)]; carry_comp[i] = 0.0f; }
+        });
+      }
+    }
+    s_cur = next_s;                                              // written before the barrier above, by the one thread that saw it
+  }
+
+  // what is still open where the block's run of tiles ends
+  if (threadIdx.x == 0 && carry_seg >= 0) {
+    uint32_t* r = rec + ((size_t)blockIdx.x * 2 + (carry_from_here ? 1 : 0)) * REC;
+    r[0] = (uint32_t)carry_seg + 1u;
+    static_for<0, N>([&](auto ic) {
+      constexpr int i = decltype(ic)::value;
+      if constexpr (is_segfold_root(CL::c.nodes[i])) r[2 + fold_slot_of(i)] = carry[i];
+    });
+  }
+}
+
+// Second launch of a segmented-fold cluster: segments that cross the blocks of k_segfold.  A warp per block
+// that left a `tail` (the part of a segment after its start): its lanes look at the blocks that follow, 32 at a
+// time, take the `head` records that continue the segment, and combine them in a fixed order.
+template <class CL>
+__global__ void __launch_bounds__(kBlock) k_segfold_across(const __grid_constant__ Args<CL::c.n> a, int n_blocks) {
+  constexpr int N = CL::c.n;
+  constexpr int NF = count_if<CL>(is_segfold_root);
+  constexpr int REC = 2 + NF;
+  auto fold_slot_of = [](int i) { return count_if<CL>(is_segfold_root, i); };
+  const int lane = threadIdx.x & 31;
+  const int b = blockIdx.x * (kBlock / 32) + ((int)threadIdx.x >> 5);
+  if (b >= n_blocks) return;
+  const uint32_t* rec = a.scratch + 4;
+  const uint32_t* tail = rec + ((size_t)b * 2 + 1) * REC;
+  const uint32_t key = tail[0];
+  if (key == 0) return;                                          // the same for the whole warp
+  uint32_t v[N];
+  static_for<0, N>([&](auto ic) {
+    constexpr int i = decltype(ic)::value;
+    if constexpr (is_segfold_root(CL::c.nodes[i])) v[i] = tail[2 + fold_slot_of(i)];
+  });
+  for (int base = b + 1; base < n_blocks; base += 32) {
+    const int b2 = base + lane;
+    const uint32_t* head = rec + (size_t)min(b2, n_blocks - 1) * 2 * REC;
+    const bool same = b2 < n_blocks && head[0] == key;
+    const unsigned others = ~__ballot_sync(0xFFFFFFFFu, same);
+    const int n = others ? __ffs(others) - 1 : 32;               // blocks of this round that continue the segment
+    static_for<0, N>([&](auto ic) {
+      constexpr int i = decltype(ic)::value;
+      constexpr CNode nd = CL::c.nodes[i];
+      if constexpr (is_segfold_root(nd)) {
+        const uint32_t x = lane < n ? head[2 + fold_slot_of(i)] : identity_of<nd.fn, nd.dtype>();
+        v[i] = combine<nd.fn, nd.dtype>(v[i], warp_reduce<nd.fn, nd.dtype>(x));
+      }
+    });
+    if (n < 32) break;
+  }
+  if (lane == 0) {
+    static_for<0, N>([&](auto ic) {
+      constexpr int i = decltype(ic)::value;
+      if constexpr (is_segfold_root(CL::c.nodes[i])) reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr))[key - 1] = v[i];
+    });
   }
 }
 

@@ -19,7 +19,9 @@ def check_program(prog, partitions="all", runs=1, passes=False, inputs_t=None):
     inputs_t = W.make_inputs(prog) if inputs_t is None else inputs_t
     ref = oracle_run(prog, np_inputs(inputs_t))
     got, g = gpu_run(prog, inputs_t, None, B.UNFUSED)
-    assert g.launch_count() == sum(nd.kind != "input" for nd in prog.nodes)
+    # one launch per combinator; a segmented fold takes a second, small one for the segments that cross its blocks
+    assert g.launch_count() == sum((nd.kind != "input") + (nd.kind == "foldseg") for nd in prog.nodes)
+    passes = passes or any(nd.kind == "foldseg" for nd in prog.nodes)
     compare(prog, ref, got, f"{prog.name} unfused")
     pis = all_partitions(prog) if partitions == "all" else partitions
     for pi in pis:
@@ -417,10 +419,12 @@ def compare_hist(prog, ref, got, what):
     assert 3 not in got or np.array_equal(got[3], ref.values[3]), what
 
 
-@pytest.mark.parametrize("n,segments", [(5, 1), (64, 5), (1000, 16), (100000, 300), (1 << 20, 1 << 12), (1 << 20, 6)])
+@pytest.mark.parametrize("n,segments", [(5, 1), (64, 5), (1000, 16), (100000, 300), (1 << 20, 1 << 12), (1 << 20, 6), (1 << 22, 1 << 18),
+                                        ((1 << 21) + 3, 1 << 10)])
 def test_segmented_fold(n, segments):
-    # warp-per-segment walk, segments longer than 2^14 elements by the whole block (the last two shapes),
-    # a sum fed by a fused map and a maximum sharing the same walk
+    # the source is walked in tiles of 4096 elements; pieces of segments by a thread, a warp or the block according to
+    # their length; segments that cross tiles and blocks; a sum fed by a fused map and a maximum sharing the same walk;
+    # a source without 128-bit rows (the last shape)
     from paper_2407_13585_b200 import binding as B
     prog = W.segmented_sums(n, segments)
     runnable = [pi for pi in all_partitions(prog) if pi != [-1, -1, 0, 1, 0]]
@@ -432,6 +436,37 @@ def test_segmented_fold(n, segments):
     with pytest.raises(B.AccError) as e:
         gpu_run(prog, inputs, [-1, -1, 0, 1, 0], B.FUSED)
     assert e.value.status == "ACC_ERR_NO_KERNEL"
+
+
+def test_segmented_fold_with_skewed_and_awkward_segments():
+    """One segment with 90 % of 2^22 elements among short ones; segments that begin or end exactly on tile and block
+    boundaries, single elements on either side of a boundary, and offsets that leave the ends of the source out."""
+    import torch
+    from paper_2407_13585_b200 import binding as B
+    n = 1 << 22
+    T = 4096
+    cuts = {100, 101, 117, 130, T - 1, T, T + 1, 2 * T, 2 * T + 16, 2 * T + 17, 5 * T + 2000}      # short pieces around tile ends
+    big_lo = 6 * T + 123
+    big_hi = big_lo + (n * 9) // 10                                                             # 90 % of the elements in one segment
+    cuts |= {big_lo, big_hi}
+    x = big_hi
+    k = 0
+    while x < n - 40000:                                                                           # lengths 1, 2, 3, ... 1500 after it
+        k = k % 1500 + 1
+        x += k
+        cuts.add(x)
+    cuts |= {n - 40000 + 3 * T, n - 9}                                                             # a last long piece; the source's end is left out
+    offsets = torch.tensor(sorted(cuts), dtype=torch.int32)
+    segments = offsets.numel() - 1
+    prog = W.segmented_sums(n, segments)
+    inputs = W.make_inputs(prog)
+    inputs[1] = offsets
+    check_program(prog, [[-1, -1, 0, 0, 0], [-1, -1, 0, 1, 2]], inputs_t=inputs)
+    # the same walk on equal addends: the long segment's sum crosses hundreds of tiles and dozens of blocks
+    inputs[0] = torch.full((n,), 0.1)
+    ref = oracle_run(prog, np_inputs(inputs))
+    got, _ = gpu_run(prog, inputs, [-1, -1, 0, 0, 0], B.FUSED)
+    compare(prog, ref, got, "skewed segments, equal addends")
 
 
 def test_segmented_fold_reports_bad_offsets():
