@@ -9,6 +9,7 @@
 #include "hist.cuh"
 #include "segfold.cuh"
 #include "skeletons.cuh"
+#include "slabgather.cuh"
 #include "stencil.cuh"
 #include "tile.cuh"
 
@@ -138,6 +139,19 @@ struct Launcher {
     return true;
   }
 
+  // Whether the gather below the scan runs as slab passes: decided by shapes alone, so that the scratch
+  // layout (which is fixed before any pointer is known) and the launch agree.
+  static constexpr bool kSlabShape = dev::slab_gather_eligible<CL>();
+  static bool slab_shapes_ok(const ClusterLaunch& L, int R, int C) {
+    if constexpr (kSlabShape) {
+      const int src = CL::c.nodes[dev::the_gather<CL>()].in[1];
+      const int64_t src_bytes = (int64_t)L.nodes[src].R * L.nodes[src].C * 4;
+      return R == 1 && C >= dev::kSlabMinElements && C % 4 == 0 && src_bytes >= dev::kSlabMinSourceBytes && src_bytes <= dev::kSlabMaxSourceBytes;
+    } else {
+      return false;
+    }
+  }
+
   static int64_t scratch_bytes(const ClusterLaunch& L) {
     int R, C;
     if (!domain(L, R, C)) return ACC_ERR_NO_KERNEL;
@@ -145,7 +159,14 @@ struct Launcher {
       const int blocks = (R + dev::kTile - 1) / dev::kTile;
       return (dev::tile_partials_off(blocks) + (int64_t)kRowFolds * blocks * R) * 4;
     }
-    if (kHasScan) return 16 + (int64_t)R * ((C + kScanTile - 1) / kScanTile) * 8;
+    if (kHasScan) {
+      int64_t bytes = 16 + (int64_t)R * ((C + kScanTile - 1) / kScanTile) * 8;
+      if (slab_shapes_ok(L, R, C)) {                      // + group sizes and slab codes of the slab passes (slabgather.cuh)
+        const int64_t full = C / dev::kSlabWarpTile;
+        bytes = ((bytes + 15) & ~int64_t(15)) + full * 4 + full * 32 * 4;
+      }
+      return bytes;
+    }
     if (kHasSegFold) return dev::seg_scratch_words(dev::count_if<CL>(dev::is_segfold_root), seg_grid(L)) * 4;
     if (kHasRowFold) return 0;
     int64_t words = dev::stream_acc64_off(kScalarFolds, sm_count() * 8);
@@ -349,6 +370,28 @@ struct Launcher {
       const int64_t tiles = (int64_t)R * per_row;
       if (tiles >= (int64_t(1) << 31)) return set_error(ACC_ERR_SHAPE, "too many rows to scan in one launch");
       const int grid = (int)std::min<int64_t>(tiles, (int64_t)sm_count() * (1536 / kScanBlock));
+      if constexpr (kSlabShape) {
+        if (vec && slab_shapes_ok(L, R, C)) {
+          // partition the indices by slab, gather slab by slab from L2, merge and scan (slabgather.cuh)
+          const int src = CL::c.nodes[dev::the_gather<CL>()].in[1];
+          const int64_t n_src = (int64_t)L.nodes[src].R * L.nodes[src].C;
+          const uint32_t mul = (uint32_t)(((uint64_t)dev::kSlabs << 32) / (uint64_t)n_src);
+          const int full = C / dev::kSlabWarpTile;
+          const int64_t states = ((16 + tiles * 8) + 15) & ~int64_t(15);
+          uint32_t* counts = L.scratch + states / 4;
+          uint32_t* codes = counts + full;
+          const int warps = dev::kBlock / 32;
+          const int pgrid = (int)std::min<int64_t>((full + warps - 1) / warps, (int64_t)sm_count() * 4);
+          const int ggrid = (int)std::min<int64_t>((full + warps - 1) / warps, (int64_t)sm_count() * 8);
+          dev::k_slab_partition<CL><<<pgrid, dev::kBlock, 0, L.stream>>>(a, codes, counts, full, mul);
+          for (int k = 0; k < dev::kSlabs; ++k) dev::k_slab_gather<CL><<<ggrid, dev::kBlock, 0, L.stream>>>(a, counts, full, (uint32_t)k);
+          dev::k_scan_merge<CL><<<grid, kScanBlock, 0, L.stream>>>(a, per_row, (int)tiles, dev::SlabIn{codes, counts, full});
+          L.extra_launches = 1 + dev::kSlabs;
+          const cudaError_t e = cudaGetLastError();
+          if (e != cudaSuccess) return set_error(ACC_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+          return ACC_OK;
+        }
+      }
       if (vec) dev::k_scan<CL, true><<<grid, kScanBlock, 0, L.stream>>>(a, per_row, (int)tiles);
       else dev::k_scan<CL, false><<<grid, kScanBlock, 0, L.stream>>>(a, per_row, (int)tiles);
     } else if constexpr (kHasRowFold) {

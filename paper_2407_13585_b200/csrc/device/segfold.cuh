@@ -30,12 +30,12 @@ namespace acc {
 namespace dev {
 
 constexpr int kSegTile = 4096;                 // elements per tile
-constexpr int kSegShort = 16;                  // pieces up to here: one thread
+constexpr int kSegShort = 32;                  // pieces up to here: one thread
 constexpr int kSegMedium = 1024;               // pieces up to here: one warp; longer ones: the block
 constexpr int kSegListCap = kSegTile / (kSegShort + 1) + 2;
 constexpr int kSegBigCap = kSegTile / (kSegMedium + 1) + 2;    // pieces of a tile the whole block reduces
 constexpr int kSegResident = 4;                // blocks per SM the kernel is built for
-constexpr int kSegTilesPerBlock = 16;          // a block's run of tiles: short enough for the block scheduler to even out slow and fast runs
+constexpr int kSegTilesPerBlock = 8;           // a block's run of tiles: short enough for the block scheduler to even out slow and fast runs
 constexpr int kSegWindow = 1024;               // offsets kept in shared memory at a time
 constexpr uint32_t kStatusEmptySegment = 4u;
 
@@ -84,7 +84,7 @@ __global__ void __launch_bounds__(kBlock, kSegResident) k_segfold(const __grid_c
   constexpr int NF = count_if<CL>(is_segfold_root);
   constexpr int WARPS = kBlock / 32;
   constexpr int REC = 2 + NF;
-  extern __shared__ uint32_t seg_vals[];                         // NF arrays of kSegTile operand values
+  extern __shared__ __align__(16) uint32_t seg_vals[];                         // NF arrays of kSegTile operand values
   __shared__ uint32_t red[WARPS];
   __shared__ int off_win[kSegWindow + 1];                        // offsets of segments win_base .. win_base + kSegWindow
   __shared__ int long_seg[kSegListCap], long_lo[kSegListCap], long_hi[kSegListCap], long_kind[kSegListCap];

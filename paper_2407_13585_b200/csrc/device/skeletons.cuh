@@ -447,6 +447,28 @@ template <class CL, int I, class B> struct reads_staged<CL, I, IxSc<B>> { static
 template <class CL, int I, class A, class B>
 __device__ __forceinline__ val_of<B> ld_staged(const A&, const IxSc<B>& ix) { return ix.sv; }
 
+// A gather whose values were brought in by an earlier launch (slabgather.cuh): the index carries them, and the
+// gather member reads as those values.  As with IxSc, only index-preserving paths may lead to that member.
+template <class B> struct IxGv : B { val_of<B> gv; };
+template <class B> struct width_of<IxGv<B>> { static constexpr int value = width_of<B>::value; };
+template <class CL> constexpr int the_gather() {
+  int g = -1;
+  for (int i = 0; i < CL::c.n; ++i)
+    if (CL::c.nodes[i].member && CL::c.nodes[i].kind == ACC_GATHER) g = g < 0 ? i : -2;
+  return g < 0 ? -1 : g;
+}
+template <class CL, int I, class B> struct reads_staged<CL, I, IxGv<B>> { static constexpr bool value = I == the_gather<CL>(); };
+template <class CL, int I, class A, class B>
+__device__ __forceinline__ val_of<B> ld_staged(const A&, const IxGv<B>& ix) { return ix.gv; }
+
+// What the merging scan needs beside its cluster arguments (see slabgather.cuh); unused by the plain scan.
+struct SlabIn {
+  const uint32_t* codes = nullptr;     // per element of a full warp tile: which slab its gathered index fell in (2 bits; a word per lane)
+  const uint32_t* counts = nullptr;    // per full warp tile: how many of its elements fell in slabs 0, 1, 2 (10 bits each)
+  int full_tiles = 0;                  // warp tiles of kSlabWarpTile elements that the earlier launches covered
+};
+constexpr int kSlabWarpTile = 512;
+
 // Whether member i needs the value of scan s (through any chain of operands inside the cluster).
 constexpr bool needs_scan(const CCluster& c, int i, int s) {
   const CNode& n = c.nodes[i];
@@ -459,8 +481,8 @@ constexpr bool needs_scan(const CCluster& c, int i, int s) {
 // Rows of a rank-2 array are scanned independently: a row is cut into tiles of its own, the
 // look-back of a tile stops at the first tile of its row.  A right-to-left scan walks its row
 // from the far end: position p of the walk is element C-1-p of the row.
-template <class CL, bool VEC>
-__global__ void __launch_bounds__(scan_block<CL>()) k_scan(const __grid_constant__ Args<CL::c.n> a, int tiles_per_row, int n_tiles) {
+template <class CL, bool VEC, bool SLAB>
+__device__ __forceinline__ void scan_tiles(const Args<CL::c.n>& a, int tiles_per_row, int n_tiles, const SlabIn& slab) {
   constexpr int N = CL::c.n;
   constexpr int W = VEC ? 4 : 1;
   constexpr int BLOCK = scan_block<CL>();
@@ -477,6 +499,8 @@ __global__ void __launch_bounds__(scan_block<CL>()) k_scan(const __grid_constant
   __shared__ uint32_t warp_total[BLOCK / 32];
   __shared__ uint32_t tile_prefix;
   __shared__ int tile_id;
+  __shared__ __align__(16) uint32_t slab_stage[SLAB ? BLOCK / 32 : 1][SLAB ? kSlabWarpTile : 1];   // read and written 128 bits at a time
+  static_assert(!SLAB || (VEC && TILE == (BLOCK / 32) * kSlabWarpTile && !REV), "the merging scan walks rank-1 tiles of eight 512-element warp tiles");
   uint64_t* states = reinterpret_cast<uint64_t*>(a.scratch + 4);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int n = a.C;                                       // length of a row
@@ -497,6 +521,47 @@ __global__ void __launch_bounds__(scan_block<CL>()) k_scan(const __grid_constant
     const int warp_base = in_row * TILE + warp * (TILE / (BLOCK / 32));
 
     uint32_t val[ROWS][W];
+    // SLAB: the gathered values of this warp's 512 elements lie, grouped by slab, where the scan's results will go;
+    // they are put back into element order (positions from the slab codes: a stable counting sort undone)
+    V4 gathered[SLAB ? ROWS : 1];
+    bool merged = false;                                   // the same for a whole warp
+    if constexpr (SLAB) {
+      const int wt = tile * (BLOCK / 32) + warp;
+      if (wt < slab.full_tiles) {
+        merged = true;
+        const uint32_t code = __ldg(slab.codes + (size_t)wt * 32 + lane), cnt3 = __ldg(slab.counts + wt);
+        const uint32_t* staged = reinterpret_cast<const uint32_t*>(a.n[S].ptr) + (size_t)wt * kSlabWarpTile;
+        uint4 st[ROWS];
+#pragma unroll
+        for (int j = 0; j < ROWS; ++j) st[j] = *reinterpret_cast<const uint4*>(staged + (j * 32 + lane) * 4);
+        const uint32_t lo1 = code & 0x55555555u, hi1 = (code >> 1) & 0x55555555u;
+        const uint32_t n3 = __popc(lo1 & hi1), n2 = __popc(hi1 & ~lo1), n1 = __popc(lo1 & ~hi1);
+        const uint32_t c01 = (16u - n1 - n2 - n3) | (n1 << 16), c23 = n2 | (n3 << 16);     // this lane's elements per slab
+        uint32_t i01 = c01, i23 = c23;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const uint32_t u0 = __shfl_up_sync(0xFFFFFFFFu, i01, o), u1 = __shfl_up_sync(0xFFFFFFFFu, i23, o);
+          if (lane >= o) { i01 += u0; i23 += u1; }
+        }
+        const uint32_t t0 = cnt3 & 1023u, t1 = (cnt3 >> 10) & 1023u, t2 = (cnt3 >> 20) & 1023u;
+        uint32_t a01 = (i01 - c01) + (t0 << 16);                             // next position in the lists of slabs 0 | 1
+        uint32_t a23 = (i23 - c23) + (t0 + t1) + ((t0 + t1 + t2) << 16);     // ... of slabs 2 | 3
+        uint32_t* mine = slab_stage[warp];
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < ROWS; ++j) *reinterpret_cast<uint4*>(mine + (j * 32 + lane) * 4) = st[j];
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < ROWS; ++j)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const uint32_t sl = (code >> (2 * (4 * j + e))) & 3u;
+            const uint32_t sh = 16 * (sl & 1);
+            gathered[j].v[e] = mine[((sl < 2 ? a01 : a23) >> sh) & (kSlabWarpTile - 1)];
+            if (sl < 2) a01 += 1u << sh; else a23 += 1u << sh;
+          }
+      }
+    }
     uint32_t carry = identity_of<FN, DT>();                // running total of this warp's earlier rows
 #pragma unroll
     for (int j = 0; j < ROWS; ++j) {
@@ -504,7 +569,19 @@ __global__ void __launch_bounds__(scan_block<CL>()) k_scan(const __grid_constant
       const bool live = c < n;
       if (live) {
         const IX ix = index_at(row, c);
-        const auto v = eval<CL, sn.in[0]>(a, ix);
+        val_of<IX> v;
+        if constexpr (SLAB) {
+          if (merged) {
+            IxGv<IX> with;
+            static_cast<IX&>(with) = ix;
+            with.gv = gathered[j];
+            v = eval<CL, sn.in[0]>(a, with);
+          } else {
+            v = eval<CL, sn.in[0]>(a, ix);
+          }
+        } else {
+          v = eval<CL, sn.in[0]>(a, ix);
+        }
         if constexpr (VEC) {
 #pragma unroll
           for (int e = 0; e < 4; ++e) val[j][e] = v.v[e];
@@ -627,6 +704,11 @@ __global__ void __launch_bounds__(scan_block<CL>()) k_scan(const __grid_constant
       }
     }
   }
+}
+
+template <class CL, bool VEC>
+__global__ void __launch_bounds__(scan_block<CL>()) k_scan(const __grid_constant__ Args<CL::c.n> a, int tiles_per_row, int n_tiles) {
+  scan_tiles<CL, VEC, false>(a, tiles_per_row, n_tiles, SlabIn{});
 }
 
 }  // namespace dev

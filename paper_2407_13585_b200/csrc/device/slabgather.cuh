@@ -1,0 +1,180 @@
+// A scan whose operand gathers from an array that does not fit the L2 cache, run as slab passes.
+//
+// A random 4-byte read of an array much larger than L2 costs a whole DRAM access (about 89 bytes of
+// traffic on B200), and a cluster such as  out = scanl(+) (f (gather idx (g x)))  runs at the rate of
+// those accesses.  The same reads served from L2 run four times faster, so the gather is cut into
+// passes, each over a quarter (a slab) of the source, small enough to stay in L2 while it is being read:
+//
+//   k_slab_partition  walks the gather's index operand once.  Per warp tile of 512 elements it writes the
+//                     index values grouped by slab (a stable counting sort in shared memory) into the
+//                     scan's own output array, which serves as the staging area, the slab of every
+//                     element (2 bits, one word per lane) into `codes`, and the group sizes into `counts`.
+//   k_slab_gather     once per slab k: replaces the indices of group k, where they lie, by the gathered
+//                     values (the gather's source, with the members fused into it, evaluated at the index).
+//                     It streams a quarter of the staging area per pass and reads one slab of the source.
+//   k_scan_merge      the look-back scan of skeletons.cuh, which first puts a warp tile's gathered values back
+//                     into element order (the counting sort undone with the codes and the counts) and reads
+//                     the gather member as those values; everything after the gather is evaluated as usual.
+//
+// Gather semantics (Section 2: ys[j] = as[is[j]]) and results are unchanged, bit for bit.  A last warp tile
+// of fewer than 512 elements is left to the scan, which gathers for it directly.
+#pragma once
+#include "skeletons.cuh"
+
+namespace acc {
+namespace dev {
+
+constexpr int kSlabs = 4;
+constexpr int64_t kSlabMinSourceBytes = 96ll << 20;     // below this the source mostly stays in L2 anyway
+constexpr int64_t kSlabMaxSourceBytes = 320ll << 20;    // beyond this a quarter of it no longer fits
+constexpr int64_t kSlabMinElements = 1ll << 22;
+
+constexpr bool depends_on(const CCluster& c, int i, int g) {
+  if (i == g) return true;
+  const CNode& n = c.nodes[i];
+  if (!n.member) return false;
+  for (int k = 0; k < n.nin; ++k)
+    if (depends_on(c, n.in[k], g)) return true;
+  return false;
+}
+// Whether every path from i down to g runs through array operands of maps and zipWiths only (so that the
+// element index is the same all the way, and g's value at that index is all that is needed of it).
+constexpr bool index_preserving_to(const CCluster& c, int i, int g) {
+  if (i == g) return true;
+  const CNode& n = c.nodes[i];
+  if (!depends_on(c, i, g)) return true;
+  if (n.kind != ACC_MAP && n.kind != ACC_ZIPWITH) return false;
+  for (int k = 0; k < n.nin; ++k) {
+    if (!depends_on(c, n.in[k], g)) continue;
+    if (k >= n.narr || !index_preserving_to(c, n.in[k], g)) return false;
+  }
+  return true;
+}
+
+// depends_on with node `stop` taken as a leaf
+constexpr bool depends_on_avoiding(const CCluster& c, int i, int g, int stop) {
+  if (i == g) return true;
+  if (i == stop) return false;
+  const CNode& n = c.nodes[i];
+  if (!n.member) return false;
+  for (int k = 0; k < n.nin; ++k)
+    if (depends_on_avoiding(c, n.in[k], g, stop)) return true;
+  return false;
+}
+
+// One left-to-right scan of a rank-1 array as the only accumulating root, one gather (fused away) below its
+// operand on index-preserving paths, and no element-wise root that would need the gather outside the scan's pass.
+template <class CL> constexpr bool slab_gather_eligible() {
+  const int S = first_scan<CL>();
+  const int G = the_gather<CL>();
+  if (S < 0 || G < 0) return false;
+  const CCluster& c = CL::c;
+  if (c.nodes[S].kind != ACC_SCANL || c.nodes[S].rank != 1 || !c.nodes[S].manifest || c.nodes[G].manifest || c.nodes[G].rank != 1) return false;
+  for (int i = 0; i < c.n; ++i) {
+    const CNode& n = c.nodes[i];
+    if (i != S && (is_scan_root(n) || is_fold_root(n) || is_permute_root(n) || is_segfold_root(n))) return false;
+    if (is_store_root(n) && depends_on_avoiding(c, i, G, S)) return false;     // it would gather on its own, outside the passes
+  }
+  if (depends_on(c, G, S)) return false;
+  return depends_on(c, c.nodes[S].in[0], G) && index_preserving_to(c, c.nodes[S].in[0], G);
+}
+
+// slab of a source index: the source is cut into kSlabs nearly equal ranges (mul = floor(2^32 * kSlabs / elements))
+__device__ __forceinline__ uint32_t slab_of(uint32_t k, uint32_t mul) { return min(__umulhi(k, mul), (uint32_t)(kSlabs - 1)); }
+
+template <class CL>
+__global__ void __launch_bounds__(kBlock, 4) k_slab_partition(const __grid_constant__ Args<CL::c.n> a, uint32_t* __restrict__ codes,
+                                                               uint32_t* __restrict__ counts, int full_tiles, uint32_t mul) {
+  constexpr int G = the_gather<CL>();
+  constexpr int S = first_scan<CL>();
+  constexpr int KEY = CL::c.nodes[G].in[0];
+  constexpr int ROWS = kSlabWarpTile / 128;
+  __shared__ __align__(16) uint32_t stage[kBlock / 32][kSlabWarpTile];       // read 128 bits at a time
+  const int lane = threadIdx.x & 31;
+  const int stride = gridDim.x * (kBlock / 32);
+  uint32_t* staging = reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[S].ptr));
+  uint32_t* mine = stage[threadIdx.x >> 5];
+  for (int wt = blockIdx.x * (kBlock / 32) + ((int)threadIdx.x >> 5); wt < full_tiles; wt += stride) {
+    V4 key[ROWS];
+#pragma unroll
+    for (int j = 0; j < ROWS; ++j) key[j] = eval<CL, KEY>(a, Ix4{0, wt * kSlabWarpTile + (j * 32 + lane) * 4});
+    uint32_t code = 0, c01 = 0, c23 = 0;                           // slabs of this lane's 16 elements; how many in slabs 0 | 1, 2 | 3
+#pragma unroll
+    for (int j = 0; j < ROWS; ++j)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const uint32_t sl = slab_of(key[j].v[e], mul);
+        code |= sl << (2 * (4 * j + e));
+        if (sl < 2) c01 += 1u << (16 * (sl & 1)); else c23 += 1u << (16 * (sl & 1));
+      }
+    uint32_t i01 = c01, i23 = c23;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t u0 = __shfl_up_sync(0xFFFFFFFFu, i01, o), u1 = __shfl_up_sync(0xFFFFFFFFu, i23, o);
+      if (lane >= o) { i01 += u0; i23 += u1; }
+    }
+    const uint32_t T01 = __shfl_sync(0xFFFFFFFFu, i01, 31), T23 = __shfl_sync(0xFFFFFFFFu, i23, 31);
+    const uint32_t t0 = T01 & 0xFFFFu, t1 = T01 >> 16, t2 = T23 & 0xFFFFu;
+    uint32_t a01 = (i01 - c01) + (t0 << 16);                          // next position in the lists of slabs 0 | 1
+    uint32_t a23 = (i23 - c23) + (t0 + t1) + ((t0 + t1 + t2) << 16);  // ... of slabs 2 | 3
+    __syncwarp();
+#pragma unroll
+    for (int j = 0; j < ROWS; ++j)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const uint32_t sl = (code >> (2 * (4 * j + e))) & 3u;
+        const uint32_t sh = 16 * (sl & 1);
+        mine[((sl < 2 ? a01 : a23) >> sh) & (kSlabWarpTile - 1)] = key[j].v[e];
+        if (sl < 2) a01 += 1u << sh; else a23 += 1u << sh;
+      }
+    __syncwarp();
+#pragma unroll
+    for (int j = 0; j < ROWS; ++j) {
+      const int q = (j * 32 + lane) * 4;
+      *reinterpret_cast<uint4*>(staging + (size_t)wt * kSlabWarpTile + q) = *reinterpret_cast<const uint4*>(mine + q);
+    }
+    codes[(size_t)wt * 32 + lane] = code;
+    if (lane == 0) counts[wt] = t0 | (t1 << 10) | (t2 << 20);
+  }
+}
+
+template <class CL>
+__global__ void __launch_bounds__(kBlock) k_slab_gather(const __grid_constant__ Args<CL::c.n> a, const uint32_t* __restrict__ counts,
+                                                         int full_tiles, uint32_t slab) {
+  constexpr int G = the_gather<CL>();
+  constexpr int S = first_scan<CL>();
+  constexpr int SRC = CL::c.nodes[G].in[1];
+  constexpr int src_rank = CL::c.nodes[SRC].rank;
+  const int lane = threadIdx.x & 31;
+  const int stride = gridDim.x * (kBlock / 32);
+  uint32_t* staging = reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[S].ptr));
+  const uint32_t n_src = (uint32_t)(a.n[SRC].R * a.n[SRC].C);
+  for (int wt = blockIdx.x * (kBlock / 32) + ((int)threadIdx.x >> 5); wt < full_tiles; wt += stride) {
+    const uint32_t c = __ldg(counts + wt);
+    const uint32_t t0 = c & 1023u, t1 = (c >> 10) & 1023u, t2 = (c >> 20) & 1023u;
+    const uint32_t lo = slab == 0 ? 0u : slab == 1 ? t0 : slab == 2 ? t0 + t1 : t0 + t1 + t2;
+    const uint32_t len = slab == 0 ? t0 : slab == 1 ? t1 : slab == 2 ? t2 : (uint32_t)kSlabWarpTile - (t0 + t1 + t2);
+    uint32_t* p = staging + (size_t)wt * kSlabWarpTile + lo;
+    for (uint32_t q = lane; q < len; q += 128) {                   // four reads in flight per lane
+      uint32_t k[4], v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (q + 32 * u < len) k[u] = min(p[q + 32 * u], n_src - 1);   // (an index outside the source is the caller's error; it reads no foreign memory here)
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (q + 32 * u < len) v[u] = eval<CL, SRC>(a, gather1<src_rank>(k[u], a.n[SRC]));
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (q + 32 * u < len) p[q + 32 * u] = v[u];
+    }
+  }
+}
+
+template <class CL>
+__global__ void __launch_bounds__(scan_block<CL>()) k_scan_merge(const __grid_constant__ Args<CL::c.n> a, int tiles_per_row, int n_tiles,
+                                                                  const SlabIn slab) {
+  scan_tiles<CL, true, true>(a, tiles_per_row, n_tiles, slab);
+}
+
+}  // namespace dev
+}  // namespace acc

@@ -236,10 +236,11 @@ int run_schedule(Graph& g, Schedule& sch, void* workspace, size_t ws_bytes, cuda
     st.launch.status = reinterpret_cast<uint32_t*>(ws);
     st.launch.stream = stream;
     st.launch.spin_limit = g.spin_limit;
+    st.launch.extra_launches = 0;
     const int rc = st.kernel->launch(st.launch);
     if (rc != ACC_OK) return rc;
     if (!mark(marks, stream)) return set_error(ACC_ERR_CUDA, "recording an event failed: %s", cudaGetErrorString(cudaGetLastError()));
-    g.launches += st.kernel->passes;
+    g.launches += st.kernel->passes + st.launch.extra_launches;
     char item[48];
     snprintf(item, sizeof item, "%s%d:%d", g.schedule.empty() ? "" : " ", st.first_node, st.n_members);
     g.schedule += item;

@@ -19,6 +19,7 @@ struct ClusterLaunch {
   uint32_t* status = nullptr;
   uint32_t spin_limit = 1u << 22;
   cudaStream_t stream = nullptr;
+  mutable int extra_launches = 0;   // set by a launcher that took more launches than its entry's `passes` (data-dependent paths)
 };
 
 struct KernelEntry {

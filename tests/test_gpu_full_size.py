@@ -48,9 +48,40 @@ def test_config2_full():
 def test_config3_full():
     prog = W.config3(1 << 26)
     got, inputs, pi, g = run_full(prog, "enumerate")
-    assert pi == [-1, -1, 0, 0, 0, 0] and g.launch_count() == 1
+    # one cluster; its gather reads a 256 MB source, twice the L2, so it runs as slab passes: the indices are
+    # partitioned once, four launches gather a quarter of the source each, and the scan merges (six launches)
+    assert pi == [-1, -1, 0, 0, 0, 0] and g.launch_count() == 6
     ref = oracle_run(prog, {k: v.cpu().numpy() for k, v in inputs.items()})
     compare(prog, ref, got, "config3 full")
+
+
+def test_gather_scan_in_slab_passes_ragged():
+    """The slab passes on shapes of their own: a 128 MB source, fewer indices than source elements, a last warp tile
+    of 260 elements (left to the scan's direct gather), under both clusterings that keep the gather with the scan."""
+    import torch
+    from workloads import Node, Program
+    from paper_2407_13585_b200 import binding as B
+    n_src, n = 1 << 25, (1 << 22) + (1 << 20) + 260
+    nodes = [Node("input", "i32", (n_src,), name="x"), Node("input", "i32", (n,), name="idx"),
+             Node("map", "i32", (n_src,), (0,), 1, fn="hash_mul_xorshift", iparam=(2654435761, 13), name="g"),
+             Node("gather", "i32", (n,), (1, 2), 2, name="h"),
+             Node("map", "i32", (n,), (3,), 1, fn="and_mask", iparam=(0xFFFF,), name="o"),
+             Node("scanl", "i32", (n,), (4,), 1, fn="add", name="out")]
+    prog = Program("gather_scan_ragged", nodes, [5])
+    inputs = {0: W.uniform_int(0, 0, n_src, 1 << 31, device="cuda"), 1: W.uniform_int(0, 1, n, n_src, device="cuda")}
+    ref = oracle_run(prog, {k: v.cpu().numpy() for k, v in inputs.items()})
+    for pi, launches in (([-1, -1, 0, 0, 0, 0], 6), ([-1, -1, 0, 1, 1, 1], 7)):
+        g = B.Graph(prog.nodes, prog.outputs)
+        g.set_partition(pi)
+        for i, t in inputs.items():
+            g.bind(i, t)
+        out = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+        g.bind(5, out)
+        g.run(B.FUSED)
+        g.run(B.FUSED)
+        assert g.launch_count() == launches, (pi, g.launch_count())
+        got = {5: out.cpu().numpy().view(np.uint32)}
+        compare(prog, ref, got, "gather + scan in slab passes, pi=%s" % pi)
 
 
 def test_config5_full():
