@@ -549,7 +549,8 @@ def run_ours(args):
             med = statistics.median(ms)
             row = {"clustering": w.pi, "planner": w.plan_mode, "clusters_split_for_lack_of_a_kernel": w.refined, "launches_fused": n_f,
                    "ms_fused": med, "ms_best": min(ms), "compulsory_bytes": w.bytes, "effective_gbs": w.bytes / med / 1e6,
-                   "frac_of_copy_peak": w.bytes / med / 1e6 / peak, "clustering_traffic_bytes": w.g.partition_cost(w.pi, "bytes")}
+                   "frac_of_copy_peak": w.bytes / med / 1e6 / peak, "clustering_traffic_bytes": w.g.partition_cost(w.pi, "bytes"),
+                   "gelem_s": w.elements / med / 1e6}      # (the largest array of the program, stored or not, per second)
             if check and args.cpu_baseline == "full":
                 row["parity"] = oracle_parity(w)
             for _ in range(3):

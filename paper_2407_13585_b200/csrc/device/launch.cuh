@@ -177,6 +177,16 @@ struct Launcher {
     return words * 4;
   }
 
+  // Counters, tickets, tile states and accumulators start from zero; what a kernel writes before it reads
+  // (partial sums per tile, the codes and group sizes of the slab passes) need not be cleared, and lies last.
+  static int64_t zeroed_bytes(const ClusterLaunch& L) {
+    int R, C;
+    if (!domain(L, R, C)) return 0;
+    if (use_tiles(L, R, C)) return dev::tile_partials_off((R + dev::kTile - 1) / dev::kTile) * 4;
+    if (kHasScan && slab_shapes_ok(L, R, C)) return ((16 + (int64_t)R * ((C + kScanTile - 1) / kScanTile) * 8) + 15) & ~int64_t(15);
+    return scratch_bytes(L);
+  }
+
   static void fill(const ClusterLaunch& L, dev::Args<N>& a, int R, int C) {
     for (int i = 0; i < N; ++i) a.n[i] = L.nodes[i];
     a.R = R;
@@ -543,6 +553,10 @@ struct Passes {
     if constexpr (plan.n <= 1) return Launcher<CL>::scratch_bytes(L);
     else return scratch_from<0>(L);
   }
+  static int64_t zeroed_bytes(const ClusterLaunch& L) {
+    if constexpr (plan.n <= 1) return Launcher<CL>::zeroed_bytes(L);
+    else return scratch_from<0>(L);                   // the passes' regions follow one another: all of it
+  }
 
   template <int P>
   static int launch_from(ClusterLaunch& L) {
@@ -572,7 +586,7 @@ struct Registrar {
   explicit Registrar(const char* name) {
     // (a cluster of segmented folds is a walk over the elements and a small second launch for the segments that
     // cross its blocks)
-    register_kernel(KernelEntry{signature(CL::c), name, &Passes<CL>::scratch_bytes, &Passes<CL>::launch,
+    register_kernel(KernelEntry{signature(CL::c), name, &Passes<CL>::scratch_bytes, &Passes<CL>::zeroed_bytes, &Passes<CL>::launch,
                                 Passes<CL>::plan.n > 1 ? Passes<CL>::plan.n : (dev::count_if<CL>(dev::is_segfold_root) > 0 ? 2 : 1)});
   }
 };

@@ -186,12 +186,22 @@ int build_schedule(Graph& g, int executor, Schedule& sch) {
     for (int li = 0; li < st.cc.n; ++li) st.launch.nodes[li] = node_arg(g.nodes[st.cc.source[li]], nullptr);
     const int64_t sb = st.kernel->scratch_bytes(st.launch);
     if (sb < 0) return set_error((int)sb, "cluster at node %d: no scratch layout", st.first_node);
+    const int64_t zb = st.kernel->zeroed_bytes(st.launch);
     st.scratch_off = ctrl;
     st.scratch_bytes = (size_t)sb;
+    st.zero_bytes = (size_t)std::min<int64_t>(std::max<int64_t>(zb, 0), sb);
     ctrl += align_up((size_t)sb, 256);
     sch.steps.push_back(st);
   }
   sch.ctrl_bytes = ctrl;
+  sch.to_clear.clear();
+  sch.to_clear.emplace_back(0, 256);                       // the status slot
+  for (const ClusterStep& st : sch.steps) {
+    if (st.zero_bytes == 0) continue;
+    auto& last = sch.to_clear.back();
+    if (last.first + align_up(last.second, 256) == st.scratch_off) last.second = st.scratch_off - last.first + st.zero_bytes;   // one piece
+    else sch.to_clear.emplace_back(st.scratch_off, st.zero_bytes);
+  }
   sch.total_bytes = ctrl + sch.array_bytes;
   sch.manifest = man;
   sch.pi = pi;
@@ -218,8 +228,9 @@ int run_schedule(Graph& g, Schedule& sch, void* workspace, size_t ws_bytes, cuda
   if (reinterpret_cast<uintptr_t>(workspace) & 255) return set_error(ACC_ERR_WORKSPACE, "workspace is not 256-byte aligned");
   if (ws_bytes < sch.total_bytes) return set_error(ACC_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", ws_bytes, sch.total_bytes);
   char* ws = static_cast<char*>(workspace);
-  if (cudaMemsetAsync(ws, 0, sch.ctrl_bytes, stream) != cudaSuccess)
-    return set_error(ACC_ERR_CUDA, "clearing the control region failed: %s", cudaGetErrorString(cudaGetLastError()));
+  for (const auto& piece : sch.to_clear)
+    if (cudaMemsetAsync(ws + piece.first, 0, piece.second, stream) != cudaSuccess)
+      return set_error(ACC_ERR_CUDA, "clearing the control region failed: %s", cudaGetErrorString(cudaGetLastError()));
   g.launches = 0;
   g.schedule.clear();
   if (!mark(marks, stream)) return set_error(ACC_ERR_CUDA, "recording an event failed: %s", cudaGetErrorString(cudaGetLastError()));

@@ -3,6 +3,7 @@
 #pragma once
 #include <cuda_runtime.h>
 
+#include <utility>
 #include <vector>
 
 #include "cluster.h"
@@ -16,7 +17,7 @@ struct ClusterStep {
   CCluster cc{};
   const KernelEntry* kernel = nullptr;
   ClusterLaunch launch;
-  size_t scratch_off = 0, scratch_bytes = 0;
+  size_t scratch_off = 0, scratch_bytes = 0, zero_bytes = 0;
 };
 
 struct Schedule {
@@ -25,6 +26,7 @@ struct Schedule {
   std::vector<uint8_t> manifest;
   std::vector<int32_t> pi;
   size_t ctrl_bytes = 0, array_bytes = 0, total_bytes = 0;
+  std::vector<std::pair<size_t, size_t>> to_clear;   // (offset, bytes) of what a run zeroes first: the status slot and the zeroed part of every scratch
 };
 
 int build_schedule(Graph& g, int executor, Schedule& sch);

@@ -15,7 +15,7 @@ namespace acc {
 struct ClusterLaunch {
   dev::NodeArg nodes[kMaxCluster];
   int n = 0;
-  uint32_t* scratch = nullptr;   // zeroed region of scratch_bytes() bytes, 16-byte aligned
+  uint32_t* scratch = nullptr;   // scratch_bytes() bytes, 16-byte aligned, the first zeroed_bytes() of them zero
   uint32_t* status = nullptr;
   uint32_t spin_limit = 1u << 22;
   cudaStream_t stream = nullptr;
@@ -26,6 +26,7 @@ struct KernelEntry {
   std::string sig;
   const char* name;
   int64_t (*scratch_bytes)(const ClusterLaunch&);   // >= 0, or a negative acc_status
+  int64_t (*zeroed_bytes)(const ClusterLaunch&);    // how much of the scratch, from its start, must be zero at launch
   int (*launch)(const ClusterLaunch&);               // acc_status; asynchronous
   int passes = 1;                                    // launches per run (see Passes in device/launch.cuh)
 };
