@@ -77,6 +77,12 @@ template <class CL> constexpr int domain_rank() {
   return 1;
 }
 
+template <class CL> constexpr bool has_reversal() {
+  for (int i = 0; i < CL::c.n; ++i)
+    if (CL::c.nodes[i].member && CL::c.nodes[i].kind == ACC_BACKPERMUTE && CL::c.nodes[i].idxfn == ACC_IDX_REVERSE) return true;
+  return false;
+}
+
 // Scratch layout of k_stream (32-bit words): [0] ticket, [4 ..) one partial per block per
 // scalar fold, then (8-byte aligned) one fp64 accumulator per bin per fp32 '+' permute.
 __host__ __device__ inline uint32_t stream_partials_off() { return 4; }
@@ -141,14 +147,24 @@ __global__ void __launch_bounds__(kBlock) k_stream(const __grid_constant__ Args<
   // same speed, 0.103 ms: the kernel is held by the load/store unit, not by L2.)
   const uint32_t per_row = (uint32_t)a.C / W;
   const uint32_t tiles_x = (per_row + 31) / 32;
-  const uint32_t trips = DR <= 1 ? (per_row + kBlock - 1) / kBlock
+  // A rank-1 cluster with a reversal reads arrays at i and at n-1-i.  Walked in mirrored pairs (a thread takes
+  // chunk q and then chunk per_row-1-q) both positions need the same two chunks of such an array, and the second
+  // evaluation finds them in L1: an array longer than the L2 crosses DRAM once instead of twice.
+  constexpr bool MIRROR = DR <= 1 && has_reversal<CL>();
+  const uint32_t half = (per_row + 1) / 2;
+  const uint32_t trips = DR <= 1 ? ((MIRROR ? half : per_row) + kBlock - 1) / kBlock
                                  : tiles_x * (((uint32_t)a.R + kStreamTileRows - 1) / kStreamTileRows);
   for (uint32_t t = blockIdx.x; t < trips; t += gridDim.x) {
+   for (int side = 0; side < (MIRROR ? 2 : 1); ++side) {
     IX ix;
     bool live;
     if constexpr (DR <= 1) {
-      const uint32_t q = t * kBlock + threadIdx.x;
-      live = q < per_row;
+      uint32_t q = t * kBlock + threadIdx.x;
+      live = q < (MIRROR ? half : per_row);
+      if (MIRROR && side == 1) {
+        live = live && per_row - 1 - q != q;               // the middle chunk of an odd count has no partner
+        q = per_row - 1 - q;
+      }
       ix.r = 0;
       ix.c = (int)(q * W);
     } else {
@@ -186,6 +202,7 @@ __global__ void __launch_bounds__(kBlock) k_stream(const __grid_constant__ Args<
         }
       }
     });
+   }
   }
 
   if constexpr (NF > 0 || NP64 > 0) {
