@@ -203,14 +203,16 @@ k_hist(const __grid_constant__ Args<CL::c.n> a, const HistPlan plan, int* overfl
   const bool fast_ok = group == 1 && S >= 0;
   const uint32_t bins_addr = (uint32_t)__cvta_generic_to_shared(bins_smem);
   uint32_t it = 0;
-  for (uint32_t q0 = team * kHistBlock + threadIdx.x; q0 < total; q0 += stride * U, it += U) {
+  // FULL: every chunk of the trip and of the trips prefetched from it lies inside the array (no test per chunk)
+  auto trip = [&](auto full_c, uint32_t q0) {
+    constexpr bool FULL = decltype(full_c)::value;
     if constexpr (VEC) {
       // ask L2 for what the trip after next will read: there are too few registers to keep
       // enough loads in flight to cover DRAM latency, so the loads should find their lines in L2
 #pragma unroll
       for (int u = 0; u < U; ++u) {
         const uint32_t q = q0 + (kHistAhead * U + u) * stride;
-        if (q < total) {
+        if (FULL || q < total) {
           const IX ix = index_of(q);
           eval<CL, pn.in[1]>(a, IxPF4{ix.r, ix.c});
           eval<CL, pn.in[2]>(a, IxPF4{ix.r, ix.c});
@@ -223,7 +225,7 @@ k_hist(const __grid_constant__ Args<CL::c.n> a, const HistPlan plan, int* overfl
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const uint32_t q = q0 + u * stride;
-      live[u] = q < total;
+      live[u] = FULL || q < total;
       if (live[u]) {
         const IX ix = index_of(q);
         key[u] = eval<CL, pn.in[1]>(a, ix);
@@ -232,7 +234,7 @@ k_hist(const __grid_constant__ Args<CL::c.n> a, const HistPlan plan, int* overfl
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      if (!live[u]) continue;
+      if (!FULL && !live[u]) continue;
       if (group == 1 || (it + u) % group == rank) {            // this CTA's turn for the element-wise side
         const IX ix = index_of(q0 + u * stride);
         static_for<0, N>([&](auto ic) {
@@ -297,6 +299,13 @@ k_hist(const __grid_constant__ Args<CL::c.n> a, const HistPlan plan, int* overfl
         scatter_one(key[u], val[u]);
       }
     }
+  };
+  {
+    const uint64_t step = (uint64_t)stride * U;
+    const uint64_t reach = (uint64_t)(kHistAhead * U + U - 1) * stride;     // the furthest chunk a trip touches, from its first
+    uint64_t q0 = (uint64_t)team * kHistBlock + threadIdx.x;
+    for (; q0 + reach < total; q0 += step, it += U) trip(std::true_type{}, (uint32_t)q0);
+    for (; q0 < total; q0 += step, it += U) trip(std::false_type{}, (uint32_t)q0);
   }
 
   __syncthreads();
