@@ -355,8 +355,8 @@ struct Launcher {
         constexpr int NFOLD = dev::count_if<CL>(dev::is_segfold_root);
         const int grid = seg_grid(L);
         const int per_block = dev::kSegTilesPerBlock;
-        const size_t smem = (size_t)NFOLD * dev::kSegTile * 4;
         const bool v4 = seg_vec_ok(L);
+        const size_t smem = v4 ? 0 : (size_t)NFOLD * dev::kSegTile * 4;    // operands are staged only where rows are not 128-bit friendly
         auto kern = v4 ? dev::k_segfold<CL, true> : dev::k_segfold<CL, false>;
         static int granted[2][64];
         if (smem > 48 * 1024 && !opt_in_shared_memory(kern, smem, granted[v4 ? 1 : 0]))

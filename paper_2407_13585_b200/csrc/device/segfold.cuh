@@ -6,10 +6,14 @@
 // short ones (skewed lengths) cost what their elements cost:
 //
 //  * the source range is cut into tiles of kSegTile elements; a block owns a contiguous run of
-//    tiles and walks it in order.  It evaluates a tile's operands with coalesced (128-bit where
-//    the arrays allow) reads into shared memory, one array per fold;
-//  * the pieces of segments inside the tile are reduced from shared memory: a thread per piece
-//    up to kSegShort elements, a warp per piece up to kSegMedium, the whole block beyond;
+//    tiles and walks it in order.  A run of tiles that lies inside one segment is streamed;
+//  * any other tile, where the arrays have 128-bit rows: its operands stay in registers, a bit per
+//    element marks where segments begin, and a segmented scan (inside a chunk, across a warp by
+//    shuffles, across the tile through 32 partial values) gives every element the sum of its
+//    segment so far; the elements that end a segment write it.  Uniform work whatever the lengths;
+//  * without 128-bit rows the tile's operands are staged in shared memory and the pieces of
+//    segments are reduced from there: a thread per piece up to kSegShort elements, a warp per
+//    piece up to kSegMedium, the whole block beyond;
 //  * a piece that is a whole segment is written at once.  A segment that crosses tiles is carried
 //    by the block from tile to tile (a compensated running value in one thread); one that crosses
 //    blocks leaves a record per block (the part after its start: `tail`; a part that continues
@@ -89,6 +93,10 @@ __global__ void __launch_bounds__(kBlock, kSegResident) k_segfold(const __grid_c
   __shared__ int off_win[kSegWindow + 1];                        // offsets of segments win_base .. win_base + kSegWindow
   __shared__ int long_seg[kSegListCap], long_lo[kSegListCap], long_hi[kSegListCap], long_kind[kSegListCap];
   __shared__ int big_seg[kSegBigCap], big_lo[kSegBigCap], big_hi[kSegBigCap], big_kind[kSegBigCap];
+  __shared__ uint32_t seg_bits[VEC ? kSegTile / 32 + 2 : 1];      // bit p: element p of the tile begins a segment
+  __shared__ int seg_before[VEC ? kSegTile / 32 : 1];            // starts before each 32-element word
+  __shared__ uint32_t seg_unit_flag[VEC ? 32 : 1], seg_unit_val[VEC ? NF : 1][VEC ? 32 : 1];
+  __shared__ int tile_open;
   __shared__ int n_long, n_big, next_s, first_open, have_first, have_last, last_seg;
   __shared__ uint32_t first_val[NF], last_val[NF];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -246,6 +254,145 @@ __global__ void __launch_bounds__(kBlock, kSegResident) k_segfold(const __grid_c
         next_s = hi_c > run_hi ? s_cur : s_cur + 1;
       }
       t += run - 1;
+    } else if constexpr (VEC) {
+      // ---- a tile with pieces of several segments, 128-bit rows: a segmented scan over the tile in registers ----
+      // Thread t holds chunks (j * kBlock + t) * 4, j = 0..3, of the tile; in the order (j, warp, lane, element) the
+      // values form one sequence.  `bits` marks the elements that begin a segment.  Every element gets the sum of
+      // its segment up to itself: inside a chunk, across the lanes of a warp (a shuffle scan that stops at lanes
+      // holding a start), across the 32 (row, warp) units through shared memory; elements that end a segment
+      // (the next one begins one, or the tile ends) then hold that segment's sum over the tile and write it.
+      constexpr int ROWS = kSegTile / (4 * kBlock);
+      static_assert(ROWS * WARPS == 32, "the (row, warp) units of a tile are scanned by the lanes of one warp");
+      uint32_t xv[N][ROWS][4];
+      static_for<0, N>([&](auto ic) {
+        constexpr int i = decltype(ic)::value;
+        constexpr CNode nd = CL::c.nodes[i];
+        if constexpr (is_segfold_root(nd)) {
+#pragma unroll
+          for (int j = 0; j < ROWS; ++j) {
+            const int c = tile_lo + (j * kBlock + (int)threadIdx.x) * 4;
+            V4 v = V4{{identity_of<nd.fn, nd.dtype>(), identity_of<nd.fn, nd.dtype>(), identity_of<nd.fn, nd.dtype>(), identity_of<nd.fn, nd.dtype>()}};
+            if (c < tile_hi) v = eval<CL, nd.in[0]>(a, Ix4{0, c});
+#pragma unroll
+            for (int e = 0; e < 4; ++e) xv[i][j][e] = c + e < tile_hi ? v.v[e] : identity_of<nd.fn, nd.dtype>();
+          }
+        }
+      });
+      for (int k = threadIdx.x; k < kSegTile / 32 + 2; k += kBlock) seg_bits[k] = 0;
+      if (threadIdx.x == 0) tile_open = 0;
+      __syncthreads();
+      for (int base = s_cur;; base += kBlock) {                  // a thread per segment: where it begins, if that is in the tile
+        if (base + kBlock > win_base + kSegWindow) {             // uniform: the window moves up to `base`
+          __syncthreads();
+          win_base = base;
+          for (int k = threadIdx.x; k <= kSegWindow; k += kBlock) off_win[k] = base + k <= S ? __ldg(off + base + k) : 0x7FFFFFFF;
+          __syncthreads();
+        }
+        const int s = base + (int)threadIdx.x;
+        const int lo_s = off_win[s - win_base], hi_s = off_win[s - win_base + 1];
+        const bool beyond = s >= S || lo_s >= tile_hi;
+        if (!beyond) {
+          if (lo_s >= lo0) atomicOr(&seg_bits[(lo_s - tile_lo) >> 5], 1u << ((lo_s - tile_lo) & 31));
+          if (hi_s >= tile_hi) { next_s = hi_s > tile_hi ? s : s + 1; tile_open = hi_s > tile_hi ? 1 : 0; }
+        }
+        if (__syncthreads_or(beyond)) break;
+      }
+      if (warp == 0) {                                           // starts before each 32-element word of the tile
+        int cnt[4], sum = 0;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) { cnt[k] = sum; sum += __popc(seg_bits[4 * lane + k]); }
+        int incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int u = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+          if (lane >= o) incl += u;
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) seg_before[4 * lane + k] = incl - sum + cnt[k];
+      }
+      __syncthreads();
+      const bool cont = lo_c < lo0, open = tile_open != 0;
+      const int lo_rel = lo0 - tile_lo, hi_rel = tile_hi - tile_lo;
+      uint32_t cin[N][ROWS];                                     // what precedes the chunk in its run, within the warp's row
+      uint32_t marks[ROWS];                                      // bits 0-3: starts in the chunk, 4: start right after it, 5: no start in earlier lanes
+      int before[ROWS];                                          // starts before the chunk, in the tile
+#pragma unroll
+      for (int j = 0; j < ROWS; ++j) {
+        const int p = (j * kBlock + (int)threadIdx.x) * 4, w = p >> 5, sh = p & 31;
+        const uint32_t word = seg_bits[w];
+        const uint32_t b5 = __funnelshift_r(word, seg_bits[w + 1], sh) & 31u, b = b5 & 15u;
+        before[j] = seg_before[w] + __popc(word & ((1u << sh) - 1u));
+        const unsigned H = __ballot_sync(0xFFFFFFFFu, b != 0);
+        const unsigned upto = H & (0xFFFFFFFFu >> (31 - lane));  // lanes up to this one that hold a start
+        const int lower = upto ? 31 - __clz(upto) : 0;            // the run this chunk's end belongs to begins in that lane
+        marks[j] = b5 | ((H & ((1u << lane) - 1u)) == 0 ? 32u : 0u);
+        static_for<0, N>([&](auto ic) {
+          constexpr int i = decltype(ic)::value;
+          constexpr CNode nd = CL::c.nodes[i];
+          if constexpr (is_segfold_root(nd)) {
+#pragma unroll
+            for (int e = 1; e < 4; ++e)
+              if (!((b >> e) & 1u)) xv[i][j][e] = combine<nd.fn, nd.dtype>(xv[i][j][e - 1], xv[i][j][e]);
+            uint32_t run = xv[i][j][3];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+              const uint32_t u = __shfl_up_sync(0xFFFFFFFFu, run, o);
+              if (lane - o >= lower) run = combine<nd.fn, nd.dtype>(u, run);
+            }
+            const uint32_t prev = __shfl_up_sync(0xFFFFFFFFu, run, 1);
+            cin[i][j] = lane == 0 ? identity_of<nd.fn, nd.dtype>() : prev;
+            if (lane == 31) seg_unit_val[fold_slot_of(i)][j * WARPS + warp] = run;
+          }
+        });
+        if (lane == 31) seg_unit_flag[j * WARPS + warp] = H != 0 ? 1u : 0u;
+      }
+      __syncthreads();
+      // the 32 (row, warp) units in sequence: what runs into each of them from the units before
+      const unsigned UH = __ballot_sync(0xFFFFFFFFu, seg_unit_flag[lane] != 0);
+      const unsigned uupto = UH & (0xFFFFFFFFu >> (31 - lane));
+      const int ulower = uupto ? 31 - __clz(uupto) : 0;
+#pragma unroll
+      for (int j = 0; j < ROWS; ++j) before[j] -= cont ? 0 : 1;  // now: the chunk's first element lies in segment s_cur + before (+ starts up to it)
+      static_for<0, N>([&](auto ic) {
+        constexpr int i = decltype(ic)::value;
+        constexpr CNode nd = CL::c.nodes[i];
+        if constexpr (is_segfold_root(nd)) {
+          uint32_t run = seg_unit_val[fold_slot_of(i)][lane];
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t u = __shfl_up_sync(0xFFFFFFFFu, run, o);
+            if (lane - o >= ulower) run = combine<nd.fn, nd.dtype>(u, run);
+          }
+#pragma unroll
+          for (int j = 0; j < ROWS; ++j) {
+            const int unit = j * WARPS + warp;
+            const uint32_t into = __shfl_sync(0xFFFFFFFFu, run, max(unit - 1, 0));
+            if ((marks[j] & 32u) && unit > 0) cin[i][j] = combine<nd.fn, nd.dtype>(into, cin[i][j]);
+          }
+        }
+      });
+#pragma unroll
+      for (int j = 0; j < ROWS; ++j) {
+        const int p = (j * kBlock + (int)threadIdx.x) * 4;
+        const uint32_t b = marks[j] & 15u;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int pos = p + e;
+          const bool ends = pos >= lo_rel && pos < hi_rel && (pos == hi_rel - 1 || ((marks[j] >> (e + 1)) & 1u));
+          if (ends) {
+            const bool led = (b & ((2u << e) - 1u)) == 0;          // no start in the chunk up to here: the run comes in from before
+            const int seg = s_cur + before[j] + __popc(b & ((2u << e) - 1u));
+            uint32_t v[N];
+            static_for<0, N>([&](auto ic) {
+              constexpr int i = decltype(ic)::value;
+              constexpr CNode nd = CL::c.nodes[i];
+              if constexpr (is_segfold_root(nd)) v[i] = led ? combine<nd.fn, nd.dtype>(cin[i][j], xv[i][j][e]) : xv[i][j][e];
+            });
+            if ((uint32_t)seg < (uint32_t)S)
+              store_piece(seg, ((seg == s_cur && cont) ? 1 : 0) | ((pos == hi_rel - 1 && open) ? 2 : 0), v);
+          }
+        }
+      }
     } else {
     // stage the operands of the tile
     static_for<0, N>([&](auto ic) {
