@@ -30,6 +30,22 @@ inline bool opt_in_shared_memory(K kern, size_t smem, int* granted) {
   return true;
 }
 
+// Blocks of `kern` (no dynamic shared memory) that are resident at once on the current device, 0 if the device
+// cannot launch a grid cooperatively; asked of the driver once per kernel and device (`fit_on`: 64 zeroed words).
+inline int resident_grid(const void* kern, int block, int* fit_on) {
+  int device = 0;
+  if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) { cudaGetLastError(); return 0; }
+  if (fit_on[device] == 0) {
+    int fit = 0;
+    if (!cooperative_launch_ok() || cudaOccupancyMaxActiveBlocksPerMultiprocessor(&fit, kern, block, 0) != cudaSuccess) {
+      cudaGetLastError();
+      fit = 0;
+    }
+    fit_on[device] = fit + 1;
+  }
+  return (fit_on[device] - 1) * sm_count();
+}
+
 template <class CL>
 struct Launcher {
   static constexpr int N = CL::c.n;
@@ -395,15 +411,36 @@ struct Launcher {
           const int ggrid = (int)std::min<int64_t>((full + warps - 1) / warps, (int64_t)sm_count() * 8);
           dev::k_slab_partition<CL><<<pgrid, dev::kBlock, 0, L.stream>>>(a, codes, counts, full, mul);
           for (int k = 0; k < dev::kSlabs; ++k) dev::k_slab_gather<CL><<<ggrid, dev::kBlock, 0, L.stream>>>(a, counts, full, (uint32_t)k);
-          dev::k_scan_merge<CL><<<grid, kScanBlock, 0, L.stream>>>(a, per_row, (int)tiles, dev::SlabIn{codes, counts, full});
+          {
+            dev::SlabIn slab{codes, counts, full};
+            int per_row_arg = per_row, tiles_arg = (int)tiles;
+            void* params[] = {&a, &per_row_arg, &tiles_arg, &slab};
+            static int fit_on[64];
+            const int resident = resident_grid(reinterpret_cast<const void*>(dev::k_scan_merge<CL, true>), kScanBlock, fit_on);
+            if (resident > 0)
+              cudaLaunchCooperativeKernel(reinterpret_cast<void*>(dev::k_scan_merge<CL, true>), dim3((unsigned)std::min<int64_t>(tiles, resident)),
+                                          dim3(kScanBlock), params, 0, L.stream);
+            else
+              dev::k_scan_merge<CL><<<grid, kScanBlock, 0, L.stream>>>(a, per_row, (int)tiles, slab);
+          }
           L.extra_launches = 1 + dev::kSlabs;
           const cudaError_t e = cudaGetLastError();
           if (e != cudaSuccess) return set_error(ACC_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
           return ACC_OK;
         }
       }
-      if (vec) dev::k_scan<CL, true><<<grid, kScanBlock, 0, L.stream>>>(a, per_row, (int)tiles);
-      else dev::k_scan<CL, false><<<grid, kScanBlock, 0, L.stream>>>(a, per_row, (int)tiles);
+      {
+        // all blocks resident at once where the device can promise it (then tiles need no ticket), else ticketed tiles
+        int per_row_arg = per_row, tiles_arg = (int)tiles;
+        void* params[] = {&a, &per_row_arg, &tiles_arg};
+        static int fit_on[2][64];
+        const void* kern = vec ? reinterpret_cast<const void*>(dev::k_scan<CL, true, true>) : reinterpret_cast<const void*>(dev::k_scan<CL, false, true>);
+        const int resident = resident_grid(kern, kScanBlock, fit_on[vec ? 1 : 0]);
+        if (resident > 0)
+          cudaLaunchCooperativeKernel(const_cast<void*>(kern), dim3((unsigned)std::min<int64_t>(tiles, resident)), dim3(kScanBlock), params, 0, L.stream);
+        else if (vec) dev::k_scan<CL, true><<<grid, kScanBlock, 0, L.stream>>>(a, per_row, (int)tiles);
+        else dev::k_scan<CL, false><<<grid, kScanBlock, 0, L.stream>>>(a, per_row, (int)tiles);
+      }
     } else if constexpr (kHasRowFold) {
       if (R == 0) return ACC_OK;
       const int grid = std::min(R, sm_count() * 16);

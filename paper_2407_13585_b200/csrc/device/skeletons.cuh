@@ -498,7 +498,12 @@ constexpr bool needs_scan(const CCluster& c, int i, int s) {
 // Rows of a rank-2 array are scanned independently: a row is cut into tiles of its own, the
 // look-back of a tile stops at the first tile of its row.  A right-to-left scan walks its row
 // from the far end: position p of the walk is element C-1-p of the row.
-template <class CL, bool VEC, bool SLAB>
+// STATIC: block b walks tiles b, b + G, b + 2G, ... of a grid of G blocks that are all resident at once (a
+// cooperative launch): no ticket, whose atomic every warp of the block would otherwise wait for at the top of every
+// tile (measured on a streaming scan of 2^26 floats: 28 barrier-stall cycles per issued instruction, 19 % of the
+// issue slots used).  A tile's predecessors belong to the blocks before this one in the same round, or to an
+// earlier round, so they are running or done.  Without that guarantee the tiles are claimed from a ticket.
+template <class CL, bool VEC, bool SLAB, bool STATIC = false>
 __device__ __forceinline__ void scan_tiles(const Args<CL::c.n>& a, int tiles_per_row, int n_tiles, const SlabIn& slab) {
   constexpr int N = CL::c.n;
   constexpr int W = VEC ? 4 : 1;
@@ -528,11 +533,18 @@ __device__ __forceinline__ void scan_tiles(const Args<CL::c.n>& a, int tiles_per
     return ix;
   };
 
-  for (;;) {
-    __syncthreads();
-    if (threadIdx.x == 0) tile_id = (int)atomicAdd(a.scratch, 1u);
-    __syncthreads();
-    const int tile = tile_id;
+  for (int round = 0;; ++round) {
+    int tile;
+    if constexpr (STATIC) {
+      // (no barrier here: what a round shares through shared memory is read before its second barrier or right
+      // after it, and written again only behind the next round's first barrier)
+      tile = (int)blockIdx.x + round * (int)gridDim.x;
+    } else {
+      __syncthreads();
+      if (threadIdx.x == 0) tile_id = (int)atomicAdd(a.scratch, 1u);
+      __syncthreads();
+      tile = tile_id;
+    }
     if (tile >= n_tiles) return;
     const int row = tile / tiles_per_row, in_row = tile - row * tiles_per_row;
     const int warp_base = in_row * TILE + warp * (TILE / (BLOCK / 32));
@@ -723,9 +735,9 @@ __device__ __forceinline__ void scan_tiles(const Args<CL::c.n>& a, int tiles_per
   }
 }
 
-template <class CL, bool VEC>
+template <class CL, bool VEC, bool STATIC = false>
 __global__ void __launch_bounds__(scan_block<CL>()) k_scan(const __grid_constant__ Args<CL::c.n> a, int tiles_per_row, int n_tiles) {
-  scan_tiles<CL, VEC, false>(a, tiles_per_row, n_tiles, SlabIn{});
+  scan_tiles<CL, VEC, false, STATIC>(a, tiles_per_row, n_tiles, SlabIn{});
 }
 
 }  // namespace dev

@@ -171,10 +171,10 @@ __global__ void __launch_bounds__(kBlock) k_slab_gather(const __grid_constant__ 
 }
 
 // (five blocks per SM: the merge is issue bound, and a quarter more warps pay for a few spilled words)
-template <class CL>
+template <class CL, bool STATIC = false>
 __global__ void __launch_bounds__(scan_block<CL>(), 5) k_scan_merge(const __grid_constant__ Args<CL::c.n> a, int tiles_per_row, int n_tiles,
                                                                   const SlabIn slab) {
-  scan_tiles<CL, true, true>(a, tiles_per_row, n_tiles, slab);
+  scan_tiles<CL, true, true, STATIC>(a, tiles_per_row, n_tiles, slab);
 }
 
 }  // namespace dev
