@@ -416,10 +416,10 @@ struct Launcher {
             int per_row_arg = per_row, tiles_arg = (int)tiles;
             void* params[] = {&a, &per_row_arg, &tiles_arg, &slab};
             static int fit_on[64];
-            const int resident = resident_grid(reinterpret_cast<const void*>(dev::k_scan_merge<CL, true>), kScanBlock, fit_on);
+            const int resident = resident_grid(reinterpret_cast<const void*>(dev::k_scan_merge_pipelined<CL>), kScanBlock + 32, fit_on);
             if (resident > 0)
-              cudaLaunchCooperativeKernel(reinterpret_cast<void*>(dev::k_scan_merge<CL, true>), dim3((unsigned)std::min<int64_t>(tiles, resident)),
-                                          dim3(kScanBlock), params, 0, L.stream);
+              cudaLaunchCooperativeKernel(reinterpret_cast<void*>(dev::k_scan_merge_pipelined<CL>), dim3((unsigned)std::min<int64_t>(tiles, resident)),
+                                          dim3(kScanBlock + 32), params, 0, L.stream);
             else
               dev::k_scan_merge<CL><<<grid, kScanBlock, 0, L.stream>>>(a, per_row, (int)tiles, slab);
           }
@@ -434,10 +434,17 @@ struct Launcher {
         int per_row_arg = per_row, tiles_arg = (int)tiles;
         void* params[] = {&a, &per_row_arg, &tiles_arg};
         static int fit_on[2][64];
-        const void* kern = vec ? reinterpret_cast<const void*>(dev::k_scan<CL, true, true>) : reinterpret_cast<const void*>(dev::k_scan<CL, false, true>);
-        const int resident = resident_grid(kern, kScanBlock, fit_on[vec ? 1 : 0]);
+        // (small tiles: with a warp of its own for the look-back, see scan_tiles_pipelined)
+        constexpr bool kPipelined = dev::scan_pipelines<CL>();
+        constexpr int kThreads = kScanBlock + (kPipelined ? 32 : 0);
+        const void* kern;
+        if constexpr (kPipelined)
+          kern = vec ? reinterpret_cast<const void*>(dev::k_scan_pipelined<CL, true>) : reinterpret_cast<const void*>(dev::k_scan_pipelined<CL, false>);
+        else
+          kern = vec ? reinterpret_cast<const void*>(dev::k_scan<CL, true, true>) : reinterpret_cast<const void*>(dev::k_scan<CL, false, true>);
+        const int resident = resident_grid(kern, kThreads, fit_on[vec ? 1 : 0]);
         if (resident > 0)
-          cudaLaunchCooperativeKernel(const_cast<void*>(kern), dim3((unsigned)std::min<int64_t>(tiles, resident)), dim3(kScanBlock), params, 0, L.stream);
+          cudaLaunchCooperativeKernel(const_cast<void*>(kern), dim3((unsigned)std::min<int64_t>(tiles, resident)), dim3(kThreads), params, 0, L.stream);
         else if (vec) dev::k_scan<CL, true><<<grid, kScanBlock, 0, L.stream>>>(a, per_row, (int)tiles);
         else dev::k_scan<CL, false><<<grid, kScanBlock, 0, L.stream>>>(a, per_row, (int)tiles);
       }

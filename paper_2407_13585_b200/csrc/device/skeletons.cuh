@@ -495,67 +495,47 @@ constexpr bool needs_scan(const CCluster& c, int i, int s) {
   return false;
 }
 
+// What one tile of a scan takes, in the three parts that the kernels below put together: a warp's share of the tile
+// evaluated and scanned in registers, the look-back of one warp for the tile's prefix, and the final values stored.
 // Rows of a rank-2 array are scanned independently: a row is cut into tiles of its own, the
 // look-back of a tile stops at the first tile of its row.  A right-to-left scan walks its row
 // from the far end: position p of the walk is element C-1-p of the row.
-// STATIC: block b walks tiles b, b + G, b + 2G, ... of a grid of G blocks that are all resident at once (a
-// cooperative launch): no ticket, whose atomic every warp of the block would otherwise wait for at the top of every
-// tile (measured on a streaming scan of 2^26 floats: 28 barrier-stall cycles per issued instruction, 19 % of the
-// issue slots used).  A tile's predecessors belong to the blocks before this one in the same round, or to an
-// earlier round, so they are running or done.  Without that guarantee the tiles are claimed from a ticket.
-template <class CL, bool VEC, bool SLAB, bool STATIC = false>
-__device__ __forceinline__ void scan_tiles(const Args<CL::c.n>& a, int tiles_per_row, int n_tiles, const SlabIn& slab) {
-  constexpr int N = CL::c.n;
-  constexpr int W = VEC ? 4 : 1;
-  constexpr int BLOCK = scan_block<CL>();
-  constexpr int ROWS = VEC ? scan_rows<CL>() : scan_rows<CL>() * 4;   // as many elements per thread either way
-  constexpr int TILE = BLOCK * scan_rows<CL>() * 4;
-  constexpr int S = first_scan<CL>();
+template <class CL, bool VEC, bool SLAB>
+struct ScanTile {
+  static constexpr int N = CL::c.n;
+  static constexpr int W = VEC ? 4 : 1;
+  static constexpr int BLOCK = scan_block<CL>();
+  static constexpr int ROWS = VEC ? scan_rows<CL>() : scan_rows<CL>() * 4;   // as many elements per thread either way
+  static constexpr int TILE = BLOCK * scan_rows<CL>() * 4;
+  static constexpr int PART = TILE / (BLOCK / 32);         // elements of a tile that one warp takes
+  static constexpr int S = first_scan<CL>();
   static_assert(S >= 0, "k_scan needs a scan member");
-  constexpr CNode sn = CL::c.nodes[S];
-  constexpr int FN = sn.fn, DT = sn.dtype;
-  constexpr bool REV = sn.kind == ACC_SCANR;
-  constexpr bool EXCL = sn.p0 == 1;                        // seeded and exclusive: element k leaves itself out
+  static constexpr CNode sn = CL::c.nodes[S];
+  static constexpr int FN = sn.fn, DT = sn.dtype;
+  static constexpr bool REV = sn.kind == ACC_SCANR;
+  static constexpr bool EXCL = sn.p0 == 1;                 // seeded and exclusive: element k leaves itself out
+  static constexpr bool WIDE = FN == ACC_FN_ADD && DT == ACC_F32;
   using IX = std::conditional_t<VEC, std::conditional_t<REV, IxR4, Ix4>, Ix>;
+  static_assert(!SLAB || (VEC && PART == kSlabWarpTile && !REV), "the merging scan walks rank-1 tiles of 512-element warp tiles");
 
-  __shared__ uint32_t warp_total[BLOCK / 32];
-  __shared__ uint32_t tile_prefix;
-  __shared__ int tile_id;
-  __shared__ __align__(16) uint32_t slab_stage[SLAB ? BLOCK / 32 : 1][SLAB ? kSlabWarpTile : 1];   // read and written 128 bits at a time
-  static_assert(!SLAB || (VEC && TILE == (BLOCK / 32) * kSlabWarpTile && !REV), "the merging scan walks rank-1 tiles of eight 512-element warp tiles");
-  uint64_t* states = reinterpret_cast<uint64_t*>(a.scratch + 4);
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int n = a.C;                                       // length of a row
-  auto index_at = [&](int row, int p) {                    // walk position p (a multiple of W) of a row -> index
+  static __device__ __forceinline__ IX index_at(int n, int row, int p) {   // walk position p (a multiple of W) of a row of n -> index
     IX ix;
     ix.r = row;
     ix.c = REV ? n - 1 - p : p;
     return ix;
-  };
+  }
 
-  for (int round = 0;; ++round) {
-    int tile;
-    if constexpr (STATIC) {
-      // (no barrier here: what a round shares through shared memory is read before its second barrier or right
-      // after it, and written again only behind the next round's first barrier)
-      tile = (int)blockIdx.x + round * (int)gridDim.x;
-    } else {
-      __syncthreads();
-      if (threadIdx.x == 0) tile_id = (int)atomicAdd(a.scratch, 1u);
-      __syncthreads();
-      tile = tile_id;
-    }
-    if (tile >= n_tiles) return;
-    const int row = tile / tiles_per_row, in_row = tile - row * tiles_per_row;
-    const int warp_base = in_row * TILE + warp * (TILE / (BLOCK / 32));
-
-    uint32_t val[ROWS][W];
-    // SLAB: the gathered values of this warp's 512 elements lie, grouped by slab, where the scan's results will go;
-    // they are put back into element order (positions from the slab codes: a stable counting sort undone)
+  // The warp's PART elements from walk position warp_base of `row` on: evaluated, stored where a root does not need
+  // the scan, and scanned within the warp (val: each element's scan over the warp's part).  Returns the part's total.
+  // SLAB: the gathered values of warp tile `wt` lie, grouped by slab, where the scan's results will go; they are put
+  // back into element order through `stage` (kSlabWarpTile words of shared memory that this warp owns).
+  static __device__ __forceinline__ uint32_t scan_part(const Args<N>& a, int row, int warp_base, int wt, const SlabIn& slab,
+                                                       uint32_t* stage, uint32_t (&val)[ROWS][W]) {
+    const int lane = threadIdx.x & 31;
+    const int n = a.C;                                     // length of a row
     V4 gathered[SLAB ? ROWS : 1];
     bool merged = false;                                   // the same for a whole warp
     if constexpr (SLAB) {
-      const int wt = tile * (BLOCK / 32) + warp;
       if (wt < slab.full_tiles) {
         merged = true;
         const uint32_t code = __ldg(slab.codes + (size_t)wt * 32 + lane), cnt3 = __ldg(slab.counts + wt);
@@ -575,10 +555,9 @@ __device__ __forceinline__ void scan_tiles(const Args<CL::c.n>& a, int tiles_per
         const uint32_t t0 = cnt3 & 1023u, t1 = (cnt3 >> 10) & 1023u, t2 = (cnt3 >> 20) & 1023u;
         uint32_t a01 = (i01 - c01) + (t0 << 16);                             // next position in the lists of slabs 0 | 1
         uint32_t a23 = (i23 - c23) + (t0 + t1) + ((t0 + t1 + t2) << 16);     // ... of slabs 2 | 3
-        uint32_t* mine = slab_stage[warp];
         __syncwarp();
 #pragma unroll
-        for (int j = 0; j < ROWS; ++j) *reinterpret_cast<uint4*>(mine + (j * 32 + lane) * 4) = st[j];
+        for (int j = 0; j < ROWS; ++j) *reinterpret_cast<uint4*>(stage + (j * 32 + lane) * 4) = st[j];
         __syncwarp();
 #pragma unroll
         for (int j = 0; j < ROWS; ++j)
@@ -586,19 +565,9 @@ __device__ __forceinline__ void scan_tiles(const Args<CL::c.n>& a, int tiles_per
           for (int e = 0; e < 4; ++e) {
             const uint32_t sl = (code >> (2 * (4 * j + e))) & 3u;
             const uint32_t sh = 16 * (sl & 1);
-            gathered[j].v[e] = mine[((sl < 2 ? a01 : a23) >> sh) & (kSlabWarpTile - 1)];
+            gathered[j].v[e] = stage[((sl < 2 ? a01 : a23) >> sh) & (kSlabWarpTile - 1)];
             if (sl < 2) a01 += 1u << sh; else a23 += 1u << sh;
           }
-      }
-    }
-    if constexpr (SLAB && STATIC) {
-      // this block's next tile is known: its staged values and codes are asked into L2 now, so that they arrive while
-      // this tile is scanned and looked back for (config-3 shape, 2^26 elements: 0.726 -> 0.704 ms for the cluster)
-      const int nwt = (tile + (int)gridDim.x) * (BLOCK / 32) + warp;
-      if (nwt < slab.full_tiles) {
-        const char* q = lane < 16 ? reinterpret_cast<const char*>(reinterpret_cast<const uint32_t*>(a.n[S].ptr) + (size_t)nwt * kSlabWarpTile) + lane * 128
-                                  : reinterpret_cast<const char*>(slab.codes + (size_t)nwt * 32);
-        if (lane <= 16) asm volatile("prefetch.global.L2 [%0];" ::"l"(q));
       }
     }
     uint32_t carry = identity_of<FN, DT>();                // running total of this warp's earlier rows
@@ -607,7 +576,7 @@ __device__ __forceinline__ void scan_tiles(const Args<CL::c.n>& a, int tiles_per
       const int c = warp_base + (j * 32 + lane) * W;
       const bool live = c < n;
       if (live) {
-        const IX ix = index_at(row, c);
+        const IX ix = index_at(n, row, c);
         val_of<IX> v;
         if constexpr (SLAB) {
           if (merged) {
@@ -659,73 +628,73 @@ __device__ __forceinline__ void scan_tiles(const Args<CL::c.n>& a, int tiles_per
       }
       carry = combine<FN, DT>(carry, __shfl_sync(0xFFFFFFFFu, incl, 31));
     }
-    if (lane == 0) warp_total[warp] = carry;
-    __syncthreads();
-    uint32_t offset = identity_of<FN, DT>();               // total of the warps before this one
-    uint32_t tile_total = identity_of<FN, DT>();
-#pragma unroll
-    for (int w = 0; w < BLOCK / 32; ++w) {
-      const uint32_t t = warp_total[w];
-      if (w < warp) offset = combine<FN, DT>(offset, t);
-      tile_total = combine<FN, DT>(tile_total, t);
-    }
+    return carry;
+  }
 
-    if (warp == 0) {
-      constexpr bool WIDE = FN == ACC_FN_ADD && DT == ACC_F32;
-      uint32_t exclusive = identity_of<FN, DT>();
-      if (in_row == 0) {
-        if (lane == 0) st_state(states + tile, kFlagPrefix, tile_total);
-      } else {
-        if (lane == 0) st_state(states + tile, kFlagAggregate, tile_total);
-        int look = in_row - 1;                             // tiles of this row before this one
-        uint32_t spins = 0;
-        bool gave_up = false;
-        double wide = 0.0;                                 // WIDE: the sum of the tiles before this one
-        for (;;) {
-          const int idx = look - lane;
-          const uint64_t* at = states + (tile - in_row) + idx;
-          uint64_t s = idx >= 0 ? ld_state(at) : ((uint64_t)identity_of<FN, DT>() << 32) | kFlagPrefix;
-          while (__any_sync(0xFFFFFFFFu, flag_of(s) == 0)) {
-            if (++spins > a.spin_limit) { gave_up = true; break; }
-            __nanosleep(20);
-            if (idx >= 0) s = ld_state(at);
-          }
-          if (gave_up) break;
-          const unsigned done = __ballot_sync(0xFFFFFFFFu, flag_of(s) == kFlagPrefix);
-          const int stop = done ? __ffs(done) - 1 : 31;
-          if constexpr (WIDE) {
-            double part = lane <= stop ? wide_of(s) : 0.0;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
-            wide += part;
-          } else {
-            uint32_t part = lane <= stop ? value_of(s) : identity_of<FN, DT>();
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) part = combine<FN, DT>(part, __shfl_xor_sync(0xFFFFFFFFu, part, o));
-            exclusive = combine<FN, DT>(part, exclusive);
-          }
-          if (done) break;
-          look -= 32;
-        }
-        if (gave_up && lane == 0) atomicOr(a.status, kStatusTimeout);
-        if constexpr (WIDE) {
-          exclusive = u_((float)wide);
-          if (lane == 0) st_wide(states + tile, wide + (double)f_(tile_total));
-        } else {
-          if (lane == 0) st_state(states + tile, kFlagPrefix, combine<FN, DT>(exclusive, tile_total));
-        }
-      }
-      if (lane == 0) tile_prefix = exclusive;
+  // One warp publishes the tile's total, looks back over the tiles of its row before it and publishes the tile's
+  // inclusive prefix.  Returns (in every lane) what came before the tile.  A wait that runs out sets the status flag.
+  static __device__ __forceinline__ uint32_t look_back(const Args<N>& a, int tile, int in_row, uint32_t tile_total) {
+    const int lane = threadIdx.x & 31;
+    uint64_t* states = reinterpret_cast<uint64_t*>(a.scratch + 4);
+    uint32_t exclusive = identity_of<FN, DT>();
+    if (in_row == 0) {
+      if (lane == 0) st_state(states + tile, kFlagPrefix, tile_total);
+      return exclusive;
     }
-    __syncthreads();
-    uint32_t base = combine<FN, DT>(tile_prefix, offset);
+    if (lane == 0) st_state(states + tile, kFlagAggregate, tile_total);
+    int look = in_row - 1;                                 // tiles of this row before this one
+    uint32_t spins = 0;
+    bool gave_up = false;
+    double wide = 0.0;                                     // WIDE: the sum of the tiles before this one
+    for (;;) {
+      const int idx = look - lane;
+      const uint64_t* at = states + (tile - in_row) + idx;
+      uint64_t s = idx >= 0 ? ld_state(at) : ((uint64_t)identity_of<FN, DT>() << 32) | kFlagPrefix;
+      while (__any_sync(0xFFFFFFFFu, flag_of(s) == 0)) {
+        if (++spins > a.spin_limit) { gave_up = true; break; }
+        __nanosleep(20);
+        if (idx >= 0) s = ld_state(at);
+      }
+      if (gave_up) break;
+      const unsigned done = __ballot_sync(0xFFFFFFFFu, flag_of(s) == kFlagPrefix);
+      const int stop = done ? __ffs(done) - 1 : 31;
+      if constexpr (WIDE) {
+        double part = lane <= stop ? wide_of(s) : 0.0;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
+        wide += part;
+      } else {
+        uint32_t part = lane <= stop ? value_of(s) : identity_of<FN, DT>();
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) part = combine<FN, DT>(part, __shfl_xor_sync(0xFFFFFFFFu, part, o));
+        exclusive = combine<FN, DT>(part, exclusive);
+      }
+      if (done) break;
+      look -= 32;
+    }
+    if (gave_up && lane == 0) atomicOr(a.status, kStatusTimeout);
+    if constexpr (WIDE) {
+      exclusive = u_((float)wide);
+      if (lane == 0) st_wide(states + tile, wide + (double)f_(tile_total));
+    } else {
+      if (lane == 0) st_state(states + tile, kFlagPrefix, combine<FN, DT>(exclusive, tile_total));
+    }
+    return exclusive;
+  }
+
+  // The warp's part once `before` (everything of the row ahead of the part) is known: the scan is stored, and so is
+  // every root that reads it.
+  static __device__ __forceinline__ void finish_part(const Args<N>& a, int row, int warp_base, uint32_t before, const uint32_t (&val)[ROWS][W]) {
+    const int lane = threadIdx.x & 31;
+    const int n = a.C;
+    uint32_t base = before;
     if constexpr (EXCL) base = combine<FN, DT>(DT == ACC_F32 ? u_(a.n[S].fp0) : (uint32_t)a.n[S].ip0, base);   // the seed comes first
     uint32_t* out = reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[S].ptr));
 #pragma unroll
     for (int j = 0; j < ROWS; ++j) {
       const int c = warp_base + (j * 32 + lane) * W;
       if (c < n) {
-        const IX ix = index_at(row, c);
+        const IX ix = index_at(n, row, c);
         IxSc<IX> scanned;
         static_cast<IX&>(scanned) = ix;
         if constexpr (VEC) {
@@ -743,11 +712,178 @@ __device__ __forceinline__ void scan_tiles(const Args<CL::c.n>& a, int tiles_per
       }
     }
   }
+
+  // SLAB: the staged values and codes of warp tile `wt` are asked into L2 ahead of their use
+  static __device__ __forceinline__ void prefetch_part(const Args<N>& a, int wt, const SlabIn& slab) {
+    const int lane = threadIdx.x & 31;
+    if (wt < slab.full_tiles) {
+      const char* q = lane < 16 ? reinterpret_cast<const char*>(reinterpret_cast<const uint32_t*>(a.n[S].ptr) + (size_t)wt * kSlabWarpTile) + lane * 128
+                                : reinterpret_cast<const char*>(slab.codes + (size_t)wt * 32);
+      if (lane <= 16) asm volatile("prefetch.global.L2 [%0];" ::"l"(q));
+    }
+  }
+};
+
+// Tile after tile with the whole block in step: every warp scans its part, one warp looks back, every warp stores.
+// STATIC: block b walks tiles b, b + G, b + 2G, ... of a grid of G blocks that are all resident at once (a
+// cooperative launch): no ticket, whose atomic every warp of the block would otherwise wait for at the top of every
+// tile (measured on a streaming scan of 2^26 floats: 28 barrier-stall cycles per issued instruction, 19 % of the
+// issue slots used).  A tile's predecessors belong to the blocks before this one in the same round, or to an
+// earlier round, so they are running or done.  Without that guarantee the tiles are claimed from a ticket.
+template <class CL, bool VEC, bool SLAB, bool STATIC = false>
+__device__ __forceinline__ void scan_tiles(const Args<CL::c.n>& a, int tiles_per_row, int n_tiles, const SlabIn& slab) {
+  using T = ScanTile<CL, VEC, SLAB>;
+  constexpr int BLOCK = T::BLOCK, FN = T::FN, DT = T::DT;
+  __shared__ uint32_t warp_total[BLOCK / 32];
+  __shared__ uint32_t tile_prefix;
+  __shared__ int tile_id;
+  __shared__ __align__(16) uint32_t slab_stage[SLAB ? BLOCK / 32 : 1][SLAB ? kSlabWarpTile : 1];   // read and written 128 bits at a time
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+  for (int round = 0;; ++round) {
+    int tile;
+    if constexpr (STATIC) {
+      // (no barrier here: what a round shares through shared memory is read before its second barrier or right
+      // after it, and written again only behind the next round's first barrier)
+      tile = (int)blockIdx.x + round * (int)gridDim.x;
+    } else {
+      __syncthreads();
+      if (threadIdx.x == 0) tile_id = (int)atomicAdd(a.scratch, 1u);
+      __syncthreads();
+      tile = tile_id;
+    }
+    if (tile >= n_tiles) return;
+    const int row = tile / tiles_per_row, in_row = tile - row * tiles_per_row;
+    const int warp_base = in_row * T::TILE + warp * T::PART;
+
+    if constexpr (SLAB && STATIC) {
+      // this block's next tile is known: its staged values are on their way while this tile is scanned and looked
+      // back for (config-3 shape, 2^26 elements: 0.726 -> 0.704 ms for the cluster)
+      T::prefetch_part(a, (tile + (int)gridDim.x) * (BLOCK / 32) + warp, slab);
+    }
+    uint32_t val[T::ROWS][T::W];
+    const uint32_t carry = T::scan_part(a, row, warp_base, tile * (BLOCK / 32) + warp, slab, slab_stage[SLAB ? warp : 0], val);
+    if (lane == 0) warp_total[warp] = carry;
+    __syncthreads();
+    uint32_t offset = identity_of<FN, DT>();               // total of the warps before this one
+    uint32_t tile_total = identity_of<FN, DT>();
+#pragma unroll
+    for (int w = 0; w < BLOCK / 32; ++w) {
+      const uint32_t t = warp_total[w];
+      if (w < warp) offset = combine<FN, DT>(offset, t);
+      tile_total = combine<FN, DT>(tile_total, t);
+    }
+    if (warp == 0) {
+      const uint32_t exclusive = T::look_back(a, tile, in_row, tile_total);
+      if (lane == 0) tile_prefix = exclusive;
+    }
+    __syncthreads();
+    T::finish_part(a, row, warp_base, combine<FN, DT>(tile_prefix, offset), val);
+  }
+}
+
+// Named barriers (ids 1..4; id 0 is __syncthreads'): `count` threads take part, arriving or waiting.
+template <int ID> __device__ __forceinline__ void bar_sync_id(int count) { asm volatile("bar.sync %0, %1;" ::"n"(ID), "r"(count) : "memory"); }
+template <int ID> __device__ __forceinline__ void bar_arrive_id(int count) { asm volatile("bar.arrive %0, %1;" ::"n"(ID), "r"(count) : "memory"); }
+// (barrier `first` for half 0, `first + 1` for half 1, as immediates)
+template <int FIRST> __device__ __forceinline__ void bar_sync(int half, int count) { if (half) bar_sync_id<FIRST + 1>(count); else bar_sync_id<FIRST>(count); }
+template <int FIRST> __device__ __forceinline__ void bar_arrive(int half, int count) { if (half) bar_arrive_id<FIRST + 1>(count); else bar_arrive_id<FIRST>(count); }
+
+// The same tiles with the look-back taken out of the block's way: BLOCK / 32 warps scan parts and one more warp does
+// nothing but look back.  A scanning warp leaves its part's values in shared memory, tells the look-back warp that
+// the part's total is in, goes on to its part of the block's next tile, and only then comes back for the values,
+// which it finishes with what the look-back warp has found meanwhile.  Where the whole block waits for the look-back
+// (scan_tiles), the blocks of a cooperative grid fall into step and an SM's blocks all wait at once.
+// Round r uses half r & 1 of everything shared.  Barrier 1 + half: a part's total is in shared memory (the scanning
+// warps arrive, the look-back warp waits); barrier 3 + half: what comes before each part is in shared memory (the
+// look-back warp arrives, the scanning warps wait).  Every warp of a block walks the same rounds, so that each
+// barrier sees BLOCK + 32 threads once a round.  Only for grids whose blocks are all resident (STATIC tiles).
+template <class CL, bool VEC, bool SLAB>
+__device__ __forceinline__ void scan_tiles_pipelined(const Args<CL::c.n>& a, int tiles_per_row, int n_tiles, const SlabIn& slab) {
+  using T = ScanTile<CL, VEC, SLAB>;
+  constexpr int BLOCK = T::BLOCK, WARPS = BLOCK / 32, FN = T::FN, DT = T::DT, ROWS = T::ROWS, W = T::W;
+  static_assert(WARPS <= 32, "one lane of the look-back warp per scanning warp");
+  __shared__ __align__(16) uint32_t values[2][T::TILE];    // a part's scanned values between its two visits (SLAB: first the staging area of its merge)
+  __shared__ uint32_t part_total[2][WARPS];
+  __shared__ uint32_t part_before[2][WARPS];               // what of the row comes before each part
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int G = (int)gridDim.x;
+
+  if (warp == WARPS) {
+    for (int round = 0;; ++round) {
+      const int tile = (int)blockIdx.x + round * G;
+      if (tile >= n_tiles) return;
+      const int half = round & 1;
+      const int row = tile / tiles_per_row, in_row = tile - row * tiles_per_row;
+      bar_sync<1>(half, BLOCK + 32);
+      uint32_t incl = lane < WARPS ? part_total[half][lane] : identity_of<FN, DT>();
+#pragma unroll
+      for (int o = 1; o < WARPS; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl = combine<FN, DT>(t, incl);
+      }
+      uint32_t earlier = __shfl_up_sync(0xFFFFFFFFu, incl, 1);                 // total of the parts before lane's
+      if (lane == 0) earlier = identity_of<FN, DT>();
+      const uint32_t tile_total = __shfl_sync(0xFFFFFFFFu, incl, WARPS - 1);
+      const uint32_t exclusive = T::look_back(a, tile, in_row, tile_total);
+      if (lane < WARPS) part_before[half][lane] = combine<FN, DT>(exclusive, earlier);
+      bar_arrive<3>(half, BLOCK + 32);
+    }
+  }
+
+  auto finish = [&](int tile, int half) {
+    const int row = tile / tiles_per_row, in_row = tile - row * tiles_per_row;
+    bar_sync<3>(half, BLOCK + 32);
+    const uint32_t before = part_before[half][warp];
+    const uint32_t* mine = values[half] + warp * T::PART;
+    uint32_t val[ROWS][W];
+#pragma unroll
+    for (int j = 0; j < ROWS; ++j) {
+      if constexpr (VEC) {
+        const uint4 q = *reinterpret_cast<const uint4*>(mine + (j * 32 + lane) * 4);
+        val[j][0] = q.x; val[j][1] = q.y; val[j][2] = q.z; val[j][3] = q.w;
+      } else {
+        val[j][0] = mine[j * 32 + lane];
+      }
+    }
+    T::finish_part(a, row, in_row * T::TILE + warp * T::PART, before, val);
+  };
+
+  int round = 0;
+  for (;; ++round) {
+    const int tile = (int)blockIdx.x + round * G;
+    if (tile >= n_tiles) break;
+    const int half = round & 1;
+    const int row = tile / tiles_per_row, in_row = tile - row * tiles_per_row;
+    uint32_t* mine = values[half] + warp * T::PART;
+    if constexpr (SLAB) T::prefetch_part(a, (tile + G) * WARPS + warp, slab);
+    {
+      uint32_t val[ROWS][W];
+      const uint32_t total = T::scan_part(a, row, in_row * T::TILE + warp * T::PART, tile * WARPS + warp, slab, mine, val);
+      __syncwarp();                                        // (SLAB: every lane has taken its merged values out of `mine`)
+#pragma unroll
+      for (int j = 0; j < ROWS; ++j) {
+        if constexpr (VEC) *reinterpret_cast<uint4*>(mine + (j * 32 + lane) * 4) = make_uint4(val[j][0], val[j][1], val[j][2], val[j][3]);
+        else mine[j * 32 + lane] = val[j][0];
+      }
+      if (lane == 0) part_total[half][warp] = total;
+    }
+    bar_arrive<1>(half, BLOCK + 32);
+    if (round > 0) finish(tile - G, half ^ 1);
+  }
+  if (round > 0) finish((int)blockIdx.x + (round - 1) * G, (round - 1) & 1);
 }
 
 template <class CL, bool VEC, bool STATIC = false>
 __global__ void __launch_bounds__(scan_block<CL>()) k_scan(const __grid_constant__ Args<CL::c.n> a, int tiles_per_row, int n_tiles) {
   scan_tiles<CL, VEC, false, STATIC>(a, tiles_per_row, n_tiles, SlabIn{});
+}
+
+// (a tile's values stay in shared memory twice over: only for tiles of at most 16 KB)
+template <class CL> constexpr bool scan_pipelines() { return scan_block<CL>() * scan_rows<CL>() * 4 <= 4096; }
+template <class CL, bool VEC>
+__global__ void __launch_bounds__(scan_block<CL>() + 32) k_scan_pipelined(const __grid_constant__ Args<CL::c.n> a, int tiles_per_row, int n_tiles) {
+  if constexpr (scan_pipelines<CL>()) scan_tiles_pipelined<CL, VEC, false>(a, tiles_per_row, n_tiles, SlabIn{});
 }
 
 }  // namespace dev

@@ -177,5 +177,11 @@ __global__ void __launch_bounds__(scan_block<CL>(), 5) k_scan_merge(const __grid
   scan_tiles<CL, true, true, STATIC>(a, tiles_per_row, n_tiles, slab);
 }
 
+template <class CL>
+__global__ void __launch_bounds__(scan_block<CL>() + 32, 5) k_scan_merge_pipelined(const __grid_constant__ Args<CL::c.n> a, int tiles_per_row, int n_tiles,
+                                                                                  const SlabIn slab) {
+  scan_tiles_pipelined<CL, true, true>(a, tiles_per_row, n_tiles, slab);
+}
+
 }  // namespace dev
 }  // namespace acc
