@@ -85,6 +85,39 @@ def test_gather_scan_in_slab_passes_ragged():
         compare(prog, ref, got, "gather + scan in slab passes, pi=%s" % pi)
 
 
+def test_gathering_scans_over_several_rounds_of_a_resident_grid():
+    """Scans with a gather in their cluster walk tiles of 4096 elements with a warp that only looks back; here a block
+    takes several tiles in turn (2^23 elements are 2048 tiles, more than the blocks one launch holds), and the last
+    tile of the second program is ragged."""
+    prog = W.offsets_then_gather(1 << 23)
+    got, inputs, pi, g = run_full(prog, "enumerate")
+    ref = oracle_run(prog, {k: v.cpu().numpy() for k, v in inputs.items()})
+    compare(prog, ref, got, "offsets_then_gather, 2^23")
+    # gather + scan with a 32 MB source (no slab passes) and an odd count of indices: element by element, ragged last tile
+    import torch
+    from workloads import Node, Program
+    from paper_2407_13585_b200 import binding as B
+    n_src, n = 1 << 23, (1 << 23) - 1029
+    nodes = [Node("input", "i32", (n_src,), name="x"), Node("input", "i32", (n,), name="idx"),
+             Node("map", "i32", (n_src,), (0,), 1, fn="hash_mul_xorshift", iparam=(2654435761, 13), name="g"),
+             Node("gather", "i32", (n,), (1, 2), 2, name="h"),
+             Node("map", "i32", (n,), (3,), 1, fn="and_mask", iparam=(0xFFFF,), name="o"),
+             Node("scanl", "i32", (n,), (4,), 1, fn="add", name="out")]
+    prog = Program("gather_scan_odd", nodes, [5])
+    inputs = {0: W.uniform_int(0, 0, n_src, 1 << 31, device="cuda"), 1: W.uniform_int(0, 1, n, n_src, device="cuda")}
+    ref = oracle_run(prog, {k: v.cpu().numpy() for k, v in inputs.items()})
+    g = B.Graph(prog.nodes, prog.outputs)
+    g.set_partition([-1, -1, 0, 0, 0, 0])
+    for i, t in inputs.items():
+        g.bind(i, t)
+    out = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+    g.bind(5, out)
+    g.run(B.FUSED)
+    g.run(B.FUSED)
+    assert g.launch_count() == 1
+    compare(prog, ref, {5: out.cpu().numpy().view(np.uint32)}, "gather + scan, 2^23 - 1029 indices")
+
+
 def test_config5_full():
     prog = W.config5(1 << 27, 1 << 16)
     got, inputs, pi, g = run_full(prog, "enumerate")
