@@ -6,9 +6,11 @@
 //              with atomics.
 //   k_rowfold  one block per row of a rank-2 domain; folds of the innermost extent end in a
 //              block reduction, no atomics.
-//   k_scan     single-pass inclusive scan with decoupled look-back (tiles are claimed from
-//              an atomic ticket so that a tile's predecessors are always already running);
-//              the scanned operand is evaluated in registers.
+//   k_scan     single-pass scan with decoupled look-back; the scanned operand is evaluated in
+//              registers.  A tile's predecessors are always running or done: the grid is
+//              cooperative and block b takes tiles b, b + G, ..., or tiles are claimed from an
+//              atomic ticket.  k_scan_pipelined is the same scan with a warp that only looks
+//              back, for small tiles.
 //
 // Each is templated on the cluster description (what to evaluate) and on VEC (whether four
 // consecutive elements move as one 128-bit access).
