@@ -605,6 +605,31 @@ def test_lookback_wait_that_runs_out_is_reported():
     assert np.array_equal(out.cpu().numpy(), want)
 
 
+def test_lookback_wait_that_runs_out_where_a_warp_of_its_own_looks_back():
+    """The same wait in the scan that parks a tile's values and leaves the look-back to a ninth warp (scans with a
+    gather in their cluster): that warp gives up at once, still hands the other warps a prefix at their barrier, the
+    kernel ends normally and the run reports the time-out; with the default bound the graph gives the oracle's result."""
+    import torch
+    from paper_2407_13585_b200 import binding as B
+    prog = W.config3(1 << 22)
+    inputs = W.make_inputs(prog, device="cuda")
+    ref = oracle_run(prog, {k: v.cpu().numpy() for k, v in inputs.items()})
+    g = B.Graph(prog.nodes, prog.outputs)
+    g.set_partition([-1, -1, 0, 0, 0, 0])
+    for i, t in inputs.items():
+        g.bind(i, t)
+    out = torch.zeros(1 << 22, dtype=torch.int32, device="cuda")
+    g.bind(5, out)
+    g.set_spin_limit(0)
+    with pytest.raises(B.AccError) as e:
+        g.run(B.FUSED)
+    assert e.value.status == "ACC_ERR_DEVICE_TIMEOUT"
+    g.set_spin_limit(1 << 22)
+    g.run(B.FUSED)
+    assert g.launch_count() == 1
+    compare(prog, ref, {5: out.cpu().numpy().view(np.uint32)}, "config3 after a look-back that ran out")
+
+
 def test_runs_do_not_depend_on_what_the_workspace_held():
     """A run clears the status word and the part of every cluster's scratch that must start at zero, nothing else
     (partial sums per tile, records, staged operands are written before they are read): a workspace full of 0xFF
