@@ -488,6 +488,17 @@ struct SlabIn {
 };
 constexpr int kSlabWarpTile = 512;
 
+// Whether `leaf` (an array from outside the cluster) is read by member i at i's own index: through array operands
+// of maps and zipWiths only.
+constexpr bool reads_in_place(const CCluster& c, int i, int leaf) {
+  if (i == leaf) return true;
+  const CNode& n = c.nodes[i];
+  if (!n.member || (n.kind != ACC_MAP && n.kind != ACC_ZIPWITH)) return false;
+  for (int k = 0; k < n.narr; ++k)
+    if (reads_in_place(c, n.in[k], leaf)) return true;
+  return false;
+}
+
 // Whether member i needs the value of scan s (through any chain of operands inside the cluster).
 constexpr bool needs_scan(const CCluster& c, int i, int s) {
   const CNode& n = c.nodes[i];
@@ -715,6 +726,26 @@ struct ScanTile {
     }
   }
 
+  // The lines that the warp's part from walk position warp_base of `row` on will read in place, asked into L2
+  // (left-to-right scans; arrays from outside the cluster that the scanned operand reads at its own index).
+  static __device__ __forceinline__ void prefetch_operands(const Args<N>& a, int row, int warp_base) {
+    if constexpr (!REV) {
+      const int lane = threadIdx.x & 31;
+      const int n = a.C;
+      static_for<0, N>([&](auto ic) {
+        constexpr int i = decltype(ic)::value;
+        if constexpr (!CL::c.nodes[i].member && reads_in_place(CL::c, sn.in[0], i)) {
+          const char* base = reinterpret_cast<const char*>(a.n[i].ptr) + (size_t)row * n * 4;
+#pragma unroll
+          for (int k = 0; k < PART; k += 1024) {
+            const int at = warp_base + k + lane * 32;
+            if (at < n) asm volatile("prefetch.global.L2 [%0];" ::"l"(base + (size_t)at * 4));
+          }
+        }
+      });
+    }
+  }
+
   // SLAB: the staged values and codes of warp tile `wt` are asked into L2 ahead of their use
   static __device__ __forceinline__ void prefetch_part(const Args<N>& a, int wt, const SlabIn& slab) {
     const int lane = threadIdx.x & 31;
@@ -758,10 +789,16 @@ __device__ __forceinline__ void scan_tiles(const Args<CL::c.n>& a, int tiles_per
     const int row = tile / tiles_per_row, in_row = tile - row * tiles_per_row;
     const int warp_base = in_row * T::TILE + warp * T::PART;
 
-    if constexpr (SLAB && STATIC) {
-      // this block's next tile is known: its staged values are on their way while this tile is scanned and looked
-      // back for (config-3 shape, 2^26 elements: 0.726 -> 0.704 ms for the cluster)
-      T::prefetch_part(a, (tile + (int)gridDim.x) * (BLOCK / 32) + warp, slab);
+    if constexpr (STATIC) {
+      // this block's next tile is known: what it reads is on its way while this tile is scanned and looked back
+      // for (config-3 shape, 2^26 elements: 0.726 -> 0.704 ms for the cluster)
+      const int next = tile + (int)gridDim.x;
+      if constexpr (SLAB) {
+        T::prefetch_part(a, next * (BLOCK / 32) + warp, slab);
+      } else if (next < n_tiles) {
+        const int nrow = next / tiles_per_row;
+        T::prefetch_operands(a, nrow, (next - nrow * tiles_per_row) * T::TILE + warp * T::PART);
+      }
     }
     uint32_t val[T::ROWS][T::W];
     const uint32_t carry = T::scan_part(a, row, warp_base, tile * (BLOCK / 32) + warp, slab, slab_stage[SLAB ? warp : 0], val);
@@ -858,7 +895,12 @@ __device__ __forceinline__ void scan_tiles_pipelined(const Args<CL::c.n>& a, int
     const int half = round & 1;
     const int row = tile / tiles_per_row, in_row = tile - row * tiles_per_row;
     uint32_t* mine = values[half] + warp * T::PART;
-    if constexpr (SLAB) T::prefetch_part(a, (tile + G) * WARPS + warp, slab);
+    if constexpr (SLAB) {
+      T::prefetch_part(a, (tile + G) * WARPS + warp, slab);
+    } else if (tile + G < n_tiles) {
+      const int nrow = (tile + G) / tiles_per_row;
+      T::prefetch_operands(a, nrow, (tile + G - nrow * tiles_per_row) * T::TILE + warp * T::PART);
+    }
     {
       uint32_t val[ROWS][W];
       const uint32_t total = T::scan_part(a, row, in_row * T::TILE + warp * T::PART, tile * WARPS + warp, slab, mine, val);
