@@ -168,6 +168,25 @@ struct Launcher {
     }
   }
 
+  // The same for a cluster of element-wise roots only (k_stream_merge): every root a rank-1 array of the domain's length.
+  static constexpr bool kStreamSlabShape = dev::slab_stream_eligible<CL>();
+  static bool stream_slab_shapes_ok(const ClusterLaunch& L, int R, int C) {
+    if constexpr (kStreamSlabShape) {
+      const int src = CL::c.nodes[dev::the_gather<CL>()].in[1];
+      const int64_t src_bytes = (int64_t)L.nodes[src].R * L.nodes[src].C * 4;
+      for (int i = 0; i < N; ++i)
+        if (dev::is_store_root(CL::c.nodes[i]) && (L.nodes[i].R != 1 || L.nodes[i].C != C)) return false;
+      return R == 1 && C >= dev::kSlabMinElements && C % 4 == 0 && src_bytes >= dev::kSlabMinSourceBytes && src_bytes <= dev::kSlabMaxSourceBytes;
+    } else {
+      return false;
+    }
+  }
+  // bytes of the group sizes and slab codes of the slab passes, which lie behind `base` bytes of other scratch
+  static int64_t with_slab_area(int64_t base, int C) {
+    const int64_t full = C / dev::kSlabWarpTile;
+    return ((base + 15) & ~int64_t(15)) + full * 4 + full * 32 * 4;
+  }
+
   static int64_t scratch_bytes(const ClusterLaunch& L) {
     int R, C;
     if (!domain(L, R, C)) return ACC_ERR_NO_KERNEL;
@@ -190,6 +209,7 @@ struct Launcher {
       if (dev::is_f32_add_permute(CL::c.nodes[i])) words += 2 * (int64_t)L.nodes[i].R * L.nodes[i].C;
     dev::HistPlan plan;
     if (use_hist(L, R, C, plan)) words += (int64_t)sm_count() * plan.overflow;   // private overflow bins per CTA
+    if (stream_slab_shapes_ok(L, R, C)) return with_slab_area(words * 4, C);
     return words * 4;
   }
 
@@ -200,6 +220,7 @@ struct Launcher {
     if (!domain(L, R, C)) return 0;
     if (use_tiles(L, R, C)) return dev::tile_partials_off((R + dev::kTile - 1) / dev::kTile) * 4;
     if (kHasScan && slab_shapes_ok(L, R, C)) return ((16 + (int64_t)R * ((C + kScanTile - 1) / kScanTile) * 8) + 15) & ~int64_t(15);
+    if (stream_slab_shapes_ok(L, R, C)) return (((int64_t)dev::stream_acc64_off(kScalarFolds, sm_count() * 8) * 4) + 15) & ~int64_t(15);
     return scratch_bytes(L);
   }
 
@@ -457,6 +478,28 @@ struct Launcher {
       if constexpr (kHistShape) {
         const int rc = launch_hist(L, a, R, C, vec);
         if (rc != 1) return rc;                        // 1 = not worth it or does not fit: stream instead
+      }
+      if constexpr (kStreamSlabShape) {
+        if (vec && stream_slab_shapes_ok(L, R, C)) {
+          // the gather's source does not fit L2: partition the indices by slab, gather slab by slab, store from the merged values
+          const int src = CL::c.nodes[dev::the_gather<CL>()].in[1];
+          const int64_t n_src = (int64_t)L.nodes[src].R * L.nodes[src].C;
+          const uint32_t mul = (uint32_t)(((uint64_t)dev::kSlabs << 32) / (uint64_t)n_src);
+          const int full = C / dev::kSlabWarpTile;
+          const int64_t base = (((int64_t)dev::stream_acc64_off(kScalarFolds, sm_count() * 8) * 4) + 15) & ~int64_t(15);
+          uint32_t* counts = L.scratch + base / 4;
+          uint32_t* codes = counts + full;
+          const int warps = dev::kBlock / 32;
+          const int pgrid = (int)std::min<int64_t>((full + warps - 1) / warps, (int64_t)sm_count() * 4);
+          const int ggrid = (int)std::min<int64_t>((full + warps - 1) / warps, (int64_t)sm_count() * 8);
+          dev::k_slab_partition<CL><<<pgrid, dev::kBlock, 0, L.stream>>>(a, codes, counts, full, mul);
+          for (int k = 0; k < dev::kSlabs; ++k) dev::k_slab_gather<CL><<<ggrid, dev::kBlock, 0, L.stream>>>(a, counts, full, (uint32_t)k);
+          dev::k_stream_merge<CL><<<pgrid, dev::kBlock, 0, L.stream>>>(a, dev::SlabIn{codes, counts, full});
+          L.extra_launches = 1 + dev::kSlabs;
+          const cudaError_t e = cudaGetLastError();
+          if (e != cudaSuccess) return set_error(ACC_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+          return ACC_OK;
+        }
       }
       // an empty domain still runs one block: a scatter must copy its defaults out
       const int grid = stream_grid(R, C, vec);

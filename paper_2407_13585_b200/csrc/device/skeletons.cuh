@@ -499,6 +499,45 @@ constexpr bool reads_in_place(const CCluster& c, int i, int leaf) {
   return false;
 }
 
+// The gathered values of warp tile `wt` (kSlabWarpTile elements, grouped by slab where `staged` holds them) in element
+// order: lane's elements (j * 32 + lane) * 4 .. + 3 in gathered[j].  The stable counting sort of k_slab_partition is undone
+// from the slab codes and the group sizes, through `stage` (kSlabWarpTile words of shared memory that the warp owns).
+template <int ROWS>
+__device__ __forceinline__ void unpermute_warp_tile(const uint32_t* staged_array, const SlabIn& slab, int wt, uint32_t* stage, V4 (&gathered)[ROWS]) {
+  static_assert(ROWS * 128 == kSlabWarpTile, "a lane holds 16 elements of the warp tile");
+  const int lane = threadIdx.x & 31;
+  const uint32_t code = __ldg(slab.codes + (size_t)wt * 32 + lane), cnt3 = __ldg(slab.counts + wt);
+  const uint32_t* staged = staged_array + (size_t)wt * kSlabWarpTile;
+  uint4 st[ROWS];
+#pragma unroll
+  for (int j = 0; j < ROWS; ++j) st[j] = *reinterpret_cast<const uint4*>(staged + (j * 32 + lane) * 4);
+  const uint32_t lo1 = code & 0x55555555u, hi1 = (code >> 1) & 0x55555555u;
+  const uint32_t n3 = __popc(lo1 & hi1), n2 = __popc(hi1 & ~lo1), n1 = __popc(lo1 & ~hi1);
+  const uint32_t c01 = (16u - n1 - n2 - n3) | (n1 << 16), c23 = n2 | (n3 << 16);     // this lane's elements per slab
+  uint32_t i01 = c01, i23 = c23;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t u0 = __shfl_up_sync(0xFFFFFFFFu, i01, o), u1 = __shfl_up_sync(0xFFFFFFFFu, i23, o);
+    if (lane >= o) { i01 += u0; i23 += u1; }
+  }
+  const uint32_t t0 = cnt3 & 1023u, t1 = (cnt3 >> 10) & 1023u, t2 = (cnt3 >> 20) & 1023u;
+  uint32_t a01 = (i01 - c01) + (t0 << 16);                             // next position in the lists of slabs 0 | 1
+  uint32_t a23 = (i23 - c23) + (t0 + t1) + ((t0 + t1 + t2) << 16);     // ... of slabs 2 | 3
+  __syncwarp();
+#pragma unroll
+  for (int j = 0; j < ROWS; ++j) *reinterpret_cast<uint4*>(stage + (j * 32 + lane) * 4) = st[j];
+  __syncwarp();
+#pragma unroll
+  for (int j = 0; j < ROWS; ++j)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const uint32_t sl = (code >> (2 * (4 * j + e))) & 3u;
+      const uint32_t sh = 16 * (sl & 1);
+      gathered[j].v[e] = stage[((sl < 2 ? a01 : a23) >> sh) & (kSlabWarpTile - 1)];
+      if (sl < 2) a01 += 1u << sh; else a23 += 1u << sh;
+    }
+}
+
 // Whether member i needs the value of scan s (through any chain of operands inside the cluster).
 constexpr bool needs_scan(const CCluster& c, int i, int s) {
   const CNode& n = c.nodes[i];
@@ -551,36 +590,7 @@ struct ScanTile {
     if constexpr (SLAB) {
       if (wt < slab.full_tiles) {
         merged = true;
-        const uint32_t code = __ldg(slab.codes + (size_t)wt * 32 + lane), cnt3 = __ldg(slab.counts + wt);
-        const uint32_t* staged = reinterpret_cast<const uint32_t*>(a.n[S].ptr) + (size_t)wt * kSlabWarpTile;
-        uint4 st[ROWS];
-#pragma unroll
-        for (int j = 0; j < ROWS; ++j) st[j] = *reinterpret_cast<const uint4*>(staged + (j * 32 + lane) * 4);
-        const uint32_t lo1 = code & 0x55555555u, hi1 = (code >> 1) & 0x55555555u;
-        const uint32_t n3 = __popc(lo1 & hi1), n2 = __popc(hi1 & ~lo1), n1 = __popc(lo1 & ~hi1);
-        const uint32_t c01 = (16u - n1 - n2 - n3) | (n1 << 16), c23 = n2 | (n3 << 16);     // this lane's elements per slab
-        uint32_t i01 = c01, i23 = c23;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const uint32_t u0 = __shfl_up_sync(0xFFFFFFFFu, i01, o), u1 = __shfl_up_sync(0xFFFFFFFFu, i23, o);
-          if (lane >= o) { i01 += u0; i23 += u1; }
-        }
-        const uint32_t t0 = cnt3 & 1023u, t1 = (cnt3 >> 10) & 1023u, t2 = (cnt3 >> 20) & 1023u;
-        uint32_t a01 = (i01 - c01) + (t0 << 16);                             // next position in the lists of slabs 0 | 1
-        uint32_t a23 = (i23 - c23) + (t0 + t1) + ((t0 + t1 + t2) << 16);     // ... of slabs 2 | 3
-        __syncwarp();
-#pragma unroll
-        for (int j = 0; j < ROWS; ++j) *reinterpret_cast<uint4*>(stage + (j * 32 + lane) * 4) = st[j];
-        __syncwarp();
-#pragma unroll
-        for (int j = 0; j < ROWS; ++j)
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const uint32_t sl = (code >> (2 * (4 * j + e))) & 3u;
-            const uint32_t sh = 16 * (sl & 1);
-            gathered[j].v[e] = stage[((sl < 2 ? a01 : a23) >> sh) & (kSlabWarpTile - 1)];
-            if (sl < 2) a01 += 1u << sh; else a23 += 1u << sh;
-          }
+        unpermute_warp_tile<ROWS>(reinterpret_cast<const uint32_t*>(a.n[S].ptr), slab, wt, stage, gathered);
       }
     }
     uint32_t carry = identity_of<FN, DT>();                // running total of this warp's earlier rows

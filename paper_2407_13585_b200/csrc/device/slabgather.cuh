@@ -1,4 +1,5 @@
-// A scan whose operand gathers from an array that does not fit the L2 cache, run as slab passes.
+// A scan whose operand gathers from an array that does not fit the L2 cache, run as slab passes (and, further down,
+// the same for element-wise roots without a scan).
 //
 // A random 4-byte read of an array much larger than L2 costs a whole DRAM access (about 89 bytes of
 // traffic on B200), and a cluster such as  out = scanl(+) (f (gather idx (g x)))  runs at the rate of
@@ -79,6 +80,32 @@ template <class CL> constexpr bool slab_gather_eligible() {
   return depends_on(c, c.nodes[S].in[0], G) && index_preserving_to(c, c.nodes[S].in[0], G);
 }
 
+// The same passes for a cluster without a scan: element-wise roots over a rank-1 domain, one gather, nothing that
+// accumulates.  The array of the first root that the gather's values reach on index-preserving paths is the staging
+// area, and k_stream_merge takes the place of the merging scan.  -1: no such root.
+template <class CL> constexpr int stream_staging_root() {
+  const int G = the_gather<CL>();
+  if (G < 0) return -1;
+  const CCluster& c = CL::c;
+  for (int i = 0; i < c.n; ++i)
+    if (is_store_root(c.nodes[i]) && c.nodes[i].rank == 1 && depends_on(c, i, G) && index_preserving_to(c, i, G)) return i;
+  return -1;
+}
+template <class CL> constexpr bool slab_stream_eligible() {
+  const int G = the_gather<CL>();
+  if (G < 0 || first_scan<CL>() >= 0 || stream_staging_root<CL>() < 0) return false;
+  const CCluster& c = CL::c;
+  if (c.nodes[G].rank != 1) return false;
+  for (int i = 0; i < c.n; ++i) {
+    const CNode& n = c.nodes[i];
+    if (is_scan_root(n) || is_fold_root(n) || is_permute_root(n) || is_segfold_root(n)) return false;
+    if (is_store_root(n) && (n.rank != 1 || (depends_on(c, i, G) && !index_preserving_to(c, i, G)))) return false;
+  }
+  return true;
+}
+// whose array the staged indices and values live in
+template <class CL> constexpr int slab_staging() { return slab_gather_eligible<CL>() ? first_scan<CL>() : stream_staging_root<CL>(); }
+
 // slab of a source index: the source is cut into kSlabs nearly equal ranges (mul = floor(2^32 * kSlabs / elements))
 __device__ __forceinline__ uint32_t slab_of(uint32_t k, uint32_t mul) { return min(__umulhi(k, mul), (uint32_t)(kSlabs - 1)); }
 
@@ -86,7 +113,7 @@ template <class CL>
 __global__ void __launch_bounds__(kBlock, 4) k_slab_partition(const __grid_constant__ Args<CL::c.n> a, uint32_t* __restrict__ codes,
                                                                uint32_t* __restrict__ counts, int full_tiles, uint32_t mul) {
   constexpr int G = the_gather<CL>();
-  constexpr int S = first_scan<CL>();
+  constexpr int S = slab_staging<CL>();
   constexpr int KEY = CL::c.nodes[G].in[0];
   constexpr int ROWS = kSlabWarpTile / 128;
   __shared__ __align__(16) uint32_t stage[kBlock / 32][kSlabWarpTile];       // read 128 bits at a time
@@ -142,7 +169,7 @@ template <class CL>
 __global__ void __launch_bounds__(kBlock) k_slab_gather(const __grid_constant__ Args<CL::c.n> a, const uint32_t* __restrict__ counts,
                                                          int full_tiles, uint32_t slab) {
   constexpr int G = the_gather<CL>();
-  constexpr int S = first_scan<CL>();
+  constexpr int S = slab_staging<CL>();
   constexpr int SRC = CL::c.nodes[G].in[1];
   constexpr int src_rank = CL::c.nodes[SRC].rank;
   const int lane = threadIdx.x & 31;
@@ -175,6 +202,50 @@ template <class CL, bool STATIC = false>
 __global__ void __launch_bounds__(scan_block<CL>(), 5) k_scan_merge(const __grid_constant__ Args<CL::c.n> a, int tiles_per_row, int n_tiles,
                                                                   const SlabIn slab) {
   scan_tiles<CL, true, true, STATIC>(a, tiles_per_row, n_tiles, slab);
+}
+
+// Every root of a scan-less cluster stored from the gathered values of the earlier launches: a warp puts a warp tile
+// back into element order and evaluates the roots there (the gather member reads as those values).  The staging
+// area is one of the roots' own arrays: a warp has read its whole tile of it before it stores any of it.  Elements
+// beyond the last full warp tile are evaluated as usual by the first block.
+template <class CL>
+__global__ void __launch_bounds__(kBlock, 4) k_stream_merge(const __grid_constant__ Args<CL::c.n> a, const SlabIn slab) {
+  constexpr int N = CL::c.n;
+  constexpr int Z = stream_staging_root<CL>();
+  constexpr int ROWS = kSlabWarpTile / 128;
+  __shared__ __align__(16) uint32_t stage[kBlock / 32][kSlabWarpTile];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int stride = gridDim.x * (kBlock / 32);
+  for (int wt = blockIdx.x * (kBlock / 32) + warp; wt < slab.full_tiles; wt += stride) {
+    V4 gathered[ROWS];
+    unpermute_warp_tile<ROWS>(reinterpret_cast<const uint32_t*>(a.n[Z].ptr), slab, wt, stage[warp], gathered);
+#pragma unroll
+    for (int j = 0; j < ROWS; ++j) {
+      IxGv<Ix4> with;
+      with.r = 0;
+      with.c = wt * kSlabWarpTile + (j * 32 + lane) * 4;
+      with.gv = gathered[j];
+      static_for<0, N>([&](auto ic) {
+        constexpr int i = decltype(ic)::value;
+        if constexpr (is_store_root(CL::c.nodes[i])) {
+          const Ix4& ix = with;
+          uint32_t* out = reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr));
+          if constexpr (depends_on(CL::c, i, the_gather<CL>())) st(out, a.n[i].C, ix, eval<CL, i>(a, with));
+          else st(out, a.n[i].C, ix, eval<CL, i>(a, ix));
+        }
+      });
+    }
+  }
+  if (blockIdx.x == 0) {
+    for (int c = slab.full_tiles * kSlabWarpTile + (int)threadIdx.x; c < a.C; c += kBlock) {
+      const Ix ix{0, c};
+      static_for<0, N>([&](auto ic) {
+        constexpr int i = decltype(ic)::value;
+        if constexpr (is_store_root(CL::c.nodes[i]))
+          st(reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr)), a.n[i].C, ix, eval<CL, i>(a, ix));
+      });
+    }
+  }
 }
 
 template <class CL>

@@ -57,7 +57,8 @@ def test_config3_full():
 
 def test_gather_scan_in_slab_passes_ragged():
     """The slab passes on shapes of their own: a 128 MB source, fewer indices than source elements, a last warp tile
-    of 260 elements (left to the scan's direct gather), under both clusterings that keep the gather with the scan."""
+    of 260 elements (left to the last kernel's direct gather), under both clusterings that keep the gather with the
+    scan, under one that ends the gather's cluster at the masked values, and with every combinator alone."""
     import torch
     from workloads import Node, Program
     from paper_2407_13585_b200 import binding as B
@@ -70,7 +71,9 @@ def test_gather_scan_in_slab_passes_ragged():
     prog = Program("gather_scan_ragged", nodes, [5])
     inputs = {0: W.uniform_int(0, 0, n_src, 1 << 31, device="cuda"), 1: W.uniform_int(0, 1, n, n_src, device="cuda")}
     ref = oracle_run(prog, {k: v.cpu().numpy() for k, v in inputs.items()})
-    for pi, launches in (([-1, -1, 0, 0, 0, 0], 6), ([-1, -1, 0, 1, 1, 1], 7)):
+    # ... and under one that stores the masked values and scans them in a cluster of its own: the element-wise
+    # cluster takes the same passes, with a kernel that only merges and stores in place of the merging scan
+    for pi, launches in (([-1, -1, 0, 0, 0, 0], 6), ([-1, -1, 0, 1, 1, 1], 7), ([-1, -1, 0, 0, 0, 1], 7), ([-1, -1, 0, 1, 2, 3], 9)):
         g = B.Graph(prog.nodes, prog.outputs)
         g.set_partition(pi)
         for i, t in inputs.items():
