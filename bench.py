@@ -509,7 +509,7 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
-    # the kernel that takes the largest share of a step (for config 3 the cluster's six launches count as one:
+    # the kernel that takes the largest share of a step (for config 3 the cluster's seven launches count as one:
     # they are the passes of one gather + scan, and the algorithmic bytes are those of the cluster)
     kernel_bytes = {2: lambda w: w.bytes, 3: lambda w: w.bytes, 4: lambda w: 8 * w.elements, 5: lambda w: w.bytes, 1: lambda w: w.bytes}
     kernel_launches = {2: 1, 3: 1, 4: 4, 5: 1, 1: 1}
@@ -525,7 +525,7 @@ def run_ours(args):
             per[w.cfg]["kernel_algorithmic_gbs"] = gbs
             per[w.cfg]["kernel_frac_of_copy_peak"] = gbs / peak
             per[w.cfg]["kernel_pct_of_8TBs"] = 100.0 * gbs / NOMINAL_HBM_GBS
-    names = {2: "k_tile_pair_tma<transpose+zip+fold>", 3: "k_slab_partition + 4 x k_slab_gather + k_scan_merge_pipelined<hash+gather+mask+scan> (one cluster, six launches)", 4: "k_stencil<jacobi iteration>",
+    names = {2: "k_tile_pair_tma<transpose+zip+fold>", 3: "k_slab_probe + k_slab_partition + 4 x k_slab_gather + k_scan_merge_pipelined<hash+gather+mask+scan> (one cluster, seven launches)", 4: "k_stencil<jacobi iteration>",
              5: "k_hist<hash+generate+permute+fold>", 1: "k_stream<chain>"}
     traffic = NCU_TRAFFIC.get(top) if args.shrink == 0 else None
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,

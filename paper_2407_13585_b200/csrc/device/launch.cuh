@@ -430,12 +430,16 @@ struct Launcher {
           const int warps = dev::kBlock / 32;
           const int pgrid = (int)std::min<int64_t>((full + warps - 1) / warps, (int64_t)sm_count() * 4);
           const int ggrid = (int)std::min<int64_t>((full + warps - 1) / warps, (int64_t)sm_count() * 8);
-          dev::k_slab_partition<CL><<<pgrid, dev::kBlock, 0, L.stream>>>(a, codes, counts, full, mul);
-          for (int k = 0; k < dev::kSlabs; ++k) dev::k_slab_gather<CL><<<ggrid, dev::kBlock, 0, L.stream>>>(a, counts, full, (uint32_t)k);
+          // (word 1 of the scratch, cleared with the tile states: how many sampled warp tiles have local indices)
+          const int probes = (int)std::min<int64_t>((full + warps - 1) / warps, (int64_t)sm_count());
+          const dev::SlabIn slab{codes, counts, full, L.scratch + 1, (uint32_t)(probes * warps)};
+          dev::k_slab_probe<CL><<<probes, dev::kBlock, 0, L.stream>>>(a, full, L.scratch + 1);
+          dev::k_slab_partition<CL><<<pgrid, dev::kBlock, 0, L.stream>>>(a, codes, counts, full, mul, slab);
+          for (int k = 0; k < dev::kSlabs; ++k) dev::k_slab_gather<CL><<<ggrid, dev::kBlock, 0, L.stream>>>(a, counts, full, (uint32_t)k, slab);
           {
-            dev::SlabIn slab{codes, counts, full};
             int per_row_arg = per_row, tiles_arg = (int)tiles;
-            void* params[] = {&a, &per_row_arg, &tiles_arg, &slab};
+            dev::SlabIn slab_arg = slab;
+            void* params[] = {&a, &per_row_arg, &tiles_arg, &slab_arg};
             static int fit_on[64];
             const int resident = resident_grid(reinterpret_cast<const void*>(dev::k_scan_merge_pipelined<CL>), kScanBlock + 32, fit_on);
             if (resident > 0)
@@ -444,7 +448,7 @@ struct Launcher {
             else
               dev::k_scan_merge<CL><<<grid, kScanBlock, 0, L.stream>>>(a, per_row, (int)tiles, slab);
           }
-          L.extra_launches = 1 + dev::kSlabs;
+          L.extra_launches = 2 + dev::kSlabs;
           const cudaError_t e = cudaGetLastError();
           if (e != cudaSuccess) return set_error(ACC_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
           return ACC_OK;
@@ -492,10 +496,13 @@ struct Launcher {
           const int warps = dev::kBlock / 32;
           const int pgrid = (int)std::min<int64_t>((full + warps - 1) / warps, (int64_t)sm_count() * 4);
           const int ggrid = (int)std::min<int64_t>((full + warps - 1) / warps, (int64_t)sm_count() * 8);
-          dev::k_slab_partition<CL><<<pgrid, dev::kBlock, 0, L.stream>>>(a, codes, counts, full, mul);
-          for (int k = 0; k < dev::kSlabs; ++k) dev::k_slab_gather<CL><<<ggrid, dev::kBlock, 0, L.stream>>>(a, counts, full, (uint32_t)k);
-          dev::k_stream_merge<CL><<<pgrid, dev::kBlock, 0, L.stream>>>(a, dev::SlabIn{codes, counts, full});
-          L.extra_launches = 1 + dev::kSlabs;
+          const int probes = (int)std::min<int64_t>((full + warps - 1) / warps, (int64_t)sm_count());
+          const dev::SlabIn slab{codes, counts, full, L.scratch + 1, (uint32_t)(probes * warps)};
+          dev::k_slab_probe<CL><<<probes, dev::kBlock, 0, L.stream>>>(a, full, L.scratch + 1);
+          dev::k_slab_partition<CL><<<pgrid, dev::kBlock, 0, L.stream>>>(a, codes, counts, full, mul, slab);
+          for (int k = 0; k < dev::kSlabs; ++k) dev::k_slab_gather<CL><<<ggrid, dev::kBlock, 0, L.stream>>>(a, counts, full, (uint32_t)k, slab);
+          dev::k_stream_merge<CL><<<pgrid, dev::kBlock, 0, L.stream>>>(a, slab);
+          L.extra_launches = 2 + dev::kSlabs;
           const cudaError_t e = cudaGetLastError();
           if (e != cudaSuccess) return set_error(ACC_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
           return ACC_OK;

@@ -485,7 +485,12 @@ struct SlabIn {
   const uint32_t* codes = nullptr;     // per element of a full warp tile: which slab its gathered index fell in (2 bits; a word per lane)
   const uint32_t* counts = nullptr;    // per full warp tile: how many of its elements fell in slabs 0, 1, 2 (10 bits each)
   int full_tiles = 0;                  // warp tiles of kSlabWarpTile elements that the earlier launches covered
+  const uint32_t* local = nullptr;     // how many of the `sampled` warp tiles that k_slab_probe looked at hold indices close together
+  uint32_t sampled = 0;
 };
+// Whether the probe found the gather's indices local (most sampled warp tiles span few elements of the source): then
+// the gather reads whole sectors and lines as it is, the slab passes stand back and their kernels return at once.
+__device__ __forceinline__ bool slab_passes_stand_back(const SlabIn& slab) { return 2u * __ldg(slab.local) > slab.sampled; }
 constexpr int kSlabWarpTile = 512;
 
 // Whether `leaf` (an array from outside the cluster) is read by member i at i's own index: through array operands

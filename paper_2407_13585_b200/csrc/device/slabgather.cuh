@@ -29,6 +29,7 @@ constexpr int kSlabs = 4;
 constexpr int64_t kSlabMinSourceBytes = 96ll << 20;     // below this the source mostly stays in L2 anyway
 constexpr int64_t kSlabMaxSourceBytes = 320ll << 20;    // beyond this a quarter of it no longer fits
 constexpr int64_t kSlabMinElements = 1ll << 22;
+constexpr uint32_t kSlabLocalSpan = 8192;               // a warp tile whose 512 indices span fewer source elements than this is local
 
 constexpr bool depends_on(const CCluster& c, int i, int g) {
   if (i == g) return true;
@@ -109,9 +110,37 @@ template <class CL> constexpr int slab_staging() { return slab_gather_eligible<C
 // slab of a source index: the source is cut into kSlabs nearly equal ranges (mul = floor(2^32 * kSlabs / elements))
 __device__ __forceinline__ uint32_t slab_of(uint32_t k, uint32_t mul) { return min(__umulhi(k, mul), (uint32_t)(kSlabs - 1)); }
 
+// Looks at one warp tile in every (full_tiles / warps launched): the span of its 512 index values.  Indices that
+// run through the source in order, or stay within a few KB per warp tile, are served well by the plain gather (a
+// monotone index array reads every sector once); random ones are what the passes are for.
+template <class CL>
+__global__ void __launch_bounds__(kBlock) k_slab_probe(const __grid_constant__ Args<CL::c.n> a, int full_tiles, uint32_t* __restrict__ local) {
+  constexpr int G = the_gather<CL>();
+  constexpr int KEY = CL::c.nodes[G].in[0];
+  constexpr int ROWS = kSlabWarpTile / 128;
+  const int lane = threadIdx.x & 31;
+  const int warps = gridDim.x * (kBlock / 32);
+  const int w = blockIdx.x * (kBlock / 32) + ((int)threadIdx.x >> 5);
+  const int wt = (int)(((int64_t)w * full_tiles) / warps);
+  uint32_t lo = 0xFFFFFFFFu, hi = 0u;
+#pragma unroll
+  for (int j = 0; j < ROWS; ++j) {
+    const V4 key = eval<CL, KEY>(a, Ix4{0, wt * kSlabWarpTile + (j * 32 + lane) * 4});
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { lo = min(lo, key.v[e]); hi = max(hi, key.v[e]); }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    lo = min(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, o));
+    hi = max(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, o));
+  }
+  if (lane == 0 && hi - lo < kSlabLocalSpan) atomicAdd(local, 1u);
+}
+
 template <class CL>
 __global__ void __launch_bounds__(kBlock, 4) k_slab_partition(const __grid_constant__ Args<CL::c.n> a, uint32_t* __restrict__ codes,
-                                                               uint32_t* __restrict__ counts, int full_tiles, uint32_t mul) {
+                                                               uint32_t* __restrict__ counts, int full_tiles, uint32_t mul, const SlabIn probe) {
+  if (slab_passes_stand_back(probe)) return;
   constexpr int G = the_gather<CL>();
   constexpr int S = slab_staging<CL>();
   constexpr int KEY = CL::c.nodes[G].in[0];
@@ -167,7 +196,8 @@ __global__ void __launch_bounds__(kBlock, 4) k_slab_partition(const __grid_const
 
 template <class CL>
 __global__ void __launch_bounds__(kBlock) k_slab_gather(const __grid_constant__ Args<CL::c.n> a, const uint32_t* __restrict__ counts,
-                                                         int full_tiles, uint32_t slab) {
+                                                         int full_tiles, uint32_t slab, const SlabIn probe) {
+  if (slab_passes_stand_back(probe)) return;
   constexpr int G = the_gather<CL>();
   constexpr int S = slab_staging<CL>();
   constexpr int SRC = CL::c.nodes[G].in[1];
@@ -200,7 +230,9 @@ __global__ void __launch_bounds__(kBlock) k_slab_gather(const __grid_constant__ 
 // (five blocks per SM: the merge is issue bound, and a quarter more warps pay for a few spilled words)
 template <class CL, bool STATIC = false>
 __global__ void __launch_bounds__(scan_block<CL>(), 5) k_scan_merge(const __grid_constant__ Args<CL::c.n> a, int tiles_per_row, int n_tiles,
-                                                                  const SlabIn slab) {
+                                                                  const SlabIn slab_in) {
+  SlabIn slab = slab_in;
+  if (slab_passes_stand_back(slab)) slab.full_tiles = 0;     // every warp tile gathers for itself
   scan_tiles<CL, true, true, STATIC>(a, tiles_per_row, n_tiles, slab);
 }
 
@@ -216,24 +248,39 @@ __global__ void __launch_bounds__(kBlock, 4) k_stream_merge(const __grid_constan
   __shared__ __align__(16) uint32_t stage[kBlock / 32][kSlabWarpTile];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int stride = gridDim.x * (kBlock / 32);
-  for (int wt = blockIdx.x * (kBlock / 32) + warp; wt < slab.full_tiles; wt += stride) {
-    V4 gathered[ROWS];
-    unpermute_warp_tile<ROWS>(reinterpret_cast<const uint32_t*>(a.n[Z].ptr), slab, wt, stage[warp], gathered);
+  if (slab_passes_stand_back(slab)) {
+    // nothing was staged: every warp tile is evaluated as it stands
+    for (int wt = blockIdx.x * (kBlock / 32) + warp; wt < slab.full_tiles; wt += stride) {
 #pragma unroll
-    for (int j = 0; j < ROWS; ++j) {
-      IxGv<Ix4> with;
-      with.r = 0;
-      with.c = wt * kSlabWarpTile + (j * 32 + lane) * 4;
-      with.gv = gathered[j];
-      static_for<0, N>([&](auto ic) {
-        constexpr int i = decltype(ic)::value;
-        if constexpr (is_store_root(CL::c.nodes[i])) {
-          const Ix4& ix = with;
-          uint32_t* out = reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr));
-          if constexpr (depends_on(CL::c, i, the_gather<CL>())) st(out, a.n[i].C, ix, eval<CL, i>(a, with));
-          else st(out, a.n[i].C, ix, eval<CL, i>(a, ix));
-        }
-      });
+      for (int j = 0; j < ROWS; ++j) {
+        const Ix4 ix{0, wt * kSlabWarpTile + (j * 32 + lane) * 4};
+        static_for<0, N>([&](auto ic) {
+          constexpr int i = decltype(ic)::value;
+          if constexpr (is_store_root(CL::c.nodes[i]))
+            st(reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr)), a.n[i].C, ix, eval<CL, i>(a, ix));
+        });
+      }
+    }
+  } else {
+    for (int wt = blockIdx.x * (kBlock / 32) + warp; wt < slab.full_tiles; wt += stride) {
+      V4 gathered[ROWS];
+      unpermute_warp_tile<ROWS>(reinterpret_cast<const uint32_t*>(a.n[Z].ptr), slab, wt, stage[warp], gathered);
+#pragma unroll
+      for (int j = 0; j < ROWS; ++j) {
+        IxGv<Ix4> with;
+        with.r = 0;
+        with.c = wt * kSlabWarpTile + (j * 32 + lane) * 4;
+        with.gv = gathered[j];
+        static_for<0, N>([&](auto ic) {
+          constexpr int i = decltype(ic)::value;
+          if constexpr (is_store_root(CL::c.nodes[i])) {
+            const Ix4& ix = with;
+            uint32_t* out = reinterpret_cast<uint32_t*>(const_cast<void*>(a.n[i].ptr));
+            if constexpr (depends_on(CL::c, i, the_gather<CL>())) st(out, a.n[i].C, ix, eval<CL, i>(a, with));
+            else st(out, a.n[i].C, ix, eval<CL, i>(a, ix));
+          }
+        });
+      }
     }
   }
   if (blockIdx.x == 0) {
@@ -250,7 +297,9 @@ __global__ void __launch_bounds__(kBlock, 4) k_stream_merge(const __grid_constan
 
 template <class CL>
 __global__ void __launch_bounds__(scan_block<CL>() + 32, 5) k_scan_merge_pipelined(const __grid_constant__ Args<CL::c.n> a, int tiles_per_row, int n_tiles,
-                                                                                  const SlabIn slab) {
+                                                                                  const SlabIn slab_in) {
+  SlabIn slab = slab_in;
+  if (slab_passes_stand_back(slab)) slab.full_tiles = 0;     // every warp tile gathers for itself
   scan_tiles_pipelined<CL, true, true>(a, tiles_per_row, n_tiles, slab);
 }
 

@@ -49,8 +49,9 @@ def test_config3_full():
     prog = W.config3(1 << 26)
     got, inputs, pi, g = run_full(prog, "enumerate")
     # one cluster; its gather reads a 256 MB source, twice the L2, so it runs as slab passes: the indices are
-    # partitioned once, four launches gather a quarter of the source each, and the scan merges (six launches)
-    assert pi == [-1, -1, 0, 0, 0, 0] and g.launch_count() == 6
+    # probed (random or local?), partitioned once, four launches gather a quarter of the source each, and the scan
+    # merges (seven launches)
+    assert pi == [-1, -1, 0, 0, 0, 0] and g.launch_count() == 7
     ref = oracle_run(prog, {k: v.cpu().numpy() for k, v in inputs.items()})
     compare(prog, ref, got, "config3 full")
 
@@ -73,7 +74,7 @@ def test_gather_scan_in_slab_passes_ragged():
     ref = oracle_run(prog, {k: v.cpu().numpy() for k, v in inputs.items()})
     # ... and under one that stores the masked values and scans them in a cluster of its own: the element-wise
     # cluster takes the same passes, with a kernel that only merges and stores in place of the merging scan
-    for pi, launches in (([-1, -1, 0, 0, 0, 0], 6), ([-1, -1, 0, 1, 1, 1], 7), ([-1, -1, 0, 0, 0, 1], 7), ([-1, -1, 0, 1, 2, 3], 9)):
+    for pi, launches in (([-1, -1, 0, 0, 0, 0], 7), ([-1, -1, 0, 1, 1, 1], 8), ([-1, -1, 0, 0, 0, 1], 8), ([-1, -1, 0, 1, 2, 3], 10)):
         g = B.Graph(prog.nodes, prog.outputs)
         g.set_partition(pi)
         for i, t in inputs.items():
@@ -86,6 +87,38 @@ def test_gather_scan_in_slab_passes_ragged():
         assert g.launch_count() == launches, (pi, g.launch_count())
         got = {5: out.cpu().numpy().view(np.uint32)}
         compare(prog, ref, got, "gather + scan in slab passes, pi=%s" % pi)
+
+
+def test_slab_passes_stand_back_for_local_indices():
+    """Indices that run through a 128 MB source in order (steps of 0..3 elements) are served by the plain gather: the
+    probe finds every sampled warp tile local, the partition and the four gather launches return at once, and the
+    last kernel gathers for itself.  Same launches, same results as the oracle, with the scan in the gather's cluster
+    and without; a source that is read at random between two runs of the same graph takes the passes again."""
+    import torch
+    from workloads import Node, Program
+    from paper_2407_13585_b200 import binding as B
+    n_src, n = 1 << 25, (1 << 22) + 516
+    nodes = [Node("input", "i32", (n_src,), name="x"), Node("input", "i32", (n,), name="idx"),
+             Node("gather", "i32", (n,), (1, 0), 2, name="h"),
+             Node("map", "i32", (n,), (2,), 1, fn="and_mask", iparam=(0xFFFF,), name="o"),
+             Node("scanl", "i32", (n,), (3,), 1, fn="add", name="out")]
+    prog = Program("gather_scan_local", nodes, [4])
+    x = W.uniform_int(0, 0, n_src, 1 << 31, device="cuda")
+    steps = W.uniform_int(0, 1, n, 4, device="cuda")
+    local = torch.cumsum(steps, 0, dtype=torch.int64).to(torch.int32)              # below 3 * n < n_src
+    scattered = W.uniform_int(0, 2, n, n_src, device="cuda")
+    for pi, launches in (([-1, -1, 0, 0, 0], 7), ([-1, -1, 0, 0, 1], 8)):
+        g = B.Graph(prog.nodes, prog.outputs)
+        g.set_partition(pi)
+        g.bind(0, x)
+        out = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+        g.bind(4, out)
+        for idx, what in ((local, "local"), (scattered, "scattered"), (local, "local again")):
+            g.bind(1, idx)
+            ref = oracle_run(prog, {0: x.cpu().numpy(), 1: idx.cpu().numpy()})
+            g.run(B.FUSED)
+            assert g.launch_count() == launches, (pi, g.launch_count())
+            compare(prog, ref, {4: out.cpu().numpy().view(np.uint32)}, "gather + scan, %s indices, pi=%s" % (what, pi))
 
 
 def test_gathering_scans_over_several_rounds_of_a_resident_grid():
