@@ -89,6 +89,28 @@ def test_gather_scan_in_slab_passes_ragged():
         compare(prog, ref, got, "gather + scan in slab passes, pi=%s" % pi)
 
 
+def test_slab_passes_with_several_element_wise_roots():
+    """A cluster without a scan in slab passes, with three arrays to store: the gathered values themselves (their array
+    is the staging area), a map of them, and a map of the indices that does not touch the gather."""
+    import torch
+    from paper_2407_13585_b200 import binding as B
+    n = (1 << 22) + 260
+    prog = W.gather_three_roots(1 << 25, n)
+    inputs = W.make_inputs(prog, device="cuda")
+    ref = oracle_run(prog, {k: v.cpu().numpy() for k, v in inputs.items()})
+    g = B.Graph(prog.nodes, prog.outputs)
+    g.set_partition([-1, -1, 0, 0, 0])
+    for i, t in inputs.items():
+        g.bind(i, t)
+    outs = {o: torch.full((n,), -1, dtype=torch.int32, device="cuda") for o in prog.outputs}
+    for o, t in outs.items():
+        g.bind(o, t)
+    g.run(B.FUSED)
+    g.run(B.FUSED)
+    assert g.launch_count() == 7
+    compare(prog, ref, {o: t.cpu().numpy().view(np.uint32) for o, t in outs.items()}, "gather with three roots in slab passes")
+
+
 def test_slab_passes_stand_back_for_local_indices():
     """Indices that run through a 128 MB source in order (steps of 0..3 elements) are served by the plain gather: the
     probe finds every sampled warp tile local, the partition and the four gather launches return at once, and the

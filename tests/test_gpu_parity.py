@@ -53,6 +53,12 @@ def test_config3_all_partitions(n):
     assert check_program(W.config3(n)) == 8
 
 
+# one gather stored with a map of it and a map of its indices beside it: lengths the 128-bit paths take and not
+@pytest.mark.parametrize("n", [1, 1000, 4099, 1 << 16])
+def test_gather_with_three_roots_all_partitions(n):
+    assert check_program(W.gather_three_roots(5000, n)) == 4
+
+
 def test_config3_ragged_lengths():
     # lengths that are not powers of two: the scan's last tile is partial, the scalar path runs
     for n in (5, 4097, 12289 + 3):

@@ -378,7 +378,7 @@ def test_generated_sources_match_their_programs():
     from paper_2407_13585_b200 import instantiate
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     here = os.path.join(root, "paper_2407_13585_b200", "csrc", "programs")
-    files = sorted(glob.glob(os.path.join(root, "tests", "programs", "prog_random*.cu")) + glob.glob(os.path.join(here, "prog_scan_consumers*.cu")) +
+    files = sorted(glob.glob(os.path.join(root, "tests", "programs", "prog_random*.cu")) + glob.glob(os.path.join(root, "tests", "programs", "prog_gather*.cu")) + glob.glob(os.path.join(here, "prog_scan_consumers*.cu")) +
                    glob.glob(os.path.join(here, "prog_histogram_2d.cu")))
     assert len(files) >= 18
     for f in files:

@@ -405,6 +405,19 @@ def offsets_then_gather(n=1 << 12):
     return Program("offsets_then_gather", nodes, [5, 6], index_bound={"x": 1 << 30, "src": 1 << 30})
 
 
+def gather_three_roots(n_src=1 << 12, n=1 << 10):
+    """One gather with three arrays to store: h = src[idx]; m = h & 0xFFFF; r = idx & 0xFF (which does not touch the
+    gather)."""
+    nodes = [
+        _inp("x", "i32", (n_src,)),
+        _inp("idx", "i32", (n,)),
+        Node("gather", "i32", (n,), (1, 0), 2, name="h"),
+        Node("map", "i32", (n,), (2,), 1, fn="and_mask", iparam=(0xFFFF,), name="m"),
+        Node("map", "i32", (n,), (1,), 1, fn="and_mask", iparam=(0xFF,), name="r"),
+    ]
+    return Program("gather_three_roots", nodes, [2, 3, 4], index_bound={"idx": n_src, "x": 1 << 30})
+
+
 def histogram_2d(rows=64, n=4096, bins=256):
     """The scatter histogram of config 5 over a rank-2 array of keys, with per-row totals beside it: the
     scatter and the row folds share producers but no kernel walk."""
